@@ -1,0 +1,283 @@
+"""CPU oracle for the forward pass of an FFN restructured into a sparse MoE.
+
+TEST INFRASTRUCTURE ONLY.  Plain numpy in fp64, written from the paper's
+equations, sharing no code with the CUDA path; only tests, the smoke check and
+the benchmark's CPU-baseline leg may call it.  Inputs are whatever fp32 arrays
+the caller hands in (for bf16 workloads: values already rounded to bf16);
+every product and sum here is fp64.
+
+Array conventions (the same as the C-ABI's): ``w_gate[n, :]`` and
+``w_up[n, :]`` are neuron n's gate/up vectors (column n of the paper's
+W_gate/W_up in R^{d x d_h}); ``w_down[:, n]`` is neuron n's output vector
+(row n of the paper's W_down in R^{d_h x d}).  ``neuron_perm`` lists original
+neuron indices; expert e owns ``neuron_perm[e*m:(e+1)*m]`` and experts
+``0..N_s-1`` are the shared ones (Section 4.1).
+
+Pins (tests/test_oracle_pins.py): all-experts-on = dense FFN (Eq. decompose),
+the reconstruction-error identity (Eq. recon_error), router score = dense
+hidden activation of the representative neuron (Eq. rep_neuron/router),
+closed forms of the gate (Section 4.3), brute-force top-k, scalar per-neuron
+brute force, a library fp64 SwiGLU, permutation invariants, and hierarchical
+all-on = the original MoE layer (Section 4.4).
+Parity unpinned (conventions the paper does not fix): the outer router's
+weights for an existing MoE layer (softmax over the selected logits), the
+tie-break between equal keys (lower index wins) and the NaN policy.
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+F64 = np.float64
+
+
+def _f64(a) -> np.ndarray:
+    return np.asarray(a, dtype=F64)
+
+
+# ---------------------------------------------------------------- Section 4.1
+def swish(a: np.ndarray) -> np.ndarray:
+    """Swish with beta = 1 (SiLU): a * sigmoid(a)  (Eq. ori_ffn_method)."""
+    a = _f64(a)
+    return a / (1.0 + np.exp(-a))
+
+
+def hidden_activations(x, w_gate, w_up, neurons=None) -> np.ndarray:
+    """h = Swish(W_gate^T x) * (W_up^T x) for the listed neurons, all tokens
+    (Eq. ori_ffn_method, first line).  x: [T,d] -> [T,len(neurons)]."""
+    x = _f64(x)
+    if neurons is None:
+        wg, wu = _f64(w_gate), _f64(w_up)
+    else:
+        neurons = np.asarray(neurons, dtype=np.int64)
+        wg, wu = _f64(w_gate[neurons]), _f64(w_up[neurons])
+    return swish(x @ wg.T) * (x @ wu.T)
+
+
+def dense_ffn(x, w_gate, w_up, w_down) -> np.ndarray:
+    """F(x) = W_down^T h (Eq. ori_ffn_method)."""
+    return hidden_activations(x, w_gate, w_up) @ _f64(w_down).T
+
+
+def expert_forward(x, w_gate, w_up, w_down, neurons) -> np.ndarray:
+    """An expert is the FFN restricted to its neurons: E(x) = sum over its
+    neurons of h_i w_i (Eq. decompose with the slice of Section 4.1)."""
+    neurons = np.asarray(neurons, dtype=np.int64)
+    h = hidden_activations(x, w_gate, w_up, neurons)
+    return h @ _f64(w_down[:, neurons]).T
+
+
+def expert_neurons(neuron_perm, n_experts: int, e: int) -> np.ndarray:
+    d_ff = len(neuron_perm)
+    if d_ff % n_experts:
+        raise ValueError("d_ff must be a multiple of the number of experts")
+    m = d_ff // n_experts
+    return np.asarray(neuron_perm[e * m:(e + 1) * m], dtype=np.int64)
+
+
+# ---------------------------------------------------------------- Section 4.2
+def router_scores(x, w_gate, w_up, rep_idx) -> np.ndarray:
+    """s = G(x) = Swish(W_gate^{R T} x) * (W_up^{R T} x) (Eq. router): the
+    SwiGLU activation of each routed expert's representative neuron."""
+    return hidden_activations(x, w_gate, w_up, np.asarray(rep_idx, dtype=np.int64))
+
+
+# ---------------------------------------------------------------- Section 4.3
+def softmax(s: np.ndarray) -> np.ndarray:
+    s = _f64(s)
+    z = np.exp(s - s.max(axis=-1, keepdims=True))
+    return z / z.sum(axis=-1, keepdims=True)
+
+
+def gate_logic(s, top_k: int, gate_scale_u=None, select_bias_b=None):
+    """Eq. final_gate.  s' = Softmax(s) over all N_r scores; expert i is
+    selected iff s'_i + b_i is among the N_k largest keys; a selected expert's
+    gate is 1 + s'_i u_i (the bias takes no part in the gate value).
+    Equal keys: the lower index wins.  NaN keys rank below everything.
+
+    Returns (sel_idx [T,N_k] int32 in descending-key order, gates [T,N_k],
+    s_prime [T,N_r], keys [T,N_r])."""
+    s = _f64(s)
+    n_tok, n_r = s.shape
+    if not 0 <= top_k <= n_r:
+        raise ValueError("top_k must lie in [0, N_r]")
+    u = np.zeros(n_r) if gate_scale_u is None else _f64(gate_scale_u)
+    b = np.zeros(n_r) if select_bias_b is None else _f64(select_bias_b)
+    s_prime = softmax(s)
+    keys = s_prime + b
+    rank_keys = np.where(np.isnan(keys), -np.inf, keys)
+    order = np.argsort(-rank_keys, axis=1, kind="stable")   # full sort of all N_r keys
+    sel_idx = order[:, :top_k].astype(np.int32)
+    gates = 1.0 + np.take_along_axis(s_prime, sel_idx.astype(np.int64), axis=1) * u[sel_idx]
+    return sel_idx, gates, s_prime, keys
+
+
+def logit_margin(s_prime, keys, top_k: int) -> np.ndarray:
+    """Per token: gap between the N_k-th and (N_k+1)-th key, expressed in logit
+    (pre-softmax) units: (key_p - key_q) / max(s'_p, s'_q).  With b = 0 this is
+    1 - exp(-(s_p - s_q)) ~ s_p - s_q.  +inf when no (N_k+1)-th key exists."""
+    keys = _f64(keys)
+    n_tok, n_r = keys.shape
+    if top_k == 0 or top_k >= n_r:
+        return np.full(n_tok, np.inf)
+    order = np.argsort(-keys, axis=1, kind="stable")
+    p, q = order[:, top_k - 1], order[:, top_k]
+    rows = np.arange(n_tok)
+    gap = keys[rows, p] - keys[rows, q]
+    return gap / np.maximum(s_prime[rows, p], s_prime[rows, q])
+
+
+# ------------------------------------------------------- Eq. moe_output
+def moe_forward(x, w_gate, w_up, w_down, neuron_perm, n_experts: int, n_shared: int,
+                sel_idx, gates, token_ids=None) -> np.ndarray:
+    """F_MoE(x) = E^s(x) + sum_i g_i E_i^r(x) (Eq. moe_output) with the gate
+    values given; terms with g_i = 0 (unselected experts) are skipped.  The
+    N_s shared experts form one always-on expert.  Routed experts are added in
+    ascending expert index.  ``token_ids`` restricts the evaluation to a
+    subset of tokens (used to sample outputs of large workloads)."""
+    x = _f64(x)
+    sel_idx = np.asarray(sel_idx)
+    gates = _f64(gates)
+    if token_ids is not None:
+        token_ids = np.asarray(token_ids, dtype=np.int64)
+        x, sel_idx, gates = x[token_ids], sel_idx[token_ids], gates[token_ids]
+    n_r = n_experts - n_shared
+    m = len(neuron_perm) // n_experts
+    out = np.zeros_like(x)
+    if n_shared > 0:
+        shared = np.asarray(neuron_perm[:n_shared * m], dtype=np.int64)
+        out += expert_forward(x, w_gate, w_up, w_down, shared)
+    for j in range(n_r):
+        hit_tok, hit_slot = np.nonzero(sel_idx == j)
+        if hit_tok.size == 0:
+            continue
+        neurons = expert_neurons(neuron_perm, n_experts, n_shared + j)
+        y = expert_forward(x[hit_tok], w_gate, w_up, w_down, neurons)
+        out[hit_tok] += gates[hit_tok, hit_slot][:, None] * y
+    return out
+
+
+def cmoe_layer_forward(x, w_gate, w_up, w_down, neuron_perm, rep_idx, n_experts: int,
+                       n_shared: int, top_k: int, gate_scale_u=None, select_bias_b=None):
+    """Router (Eq. router) -> gates (Eq. final_gate) -> experts and combine
+    (Eq. moe_output).  Returns (out, sel_idx, gates, s, s_prime, keys)."""
+    s = router_scores(x, w_gate, w_up, rep_idx)
+    sel_idx, gates, s_prime, keys = gate_logic(s, top_k, gate_scale_u, select_bias_b)
+    out = moe_forward(x, w_gate, w_up, w_down, neuron_perm, n_experts, n_shared,
+                      sel_idx, gates)
+    return out, sel_idx, gates, s, s_prime, keys
+
+
+# ------------------------------------------- token histogram and permutation
+def token_permutation(sel_idx, n_groups: int):
+    """Expert-contiguous order of the selected (token, expert) pairs.  The
+    paper only says that the top-N_k experts are activated; this is the one
+    canonical way to list the pairs: sorted by (expert, token).
+
+    cnt[e]      = number of tokens that selected e
+    off         = exclusive prefix sum of cnt (length n_groups + 1)
+    row_token[r]= token at row r;  rows off[e]..off[e+1]-1 belong to expert e,
+                  tokens ascending
+    row_of[t,j] = row holding the pair (t, sel_idx[t, j])
+    """
+    sel_idx = np.asarray(sel_idx)
+    n_tok, n_k = sel_idx.shape
+    cnt = np.zeros(n_groups, dtype=np.int32)
+    for t in range(n_tok):
+        for j in range(n_k):
+            cnt[sel_idx[t, j]] += 1
+    off = np.zeros(n_groups + 1, dtype=np.int32)
+    for e in range(n_groups):
+        off[e + 1] = off[e] + cnt[e]
+    fill = off[:-1].copy()
+    row_token = np.full(n_tok * n_k, -1, dtype=np.int32)
+    row_of = np.full((n_tok, n_k), -1, dtype=np.int32)
+    for t in range(n_tok):                      # ascending token => stable
+        for j in range(n_k):
+            e = sel_idx[t, j]
+            r = fill[e]
+            fill[e] += 1
+            row_token[r] = t
+            row_of[t, j] = r
+    return cnt, off, row_token, row_of
+
+
+# ---------------------------------------------------------------- Section 4.4
+def outer_router(x, w_router, outer_top_k: int):
+    """Top-level router of an existing MoE layer: logits l = W_r x, the
+    outer_top_k largest logits are selected (ties: lower index), weights =
+    softmax over the selected logits.  (The paper only says that the top-level
+    router selects primary experts; this is the Mixtral-style convention.)"""
+    logits = _f64(x) @ _f64(w_router).T
+    order = np.argsort(-np.where(np.isnan(logits), -np.inf, logits), axis=1, kind="stable")
+    outer_idx = order[:, :outer_top_k].astype(np.int32)
+    sel_logits = np.take_along_axis(logits, outer_idx.astype(np.int64), axis=1)
+    outer_w = softmax(sel_logits)
+    return outer_idx, outer_w, logits
+
+
+def hier_forward(x, w_router, outer_top_k: int, layers: Sequence[dict], token_ids=None):
+    """Section 4.4: every expert E_i of an existing MoE layer is replaced by
+    E_i^s + sum_j g'_{i,j} E^r_{i,j}; the output is sum over the selected
+    outer experts of w_i times that.  ``layers[i]`` holds the keyword
+    arguments of cmoe_layer_forward for outer expert i.
+    Returns (out, outer_idx, outer_w, per-expert routing list)."""
+    x = _f64(x)
+    outer_idx, outer_w, _ = outer_router(x, w_router, outer_top_k)
+    keep = np.arange(x.shape[0]) if token_ids is None else np.asarray(token_ids, dtype=np.int64)
+    out = np.zeros((len(keep), x.shape[1]))
+    routing = []
+    for i, layer in enumerate(layers):
+        tok, slot = np.nonzero(outer_idx == i)          # tok ascending
+        routing.append(None)
+        if tok.size == 0:
+            continue
+        s = router_scores(x[tok], layer["w_gate"], layer["w_up"], layer["rep_idx"])
+        sel_idx, gates, s_prime, keys = gate_logic(
+            s, layer["top_k"], layer.get("gate_scale_u"), layer.get("select_bias_b"))
+        routing[i] = dict(tokens=tok, sel_idx=sel_idx, gates=gates, s=s,
+                          s_prime=s_prime, keys=keys)
+        in_keep = np.isin(tok, keep)
+        if not in_keep.any():
+            continue
+        sub = np.nonzero(in_keep)[0]
+        y = moe_forward(x[tok], layer["w_gate"], layer["w_up"], layer["w_down"],
+                        layer["neuron_perm"], layer["n_experts"], layer["n_shared"],
+                        sel_idx, gates, token_ids=sub)
+        dst = np.searchsorted(keep, tok[sub])
+        out[dst] += outer_w[tok[sub], slot[sub]][:, None] * y
+    return out, outer_idx, outer_w, routing
+
+
+# ---------------------------------------------------------------- Section 4.3
+def bias_update(select_bias_b, counts, target_share=None, gamma: float = 1e-3):
+    """One step of the load-balancing rule: with p_i the fraction of routed
+    assignments that went to expert i and p* the target (uniform 1/N_r in the
+    paper), b_i decreases by gamma if p_i > p*, increases by gamma if p_i < p*."""
+    b = _f64(select_bias_b).copy()
+    counts = _f64(counts)
+    p = counts / counts.sum()
+    target = np.full_like(p, 1.0 / len(p)) if target_share is None else _f64(target_share)
+    b[p > target] -= gamma
+    b[p < target] += gamma
+    return b
+
+
+def fit_select_bias(s, top_k: int, target_share, iters: int = 4000,
+                    gamma_hi: float = 2e-2, gamma_lo: float = 1e-4, tol: float = 3e-3):
+    """Iterate bias_update on fixed router scores with a geometrically decaying
+    step until every expert's share is within ``tol`` of its target.  Produces
+    the selection bias of the skewed-load workload (an input to both sides)."""
+    s_prime = softmax(s)
+    n_tok, n_r = s_prime.shape
+    b = np.zeros(n_r)
+    target = _f64(target_share)
+    for it in range(iters):
+        order = np.argsort(-(s_prime + b), axis=1, kind="stable")[:, :top_k]
+        counts = np.bincount(order.ravel(), minlength=n_r)
+        if np.abs(counts / counts.sum() - target).max() <= tol:
+            break
+        gamma = gamma_hi * (gamma_lo / gamma_hi) ** (it / max(iters - 1, 1))
+        b = bias_update(b, counts, target, gamma)
+    return b, counts

@@ -1,0 +1,389 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix.
+
+Each ``pin_*`` takes the oracle module so that ``test_planted_mistakes_are_caught``
+can run the same pins against deliberately broken copies of it.
+"""
+import importlib.util
+import math
+import os
+import types
+
+import numpy as np
+import pytest
+
+from oracle import cmoe_oracle as oracle
+from paper_2502_04416_b200 import workloads as wl
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def small_layer(seed=0, d=24, n_experts=8, m=6, n_shared=2, top_k=2, n_tok=37, dtype="fp32"):
+    shape = wl.LayerShape(d, n_experts * m, n_experts, n_shared, top_k, dtype)
+    rng = np.random.Generator(np.random.PCG64(seed))
+    x = wl.draw_tokens(rng, n_tok, shape)
+    lay = wl.draw_layer(rng, shape)
+    # larger weights than the workloads' 0.02 so that scores are well spread
+    lay.w_gate *= 12.0
+    lay.w_up *= 12.0
+    return shape, x, lay
+
+
+def layer_kwargs(shape, lay, **over):
+    kw = dict(w_gate=lay.w_gate, w_up=lay.w_up, w_down=lay.w_down,
+              neuron_perm=lay.neuron_perm, rep_idx=lay.rep_idx,
+              n_experts=shape.n_experts, n_shared=shape.n_shared, top_k=shape.top_k,
+              gate_scale_u=lay.gate_scale_u, select_bias_b=lay.select_bias_b)
+    kw.update(over)
+    return kw
+
+
+# ------------------------------------------------------------------ dense FFN
+def pin_dense_closed_form(o):
+    """Eq. ori_ffn_method on numbers worked by hand: gate pre-activation ln 3
+    gives sigmoid 3/4; pre-activation 0 gives a dead neuron."""
+    ln3 = math.log(3.0)
+    x = np.array([[1.0, 0.0], [0.0, 1.0]])
+    w_gate = np.array([[ln3, 0.0], [0.0, -ln3], [0.0, 0.0]])      # [d_h=3, d=2]
+    w_up = np.array([[2.0, 5.0], [7.0, 4.0], [9.0, 9.0]])
+    w_down = np.array([[1.0, 10.0, 100.0], [-1.0, 0.5, 100.0]])   # [d=2, d_h=3]
+    # token 0: a = (ln3, 0, 0), v = (2, 7, 9): h = (ln3*3/4*2, 0, 0)
+    # token 1: a = (0, -ln3, 0), v = (5, 4, 9): h = (0, -ln3*1/4*4, 0)
+    want = np.array([[1.5 * ln3, -1.5 * ln3], [-10.0 * ln3, -0.5 * ln3]])
+    got = o.dense_ffn(x, w_gate, w_up, w_down)
+    np.testing.assert_allclose(got, want, rtol=1e-14, atol=1e-14)
+
+
+def pin_dense_library(o):
+    """Same FFN through a library SwiGLU in fp64 (torch)."""
+    import torch
+    import torch.nn.functional as F
+    shape, x, lay = small_layer(seed=11, d=40, m=9)
+    tx, tg, tu, td = (torch.from_numpy(np.asarray(a, dtype=np.float64))
+                      for a in (x, lay.w_gate, lay.w_up, lay.w_down))
+    want = F.linear(F.silu(F.linear(tx, tg)) * F.linear(tx, tu), td).numpy()
+    got = o.dense_ffn(x, lay.w_gate, lay.w_up, lay.w_down)
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-13)
+
+
+def pin_dense_per_neuron_brute_force(o):
+    """Eq. decompose: F(x) = sum_i h_i w_i, one neuron at a time, scalar loops."""
+    shape, x, lay = small_layer(seed=5, d=5, n_experts=2, m=3, n_shared=1, top_k=1, n_tok=3)
+    d, d_h = shape.d_model, shape.d_ff
+    got = o.dense_ffn(x, lay.w_gate, lay.w_up, lay.w_down)
+    for t in range(x.shape[0]):
+        y = [0.0] * d
+        for i in range(d_h):
+            a = sum(float(lay.w_gate[i, k]) * float(x[t, k]) for k in range(d))
+            v = sum(float(lay.w_up[i, k]) * float(x[t, k]) for k in range(d))
+            h = a / (1.0 + math.exp(-a)) * v
+            for c in range(d):
+                y[c] += h * float(lay.w_down[c, i])
+        np.testing.assert_allclose(got[t], y, rtol=1e-12, atol=1e-14)
+
+
+# ------------------------------------------------------------- MoE invariants
+def pin_all_experts_on_is_dense(o):
+    """Experts partition the neurons, so every routed expert on with unit gates
+    reproduces the dense FFN (Eq. decompose / Section 3.3)."""
+    shape, x, lay = small_layer(seed=1)
+    out, sel, gates, *_ = o.cmoe_layer_forward(x, **layer_kwargs(shape, lay, top_k=shape.n_routed))
+    assert np.all(gates == 1.0)
+    assert np.all(np.sort(sel, axis=1) == np.arange(shape.n_routed))
+    want = o.dense_ffn(x, lay.w_gate, lay.w_up, lay.w_down)
+    np.testing.assert_allclose(out, want, rtol=1e-11, atol=1e-13)
+
+
+def pin_reconstruction_error_identity(o):
+    """Eq. recon_error: F_MoE - F = - sum over deactivated routed experts."""
+    shape, x, lay = small_layer(seed=2)
+    out, sel, gates, *_ = o.cmoe_layer_forward(x, **layer_kwargs(shape, lay))
+    dense = o.dense_ffn(x, lay.w_gate, lay.w_up, lay.w_down)
+    missing = np.zeros_like(dense)
+    for j in range(shape.n_routed):
+        off = ~np.any(sel == j, axis=1)
+        neurons = o.expert_neurons(lay.neuron_perm, shape.n_experts, shape.n_shared + j)
+        missing[off] += o.expert_forward(x[off], lay.w_gate, lay.w_up, lay.w_down, neurons)
+    assert np.abs(missing).max() > 1e-3          # the identity is not vacuous
+    np.testing.assert_allclose(out - dense, -missing, rtol=1e-9, atol=1e-12)
+
+
+def pin_shared_always_on(o):
+    """N_k = 0 leaves exactly the shared expert, for every token."""
+    shape, x, lay = small_layer(seed=3)
+    out, sel, gates, *_ = o.cmoe_layer_forward(x, **layer_kwargs(shape, lay, top_k=0))
+    assert sel.shape == (x.shape[0], 0)
+    shared = lay.neuron_perm[:shape.n_shared * shape.m]
+    want = o.hidden_activations(x, lay.w_gate, lay.w_up, shared) @ \
+        np.asarray(lay.w_down[:, shared], dtype=np.float64).T
+    np.testing.assert_allclose(out, want, rtol=1e-12, atol=1e-14)
+    assert np.all(np.abs(out).max(axis=1) > 0)
+
+
+def pin_router_is_representative_activation(o):
+    """s_j = h_{R_j}: the score is column R_j of the dense hidden state."""
+    shape, x, lay = small_layer(seed=4)
+    s = o.router_scores(x, lay.w_gate, lay.w_up, lay.rep_idx)
+    h = o.hidden_activations(x, lay.w_gate, lay.w_up)
+    np.testing.assert_allclose(s, h[:, lay.rep_idx], rtol=1e-12, atol=1e-15)
+    # each representative lies in its own routed slice
+    for j, r in enumerate(lay.rep_idx):
+        assert r in o.expert_neurons(lay.neuron_perm, shape.n_experts, shape.n_shared + j)
+
+
+def pin_gate_closed_forms(o):
+    rng = np.random.default_rng(7)
+    s = rng.normal(size=(50, 6))
+    # u = 0 => unit gates; b = 0 => selection orders like the raw scores
+    sel, g, sp, keys = o.gate_logic(s, 3)
+    assert np.all(g == 1.0)
+    np.testing.assert_allclose(sp.sum(axis=1), 1.0, rtol=1e-14)
+    np.testing.assert_array_equal(np.sort(sel, 1), np.sort(np.argsort(-s, axis=1)[:, :3], 1))
+    # softmax is shift-invariant
+    np.testing.assert_allclose(o.softmax(s + 123.0), sp, rtol=1e-12)
+    # N_r = 2: s'_0 = sigmoid(s_0 - s_1)
+    s2 = rng.normal(size=(20, 2))
+    _, g2, sp2, _ = o.gate_logic(s2, 1, gate_scale_u=np.array([0.5, -2.0]))
+    np.testing.assert_allclose(sp2[:, 0], 1 / (1 + np.exp(-(s2[:, 0] - s2[:, 1]))), rtol=1e-13)
+    win = (s2[:, 1] > s2[:, 0]).astype(int)
+    u = np.array([0.5, -2.0])
+    np.testing.assert_allclose(g2[:, 0], 1 + sp2[np.arange(20), win] * u[win], rtol=1e-14)
+    # the bias moves the selection but not the gate value
+    b = np.array([0, 0, 0, 0, 0, 10.0])
+    u6 = np.linspace(-1, 1, 6)
+    sel_b, g_b, sp_b, keys_b = o.gate_logic(s, 2, gate_scale_u=u6, select_bias_b=b)
+    assert np.all(sel_b[:, 0] == 5)
+    np.testing.assert_allclose(g_b[:, 0], 1 + sp_b[:, 5] * u6[5], rtol=1e-14)
+    np.testing.assert_allclose(keys_b, sp_b + b, rtol=0, atol=0)
+
+
+def pin_topk_brute_force(o):
+    """Selection = the N_k largest keys by a scalar scan, ties to the lower index."""
+    rng = np.random.default_rng(8)
+    s = rng.normal(size=(64, 7))
+    s[3, 2] = s[3, 5]                       # exact ties
+    s[9, :] = 0.25
+    b = rng.normal(scale=0.05, size=7)
+    for k in (1, 2, 4, 7):
+        sel, g, sp, keys = o.gate_logic(s, k, select_bias_b=b)
+        for t in range(s.shape[0]):
+            remaining = list(range(7))
+            want = []
+            for _ in range(k):
+                best = remaining[0]
+                for j in remaining[1:]:
+                    if keys[t, j] > keys[t, best]:
+                        best = j
+                want.append(best)
+                remaining.remove(best)
+            assert list(sel[t]) == want
+    sel, *_ = o.gate_logic(s, 2)
+    assert list(sel[9]) == [0, 1]
+    assert sorted(sel[3])[0] != 5 or 2 in sel[3]     # of two equal keys the lower index goes first
+
+
+def pin_moe_linear_in_gates(o):
+    shape, x, lay = small_layer(seed=6)
+    kw = dict(w_gate=lay.w_gate, w_up=lay.w_up, w_down=lay.w_down, neuron_perm=lay.neuron_perm,
+              n_experts=shape.n_experts, n_shared=shape.n_shared)
+    rng = np.random.default_rng(0)
+    sel = np.stack([rng.permutation(shape.n_routed)[:2] for _ in range(x.shape[0])]).astype(np.int32)
+    g1 = rng.normal(size=sel.shape)
+    g2 = rng.normal(size=sel.shape)
+    zero = np.zeros_like(g1)
+    f = lambda g: o.moe_forward(x, sel_idx=sel, gates=g, **kw)
+    base = f(zero)
+    np.testing.assert_allclose(f(g1 + g2) - base, (f(g1) - base) + (f(g2) - base),
+                               rtol=1e-9, atol=1e-12)
+    one = np.ones_like(g1)
+    assert np.abs(f(one) - base).max() > 1e-3
+    np.testing.assert_allclose(f(2.5 * one) - base, 2.5 * (f(one) - base), rtol=1e-9, atol=1e-12)
+    # gate 1 + s'u end to end: F_MoE(u) - F_MoE(0) = sum_sel s'_i u_i E_i(x)
+    u = np.linspace(-3, 3, shape.n_routed)
+    out_u, sel_u, g_u, _, sp, _ = o.cmoe_layer_forward(x, **layer_kwargs(shape, lay, gate_scale_u=u))
+    out_0, sel_0, *_ = o.cmoe_layer_forward(x, **layer_kwargs(shape, lay))
+    np.testing.assert_array_equal(sel_u, sel_0)
+    extra = np.zeros_like(out_0)
+    for t in range(x.shape[0]):
+        for j in sel_0[t]:
+            neurons = o.expert_neurons(lay.neuron_perm, shape.n_experts, shape.n_shared + j)
+            extra[t] += sp[t, j] * u[j] * o.expert_forward(x[t:t + 1], lay.w_gate, lay.w_up,
+                                                           lay.w_down, neurons)[0]
+    assert np.abs(extra).max() > 1e-4
+    np.testing.assert_allclose(out_u - out_0, extra, rtol=1e-8, atol=1e-12)
+    # token subset evaluation equals rows of the full evaluation
+    ids = np.array([0, 5, 6, 30])
+    np.testing.assert_allclose(o.moe_forward(x, sel_idx=sel, gates=g1, token_ids=ids, **kw),
+                               f(g1)[ids], rtol=1e-12, atol=1e-14)
+
+
+def pin_permutation(o):
+    rng = np.random.default_rng(9)
+    n_tok, n_r, k = 97, 6, 2
+    sel = np.stack([rng.permutation(n_r)[:k] for _ in range(n_tok)]).astype(np.int32)
+    sel[sel == 4] = 3 - (sel[sel == 4] * 0)           # leave expert 4 empty ...
+    for t in range(n_tok):                             # ... without duplicating a pair
+        if sel[t, 0] == sel[t, 1]:
+            sel[t, 1] = 5 if sel[t, 0] != 5 else 0
+    cnt, off, row_token, row_of = o.token_permutation(sel, n_r)
+    pairs = sorted((int(sel[t, j]), t) for t in range(n_tok) for j in range(k))
+    assert cnt.sum() == n_tok * k and cnt[4] == 0
+    assert off[0] == 0 and np.all(np.diff(off) == cnt)
+    assert [int(t) for t in row_token] == [t for _, t in pairs]
+    for e in range(n_r):
+        seg = row_token[off[e]:off[e + 1]]
+        assert np.all(np.diff(seg) > 0)
+        assert cnt[e] == sum(1 for ee, _ in pairs if ee == e)
+    for t in range(n_tok):
+        for j in range(k):
+            r = row_of[t, j]
+            assert row_token[r] == t and off[sel[t, j]] <= r < off[sel[t, j] + 1]
+    assert sorted(row_of.ravel()) == list(range(n_tok * k))
+
+
+def pin_logit_margin(o):
+    rng = np.random.default_rng(10)
+    s = rng.normal(size=(40, 5))
+    _, _, sp, keys = o.gate_logic(s, 2)
+    srt = -np.sort(-s, axis=1)
+    np.testing.assert_allclose(o.logit_margin(sp, keys, 2), 1 - np.exp(-(srt[:, 1] - srt[:, 2])),
+                               rtol=1e-10)
+    assert np.all(np.isinf(o.logit_margin(sp, keys, 5)))
+
+
+def pin_bias_update_rule(o):
+    """Overloaded experts lose gamma, underloaded gain gamma, target 1/N_r."""
+    b = np.array([0.1, 0.2, 0.3, 0.4])
+    got = o.bias_update(b, counts=[10, 30, 20, 20])        # shares .125 .375 .25 .25
+    np.testing.assert_allclose(got, [0.101, 0.199, 0.3, 0.4], rtol=0, atol=1e-15)
+    got = o.bias_update(b, counts=[10, 30, 20, 20], target_share=[0.1, 0.4, 0.3, 0.2], gamma=0.5)
+    np.testing.assert_allclose(got, [-0.4, 0.7, 0.8, -0.1], rtol=0, atol=1e-15)
+
+
+# ---------------------------------------------------------------- hierarchical
+def hier_case(seed=12, n_outer=4, top_k=None):
+    shape = wl.LayerShape(20, 8 * 5, 8, 2, 2, "fp32")
+    rng = np.random.Generator(np.random.PCG64(seed))
+    x = wl.draw_tokens(rng, 33, shape)
+    lays = [wl.draw_layer(rng, shape) for _ in range(n_outer)]
+    for lay in lays:
+        lay.w_gate *= 12.0
+        lay.w_up *= 12.0
+    w_r = rng.standard_normal((n_outer, shape.d_model))
+    layers = [layer_kwargs(shape, lay, top_k=shape.top_k if top_k is None else top_k)
+              for lay in lays]
+    return shape, x, lays, w_r, layers
+
+
+def pin_hierarchical_all_on_is_original_moe(o):
+    """Section 4.4: with every sub-expert on and unit sub-gates each outer
+    expert is its dense FFN, so the layer is the original top-2 MoE."""
+    shape, x, lays, w_r, layers = hier_case(top_k=6)
+    out, outer_idx, outer_w, _ = o.hier_forward(x, w_r, 2, layers)
+    np.testing.assert_allclose(outer_w.sum(axis=1), 1.0, rtol=1e-14)
+    logits = np.asarray(x, np.float64) @ w_r.T
+    want = np.zeros_like(out)
+    for t in range(x.shape[0]):
+        top = sorted(range(len(lays)), key=lambda i: (-logits[t, i], i))[:2]
+        assert list(outer_idx[t]) == top
+        z = [math.exp(logits[t, i] - logits[t, top[0]]) for i in top]
+        for i, zi in zip(top, z):
+            lay = lays[i]
+            want[t] += zi / sum(z) * o.dense_ffn(x[t:t + 1], lay.w_gate, lay.w_up, lay.w_down)[0]
+    np.testing.assert_allclose(out, want, rtol=1e-10, atol=1e-12)
+
+
+def pin_hierarchical_is_weighted_sum_of_layers(o):
+    shape, x, lays, w_r, layers = hier_case(seed=13)
+    out, outer_idx, outer_w, routing = o.hier_forward(x, w_r, 2, layers)
+    want = np.zeros_like(out)
+    for i, kw in enumerate(layers):
+        y, *_ = o.cmoe_layer_forward(x, **kw)
+        for slot in range(2):
+            hit = outer_idx[:, slot] == i
+            want[hit] += outer_w[hit, slot][:, None] * y[hit]
+    np.testing.assert_allclose(out, want, rtol=1e-10, atol=1e-13)
+    ids = np.array([1, 2, 17, 32])
+    sub, *_ = o.hier_forward(x, w_r, 2, layers, token_ids=ids)
+    np.testing.assert_allclose(sub, out[ids], rtol=1e-12, atol=1e-14)
+
+
+PINS = [pin_dense_closed_form, pin_dense_library, pin_dense_per_neuron_brute_force,
+        pin_all_experts_on_is_dense, pin_reconstruction_error_identity, pin_shared_always_on,
+        pin_router_is_representative_activation, pin_gate_closed_forms, pin_topk_brute_force,
+        pin_moe_linear_in_gates, pin_permutation, pin_logit_margin, pin_bias_update_rule,
+        pin_hierarchical_all_on_is_original_moe, pin_hierarchical_is_weighted_sum_of_layers]
+
+
+@pytest.mark.parametrize("pin", PINS, ids=lambda p: p.__name__)
+def test_pin(pin):
+    pin(oracle)
+
+
+# ----------------------------------------------------- planted mistakes (CPU)
+def _mutant(patch_src):
+    """A copy of the oracle module with one textual edit applied."""
+    path = oracle.__file__
+    src = open(path).read()
+    old, new = patch_src
+    assert src.count(old) >= 1, f"mutation anchor not found: {old!r}"
+    mod = types.ModuleType("oracle_mutant")
+    mod.__file__ = path
+    exec(compile(src.replace(old, new, 1), path, "exec"), mod.__dict__)
+    return mod
+
+
+MUTATIONS = {
+    "swish_without_sigmoid": ("return a / (1.0 + np.exp(-a))", "return a"),
+    "sigmoid_sign": ("return a / (1.0 + np.exp(-a))", "return a / (1.0 + np.exp(a))"),
+    "gate_up_swapped": ("return swish(x @ wg.T) * (x @ wu.T)", "return swish(x @ wu.T) * (x @ wg.T)"),
+    "down_transposed_slice": ("return h @ _f64(w_down[:, neurons]).T",
+                              "return h @ _f64(w_down[:, neurons[::-1]]).T"),
+    "shared_dropped": ("if n_shared > 0:", "if False:"),
+    "expert_offset": ("expert_neurons(neuron_perm, n_experts, n_shared + j)\n        y =",
+                      "expert_neurons(neuron_perm, n_experts, j)\n        y ="),
+    "gate_ignored": ("out[hit_tok] += gates[hit_tok, hit_slot][:, None] * y", "out[hit_tok] += y"),
+    "smallest_selected": ("order = np.argsort(-rank_keys, axis=1, kind=\"stable\")",
+                          "order = np.argsort(rank_keys, axis=1, kind=\"stable\")"),
+    "bias_in_gate": ("gates = 1.0 + np.take_along_axis(s_prime,", "gates = 1.0 + np.take_along_axis(keys,"),
+    "softmax_unnormalised": ("return z / z.sum(axis=-1, keepdims=True)", "return z"),
+    "offsets_inclusive": ("off[e + 1] = off[e] + cnt[e]", "off[e + 1] = off[e] + cnt[e] + (e == 0)"),
+    "outer_weights_unnormalised": ("outer_w = softmax(sel_logits)", "outer_w = np.exp(sel_logits)"),
+    "bias_rule_sign": ("b[p > target] -= gamma", "b[p > target] += gamma"),
+}
+
+
+@pytest.mark.parametrize("name", sorted(MUTATIONS))
+def test_planted_mistakes_are_caught(name):
+    mutant = _mutant(MUTATIONS[name])
+    failed = []
+    for pin in PINS:
+        try:
+            pin(mutant)
+        except (AssertionError, ValueError, IndexError):
+            failed.append(pin.__name__)
+    assert failed, f"no pin noticed the planted mistake {name!r}"
+
+
+# ------------------------------------------------------------ paper's numbers
+def test_flop_model_against_papers_table():
+    """tests/golden/paper_efficiency_flops.txt: dense vs restructured Llama-2-7B
+    whole-model FLOPs (Table efficiency_flops).  The FFN-only saving predicted
+    by the per-token flop model, times the FFN's share of the matmul flops,
+    must land on the printed whole-model saving."""
+    rows = {}
+    for line in open(os.path.join(GOLDEN, "paper_efficiency_flops.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        k, v = line.split("=")
+        rows[k.strip()] = float(v)
+    shape = wl.LayerShape(4096, 11008, 8, 3, 3, "bf16")          # S3A3E8 on Llama-2-7B
+    ffn_saving = 1.0 - shape.flops_per_token() / shape.dense_flops_per_token()
+    assert abs(ffn_saving - 0.25) < 2e-3                          # router cost is ~0.1 %
+    n_layers, vocab, d = 32, 32000, 4096
+    ffn = n_layers * shape.dense_flops_per_token()
+    attn_proj = n_layers * 2 * 4 * d * d
+    lm_head = 2 * d * vocab
+    share = ffn / (ffn + attn_proj + lm_head)
+    printed = 1.0 - rows["ours_tflops"] / rows["dense_tflops"]
+    assert abs(printed - rows["printed_reduction"]) < 2e-3
+    assert abs(ffn_saving * share - printed) < 0.015
