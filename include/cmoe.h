@@ -1,0 +1,174 @@
+/* cmoe.h — C ABI of the B200 (sm_100a) forward pass of a SwiGLU FFN restructured
+ * into a sparse mixture of experts (shared + routed experts with an analytical
+ * router).
+ *
+ * Method (paper notation): an FFN with hidden width d_h is split, by a neuron
+ * partition, into N experts of m = d_h/N neurons, N_s shared (always on) and
+ * N_r = N - N_s routed (Section 4.1).  For a token x
+ *     F_MoE(x) = E^s(x) + sum_{i<=N_r} g_i E_i^r(x)                 (Eq. moe_output)
+ * where every expert is the SwiGLU FFN restricted to its neurons
+ *     E(x) = W_down[S]^T ( Swish(W_gate[S]^T x) * (W_up[S]^T x) )   (Eq. ori_ffn_method)
+ * the router scores are the SwiGLU activations of one representative neuron
+ * per routed expert
+ *     s = Swish(W_gate^{R T} x) * (W_up^{R T} x)                    (Eq. router)
+ * and, with s' = Softmax(s) over all N_r scores,
+ *     g_i = 1 + s'_i u_i  if s'_i + b_i is among the N_k largest keys, else 0
+ *                                                                   (Eq. final_gate).
+ * Equal keys: the lower expert index wins.  NaN keys rank below every number.
+ *
+ * All functions return CMOE_OK (0) or a negative cmoe_status; none throws,
+ * aborts or prints.  "device" pointers are CUDA global memory of the device
+ * that was current at create time; "host" pointers are ordinary memory that
+ * is only read (or written) during the call.  A stream argument is a
+ * cudaStream_t passed as void* (NULL = the legacy default stream).
+ */
+#ifndef CMOE_H_
+#define CMOE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cmoe_layer cmoe_layer;   /* opaque; owns device memory */
+
+typedef enum {
+  CMOE_OK = 0,
+  CMOE_ERR_INVALID_ARG = -1,     /* null pointer, negative size, unsupported shape */
+  CMOE_ERR_BAD_PARTITION = -2,   /* d_ff % n_experts != 0, or neuron_perm is not a bijection */
+  CMOE_ERR_BAD_REP = -3,         /* a representative lies outside its routed expert's slice */
+  CMOE_ERR_CAPACITY = -4,        /* T > max_tokens, or a size beyond a stated maximum */
+  CMOE_ERR_CUDA = -5,            /* a CUDA runtime/driver call failed (see cmoe_last_error) */
+  CMOE_ERR_DEVICE_TIMEOUT = -6,  /* a bounded device-side wait gave up (see cmoe_layer_status) */
+  CMOE_ERR_UNSUPPORTED = -7      /* the device is not compute capability 10.x */
+} cmoe_status;
+
+typedef enum { CMOE_BF16 = 0, CMOE_FP32 = 1 } cmoe_dtype;
+
+typedef struct {
+  int32_t d_model;      /* d */
+  int32_t d_ff;         /* d_h */
+  int32_t n_experts;    /* N ; m = d_ff / N must divide exactly */
+  int32_t n_shared;     /* N_s >= 0 */
+  int32_t top_k;        /* N_k, 0 <= N_k <= N_r = N - N_s ; N_r <= 32, N_k <= 8 */
+  int32_t max_tokens;   /* the workspace is sized for this many tokens at create */
+  int32_t dtype;        /* cmoe_dtype of x, out and every weight matrix */
+} cmoe_config;
+
+/* Build a layer from the dense FFN's weights, the neuron partition and the
+ * representative neurons (Sections 4.1 and 4.2).
+ *   w_gate, w_up : device, [d_ff, d_model] row-major; row n is neuron n's vector
+ *                  (column n of the paper's W_gate / W_up).
+ *   w_down       : device, [d_model, d_ff] row-major; column n is neuron n's output
+ *                  vector (row n of the paper's W_down).
+ *   neuron_perm  : host, [d_ff]; expert e owns original neurons
+ *                  neuron_perm[e*m .. (e+1)*m); experts 0..N_s-1 are shared and
+ *                  form one always-on expert of N_s*m neurons.
+ *   rep_idx      : host, [N_r]; ORIGINAL index of routed expert j's representative
+ *                  neuron R_j (Eq. rep_neuron); must lie in expert N_s+j's slice.
+ *   gate_scale_u : host, [N_r] or NULL (zeros, i.e. unit gates)   (Section 4.3)
+ *   select_bias_b: host, [N_r] or NULL (zeros)                     (Eq. final_gate)
+ * The weights are copied into expert-contiguous operand layouts on `stream`;
+ * the call synchronises that stream before returning, so the caller may free
+ * its arrays afterwards.  Requires d_model % 8 == 0.
+ * Errors: INVALID_ARG, BAD_PARTITION, BAD_REP, CUDA, UNSUPPORTED. */
+int cmoe_layer_create(const cmoe_config* cfg, const void* w_gate, const void* w_up,
+                      const void* w_down, const int32_t* neuron_perm, const int32_t* rep_idx,
+                      const float* gate_scale_u, const float* select_bias_b, void* stream,
+                      cmoe_layer** out_layer);
+
+/* Hierarchical restructuring of an existing MoE layer (Section 4.4): every one
+ * of the n_outer experts has been restructured into its own shared + routed
+ * sub-experts (inner[i], all created with the same cmoe_config); a top-level
+ * router picks outer_top_k of them per token:
+ *     logits = W_r x, selected = the outer_top_k largest logits (ties: lower
+ *     index), weights w = softmax over the selected logits,
+ *     out = sum_{i selected} w_i (E_i^s(x) + sum_j g'_{i,j} E^r_{i,j}(x)).
+ *   w_router : device, [n_outer, d_model] row-major, same dtype as the layers.
+ *   inner    : host array of n_outer layers; on success their device memory has
+ *              been moved into the new layer and the handles are dead (do not
+ *              destroy them); on failure they are untouched.
+ *   max_tokens: capacity in tokens of the new layer.
+ * forward / destroy / get_routing / status of the result are the calls below. */
+int cmoe_hier_create(int32_t n_outer, int32_t outer_top_k, const void* w_router,
+                     cmoe_layer* const* inner, int32_t max_tokens, void* stream,
+                     cmoe_layer** out_layer);
+
+/* out = F_MoE(x) for T tokens (Eq. moe_output with Eq. router and Eq. final_gate).
+ *   x   : device, [T, d_model] row-major, 16-byte aligned.
+ *   out : device, [T, d_model] row-major, 16-byte aligned, must not overlap x.
+ * Asynchronous on `stream`; allocates nothing; T == 0 is a no-op.  A layer owns
+ * one workspace: do not run two forwards of the same layer concurrently.
+ * Errors: INVALID_ARG, CAPACITY (T > max_tokens), CUDA. */
+int cmoe_ffn_forward(cmoe_layer* layer, const void* x, int32_t T, void* out, void* stream);
+
+/* Replace the learnable gate scaling u and the selection bias b (Section 4.3).
+ * host arrays [n_routed_groups] (N_r, or n_outer*N_r for a hierarchical layer,
+ * outer-major) or NULL for zeros.  Synchronises `stream`. */
+int cmoe_layer_set_gate_params(cmoe_layer* layer, const float* gate_scale_u,
+                               const float* select_bias_b, void* stream);
+
+/* Choose the expert-GEMM implementation: 0 = automatic (tensor-core path when the
+ * dtype is bf16 and the shape allows, else the plain SIMT path), 1 = always SIMT,
+ * 2 = tensor-core, or CMOE_ERR_INVALID_ARG if the layer cannot take it. */
+int cmoe_layer_set_gemm_path(cmoe_layer* layer, int32_t path);
+
+/* Sizes a caller needs to read the routing state back.  n_outer / outer_top_k
+ * are 0 for a plain layer. */
+int cmoe_layer_dims(const cmoe_layer* layer, int32_t* n_routed_groups, int32_t* top_k,
+                    int32_t* n_outer, int32_t* outer_top_k);
+
+/* Copy the routing state of the LAST forward (T tokens) to host buffers; any
+ * pointer may be NULL.  Synchronises the stream of that forward.  R = T for a
+ * plain layer, T*outer_top_k for a hierarchical one (outer rows); G = routed groups.
+ *   keys      [R, N_r] fp32  s'_i + b_i of every routed expert of the row's (outer) layer
+ *   scores    [R, N_r] fp32  s_i (Eq. router)
+ *   topk_idx  [R, N_k] int32 selected routed GROUP (outer*N_r + j), descending key
+ *   topk_gate [R, N_k] fp32  g_i = 1 + s'_i u_i
+ *   counts    [G] , offsets [G+1] int32  rows per routed group and their exclusive scan
+ *   row_token [R*N_k] int32  row r of the expert-contiguous order holds outer row row_token[r]
+ *                            (= token for a plain layer); ascending inside a group
+ *   row_of    [R, N_k] int32 inverse map: row of pair (r, j)
+ *   outer_idx [T, outer_top_k] int32, outer_w [T, outer_top_k] fp32, outer_row_token [R] int32
+ *                            hierarchical layers only. */
+int cmoe_get_routing(cmoe_layer* layer, float* keys, float* scores, int32_t* topk_idx,
+                     float* topk_gate, int32_t* counts, int32_t* offsets, int32_t* row_token,
+                     int32_t* row_of, int32_t* outer_idx, float* outer_w,
+                     int32_t* outer_row_token);
+
+/* Device-side error word of the last forward: 0, or a code written by a kernel whose
+ * bounded wait (mbarrier) ran out.  Synchronises the last stream.  Returns
+ * CMOE_ERR_DEVICE_TIMEOUT when the word is non-zero. */
+int cmoe_layer_status(cmoe_layer* layer, int32_t* device_error_word);
+
+/* Number of this library's kernels the last forward launched. */
+int cmoe_layer_launch_count(const cmoe_layer* layer, int32_t* n_launches);
+
+int cmoe_layer_destroy(cmoe_layer* layer);
+
+/* Stand-alone token histogram / exclusive scan / stable permutation: the
+ * expert-contiguous order of the selected (token, expert) pairs — the paper only
+ * states that the top-N_k routed experts of a token are activated (Eq. moe_output);
+ * the canonical listing is "sorted by (expert, token)".
+ *   topk_idx : device int32 [n_rows, n_k], entries in [0, n_groups); a row never
+ *              names the same group twice (entries out of range are ignored).
+ *   counts [n_groups], offsets [n_groups+1], row_token [n_rows*n_k], row_of [n_rows, n_k]:
+ *              device int32 outputs, as in cmoe_get_routing.
+ *   scratch  : device, at least cmoe_token_permute_scratch_bytes(n_rows, n_groups) bytes,
+ *              256-byte aligned; contents need not be initialised; may be NULL when
+ *              n_rows <= 256.
+ * Asynchronous on `stream`; allocates nothing.  n_groups <= 1024, n_k <= 8. */
+int64_t cmoe_token_permute_scratch_bytes(int32_t n_rows, int32_t n_groups);
+int cmoe_token_permute(const int32_t* topk_idx, int32_t n_rows, int32_t n_k, int32_t n_groups,
+                       int32_t* counts, int32_t* offsets, int32_t* row_token, int32_t* row_of,
+                       void* scratch, int64_t scratch_bytes, void* stream);
+
+const char* cmoe_status_string(int status);
+/* Text of the most recent error seen by this library on the calling thread. */
+const char* cmoe_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* CMOE_H_ */
