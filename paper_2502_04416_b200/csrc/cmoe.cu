@@ -1,0 +1,610 @@
+// C-ABI library: layer construction (weight repacking into expert-contiguous
+// operand layouts), the forward pass as a sequence of kernels on the caller's
+// stream, and the read-back accessors.  Declarations and contracts: include/cmoe.h.
+#include "../../include/cmoe.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "combine.cuh"
+#include "common.cuh"
+#include "permute.cuh"
+#include "router.cuh"
+#include "simt_gemm.cuh"
+#include "umma_gemm.cuh"
+
+using namespace cmoe;
+
+namespace {
+
+thread_local char g_last_error[512] = "";
+
+int cuda_fail(cudaError_t e, const char* what) {
+  snprintf(g_last_error, sizeof(g_last_error), "%s: %s", what, cudaGetErrorString(e));
+  return CMOE_ERR_CUDA;
+}
+int arg_fail(int code, const char* what) {
+  snprintf(g_last_error, sizeof(g_last_error), "%s", what);
+  return code;
+}
+
+#define CU_TRY(expr)                                          \
+  do {                                                        \
+    cudaError_t e_ = (expr);                                  \
+    if (e_ != cudaSuccess) return cuda_fail(e_, #expr);       \
+  } while (0)
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Bump allocator over one device allocation (base == nullptr: measure only).
+struct Arena {
+  char* base = nullptr;
+  size_t used = 0;
+  template <typename U> U* take(size_t n) {
+    used = align_up(used, 256);
+    U* p = base ? reinterpret_cast<U*>(base + used) : nullptr;
+    used += n * sizeof(U);
+    return p;
+  }
+};
+
+}  // namespace
+
+struct cmoe_layer {
+  cmoe_config cfg{};
+  int m = 0, n_r = 0, n_outer = 1, outer_k = 1;
+  bool hier = false;
+  int device = 0;
+  size_t esz = 2;
+  int gemm_path = 0;
+  bool umma_ok = false;
+
+  // packed weights
+  void* wg_p = nullptr;     // [n_outer*d_ff, d]   neurons in expert order
+  void* wu_p = nullptr;     // [n_outer*d_ff, d]
+  void* wd_p = nullptr;     // per outer expert: shared block [d, N_s*m], then N_r blocks [d, m]
+  void* w_rep = nullptr;    // [n_outer][2*N_r][d] representatives' gate rows, then up rows
+  void* w_router = nullptr; // [n_outer, d] (hierarchical)
+  float* u = nullptr;       // [n_outer*N_r]
+  float* b = nullptr;
+  GroupStatic* gs = nullptr;
+  std::vector<GroupStatic> gs_host;
+
+  // workspace (one allocation)
+  void* ws = nullptr;
+  size_t ws_bytes = 0;
+  float *scores = nullptr, *keys = nullptr, *topk_gate = nullptr;
+  int32_t *topk_idx = nullptr, *row_of = nullptr, *row_token = nullptr, *counts = nullptr,
+          *offsets = nullptr, *perm_scratch = nullptr;
+  GroupRows* gr = nullptr;
+  void *x_perm = nullptr, *h_s = nullptr, *h_r = nullptr, *y_s = nullptr, *y_r = nullptr;
+  // hierarchical
+  float *outer_logits = nullptr, *outer_w = nullptr;
+  int32_t *outer_idx = nullptr, *outer_counts = nullptr, *outer_off = nullptr,
+          *outer_row_token = nullptr, *outer_row_of = nullptr, *outer_scratch = nullptr;
+  void* xo = nullptr;
+  int32_t* err_word = nullptr;
+  UmmaPlan umma;
+
+  cudaStream_t last_stream = nullptr;
+  int last_T = 0;
+  int launches = 0;
+
+  int n_groups_total() const { return n_outer + n_outer * n_r; }
+  int shared_width() const { return cfg.n_shared * m; }
+};
+
+namespace {
+
+void free_layer(cmoe_layer* L) {
+  if (!L) return;
+  umma_plan_destroy(&L->umma);
+  cudaFree(L->wg_p); cudaFree(L->wu_p); cudaFree(L->wd_p); cudaFree(L->w_rep);
+  cudaFree(L->w_router); cudaFree(L->u); cudaFree(L->b); cudaFree(L->gs); cudaFree(L->ws);
+  delete L;
+}
+
+template <typename T>
+__global__ void pack_down_kernel(const T* __restrict__ w_down, const int32_t* __restrict__ perm, int d,
+                                 int d_ff, int m, int shared_w, T* __restrict__ dst) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;   // packed neuron position
+  const int c = blockIdx.y;
+  if (n >= d_ff) return;
+  const T v = w_down[(size_t)c * d_ff + perm[n]];
+  size_t o;
+  if (n < shared_w) {
+    o = (size_t)c * shared_w + n;
+  } else {
+    const int j = (n - shared_w) / m, k = (n - shared_w) % m;
+    o = (size_t)shared_w * d + (size_t)j * m * d + (size_t)c * m + k;
+  }
+  dst[o] = v;
+}
+
+int check_config(const cmoe_config& c) {
+  if (c.d_model <= 0 || c.d_ff <= 0 || c.n_experts <= 0 || c.n_shared < 0 || c.top_k < 0 ||
+      c.max_tokens <= 0)
+    return arg_fail(CMOE_ERR_INVALID_ARG, "non-positive dimension");
+  if (c.dtype != CMOE_BF16 && c.dtype != CMOE_FP32) return arg_fail(CMOE_ERR_INVALID_ARG, "dtype");
+  if (c.d_model % 8) return arg_fail(CMOE_ERR_INVALID_ARG, "d_model must be a multiple of 8");
+  if (c.d_ff % c.n_experts) return arg_fail(CMOE_ERR_BAD_PARTITION, "d_ff % n_experts != 0");
+  if (c.n_shared > c.n_experts) return arg_fail(CMOE_ERR_INVALID_ARG, "n_shared > n_experts");
+  const int n_r = c.n_experts - c.n_shared;
+  if (c.top_k > n_r) return arg_fail(CMOE_ERR_INVALID_ARG, "top_k > routed experts");
+  if (n_r > kMaxRouted) return arg_fail(CMOE_ERR_INVALID_ARG, "more than 32 routed experts");
+  if (c.top_k > kMaxTopK) return arg_fail(CMOE_ERR_INVALID_ARG, "top_k > 8");
+  return CMOE_OK;
+}
+
+int check_device() {
+  int dev = 0, major = 0;
+  CU_TRY(cudaGetDevice(&dev));
+  CU_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+  if (major != 10) return arg_fail(CMOE_ERR_UNSUPPORTED, "device is not compute capability 10.x");
+  return CMOE_OK;
+}
+
+void build_group_statics(cmoe_layer* L) {
+  const int d = L->cfg.d_model, d_ff = L->cfg.d_ff, m = L->m, sw = L->shared_width();
+  L->gs_host.assign(L->n_groups_total(), GroupStatic{});
+  for (int i = 0; i < L->n_outer; ++i) {
+    GroupStatic& s = L->gs_host[i];
+    s.w_row0 = i * d_ff; s.width = sw; s.wd_offset = (int64_t)i * d * d_ff; s.is_shared = 1; s.outer = i;
+    for (int j = 0; j < L->n_r; ++j) {
+      GroupStatic& r = L->gs_host[L->n_outer + i * L->n_r + j];
+      r.w_row0 = i * d_ff + sw + j * m; r.width = m;
+      r.wd_offset = (int64_t)i * d * d_ff + (int64_t)sw * d + (int64_t)j * m * d;
+      r.is_shared = 0; r.outer = i;
+    }
+  }
+}
+
+// Lays out the workspace; with base == nullptr only measures it.
+void carve_workspace(cmoe_layer* L, char* base) {
+  Arena a; a.base = base;
+  const size_t T = L->cfg.max_tokens, R = T * (L->hier ? L->outer_k : 1), P = R * L->cfg.top_k;
+  const size_t d = L->cfg.d_model, nr = L->n_r, G = (size_t)L->n_outer * nr, esz = L->esz;
+  L->scores = a.take<float>(R * nr);
+  L->keys = a.take<float>(R * nr);
+  L->topk_idx = a.take<int32_t>(P);
+  L->topk_gate = a.take<float>(P);
+  L->row_of = a.take<int32_t>(P);
+  L->row_token = a.take<int32_t>(P);
+  L->counts = a.take<int32_t>(G);
+  L->offsets = a.take<int32_t>(G + 1);
+  L->perm_scratch = a.take<int32_t>(permute_scratch_bytes((int)R, (int)(G ? G : 1)) / 4);
+  L->gr = a.take<GroupRows>(L->n_groups_total());
+  L->err_word = a.take<int32_t>(1);
+  L->x_perm = a.take<char>(P * d * esz);
+  L->h_s = a.take<char>(R * L->shared_width() * esz);
+  L->h_r = a.take<char>(P * L->m * esz);
+  L->y_s = a.take<char>(R * d * esz);
+  L->y_r = a.take<char>(P * d * esz);
+  if (L->hier) {
+    L->outer_logits = a.take<float>(T * L->n_outer);
+    L->outer_w = a.take<float>(T * L->outer_k);
+    L->outer_idx = a.take<int32_t>(T * L->outer_k);
+    L->outer_counts = a.take<int32_t>(L->n_outer);
+    L->outer_off = a.take<int32_t>(L->n_outer + 1);
+    L->outer_row_token = a.take<int32_t>(R);
+    L->outer_row_of = a.take<int32_t>(R);
+    L->outer_scratch = a.take<int32_t>(permute_scratch_bytes((int)T, L->n_outer) / 4);
+    L->xo = a.take<char>(R * d * esz);
+  }
+  L->ws_bytes = align_up(a.used + 256, 256);
+}
+
+int alloc_workspace(cmoe_layer* L) {
+  carve_workspace(L, nullptr);
+  CU_TRY(cudaMalloc(&L->ws, L->ws_bytes));
+  carve_workspace(L, static_cast<char*>(L->ws));
+  CU_TRY(cudaMemset(L->ws, 0, L->ws_bytes));
+  return CMOE_OK;
+}
+
+int upload_gate_params(cmoe_layer* L, const float* u, const float* b, cudaStream_t st) {
+  const size_t n = (size_t)L->n_outer * L->n_r;
+  if (n == 0) return CMOE_OK;
+  std::vector<float> zeros(n, 0.0f);
+  CU_TRY(cudaMemcpyAsync(L->u, u ? u : zeros.data(), n * sizeof(float), cudaMemcpyHostToDevice, st));
+  CU_TRY(cudaMemcpyAsync(L->b, b ? b : zeros.data(), n * sizeof(float), cudaMemcpyHostToDevice, st));
+  CU_TRY(cudaStreamSynchronize(st));
+  return CMOE_OK;
+}
+
+int finish_layer(cmoe_layer* L, cudaStream_t st) {
+  build_group_statics(L);
+  CU_TRY(cudaMalloc(&L->gs, L->gs_host.size() * sizeof(GroupStatic)));
+  CU_TRY(cudaMemcpyAsync(L->gs, L->gs_host.data(), L->gs_host.size() * sizeof(GroupStatic),
+                         cudaMemcpyHostToDevice, st));
+  int rc = alloc_workspace(L);
+  if (rc != CMOE_OK) return rc;
+  L->umma_ok = false;
+  if (L->cfg.dtype == CMOE_BF16) {
+    UmmaShape s;
+    s.d = L->cfg.d_model; s.m = L->m; s.shared_width = L->shared_width(); s.d_ff = L->cfg.d_ff;
+    s.n_outer = L->n_outer; s.n_r = L->n_r;
+    s.max_outer_rows = (size_t)L->cfg.max_tokens * (L->hier ? L->outer_k : 1);
+    s.max_routed_rows = s.max_outer_rows * L->cfg.top_k;
+    rc = umma_plan_create(&L->umma, s, L->gs_host.data(), L->n_groups_total(), L->wg_p, L->wu_p,
+                          L->wd_p, L->x_perm, L->h_s, L->h_r, L->y_s, L->y_r);
+    if (rc == CMOE_ERR_CUDA) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
+    L->umma_ok = (rc == CMOE_OK);
+  }
+  CU_TRY(cudaStreamSynchronize(st));
+  return CMOE_OK;
+}
+
+template <typename T>
+int pack_weights(cmoe_layer* L, const void* w_gate, const void* w_up, const void* w_down,
+                 const int32_t* perm_dev, const int32_t* rep_dev, cudaStream_t st) {
+  const int d = L->cfg.d_model, d_ff = L->cfg.d_ff;
+  const int row_vec = d * (int)sizeof(T) / 16;
+  gather_rows_kernel<<<d_ff, 256, 0, st>>>((const uint4*)w_gate, perm_dev, d_ff, row_vec, (uint4*)L->wg_p);
+  gather_rows_kernel<<<d_ff, 256, 0, st>>>((const uint4*)w_up, perm_dev, d_ff, row_vec, (uint4*)L->wu_p);
+  if (L->n_r > 0) {
+    gather_rows_kernel<<<L->n_r, 256, 0, st>>>((const uint4*)w_gate, rep_dev, L->n_r, row_vec,
+                                               (uint4*)L->w_rep);
+    gather_rows_kernel<<<L->n_r, 256, 0, st>>>((const uint4*)w_up, rep_dev, L->n_r, row_vec,
+                                               (uint4*)((char*)L->w_rep + (size_t)L->n_r * d * sizeof(T)));
+  }
+  dim3 grid((d_ff + 255) / 256, d);
+  pack_down_kernel<T><<<grid, 256, 0, st>>>((const T*)w_down, perm_dev, d, d_ff, L->m, L->shared_width(),
+                                            (T*)L->wd_p);
+  CU_TRY(cudaGetLastError());
+  return CMOE_OK;
+}
+
+template <typename T>
+int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) {
+  const int d = L->cfg.d_model, n_r = L->n_r, n_k = L->cfg.top_k;
+  const int R = n_tok * (L->hier ? L->outer_k : 1);
+  const int P = R * n_k;
+  const int G = L->n_outer * n_r;
+  const int row_vec = d * (int)sizeof(T) / 16;
+  int launches = 0;
+  const T* xo = x;
+
+  if (L->hier) {
+    outer_router_kernel<T><<<(n_tok + 7) / 8, 256, 0, st>>>(x, n_tok, d, L->n_outer, L->outer_k,
+                                                            (const T*)L->w_router, L->outer_logits,
+                                                            L->outer_idx, L->outer_w);
+    ++launches;
+    launches += launch_token_permute(L->outer_idx, n_tok, L->outer_k, L->n_outer, L->outer_counts,
+                                     L->outer_off, L->outer_row_token, L->outer_row_of,
+                                     L->outer_scratch, st);
+    gather_rows_kernel<<<R, 256, 0, st>>>((const uint4*)x, L->outer_row_token, R, row_vec, (uint4*)L->xo);
+    ++launches;
+    xo = (const T*)L->xo;
+  }
+
+  if (n_r > 0) {
+    const int warps = (R + 1) / 2, blocks = (warps + 7) / 8;
+    const int32_t* ooff = L->hier ? L->outer_off : nullptr;
+#define CMOE_ROUTER(NACC)                                                                         \
+  router_kernel<T, NACC><<<blocks, 256, 0, st>>>(xo, R, d, n_r, n_k, (const T*)L->w_rep, L->u,   \
+                                                 L->b, ooff, L->n_outer, L->scores, L->keys,      \
+                                                 L->topk_idx, L->topk_gate)
+    if (2 * n_r <= 16) CMOE_ROUTER(16);
+    else if (2 * n_r <= 32) CMOE_ROUTER(32);
+    else CMOE_ROUTER(64);
+#undef CMOE_ROUTER
+    ++launches;
+    launches += launch_token_permute(L->topk_idx, R, n_k, G, L->counts, L->offsets, L->row_token,
+                                     L->row_of, L->perm_scratch, st);
+  }
+  plan_groups_kernel<<<1, 256, 0, st>>>(L->n_outer, n_r, n_tok, L->hier ? L->outer_off : nullptr,
+                                        L->counts, L->offsets, L->gr);
+  ++launches;
+  if (P > 0) {
+    gather_rows_kernel<<<P, 256, 0, st>>>((const uint4*)xo, L->row_token, P, row_vec, (uint4*)L->x_perm);
+    ++launches;
+  }
+
+  const bool use_umma = L->umma_ok && L->gemm_path != 1;
+  if (use_umma) {
+    const int n = umma_forward(&L->umma, xo, R, P, L->gr, L->err_word, st);
+    if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
+    launches += n;
+  } else {
+    SimtGemmArgs<T> a;
+    a.gs = L->gs; a.gr = L->gr; a.d = d;
+    a.shared_width = L->shared_width(); a.routed_width = L->m;
+    const int max_w = a.shared_width > a.routed_width ? a.shared_width : a.routed_width;
+    a.a_shared = xo; a.a_routed = (const T*)L->x_perm;
+    a.w_gate = (const T*)L->wg_p; a.w_up = (const T*)L->wu_p;
+    a.c_shared = (T*)L->h_s; a.c_routed = (T*)L->h_r;
+    dim3 g1((R + kSimtTile - 1) / kSimtTile, (max_w + kSimtTile - 1) / kSimtTile, L->n_groups_total());
+    simt_gemm1_kernel<T><<<g1, 256, 0, st>>>(a);
+    a.a_shared = (const T*)L->h_s; a.a_routed = (const T*)L->h_r;
+    a.w_gate = (const T*)L->wd_p; a.w_up = nullptr;
+    a.c_shared = (T*)L->y_s; a.c_routed = (T*)L->y_r;
+    dim3 g2((R + kSimtTile - 1) / kSimtTile, (d + kSimtTile - 1) / kSimtTile, L->n_groups_total());
+    simt_gemm2_kernel<T><<<g2, 256, 0, st>>>(a);
+    launches += 2;
+  }
+
+  const int threads = d / 8 < 256 ? ((d / 8 + 31) / 32 * 32) : 256;
+  combine_kernel<T><<<n_tok, threads, 0, st>>>(
+      L->cfg.n_shared > 0 ? (const T*)L->y_s : nullptr, (const T*)L->y_r, L->topk_idx, L->topk_gate,
+      L->row_of, L->hier ? L->outer_row_of : nullptr, L->hier ? L->outer_w : nullptr,
+      L->hier ? L->outer_k : 1, n_k, d, out);
+  ++launches;
+  CU_TRY(cudaGetLastError());
+  L->launches = launches;
+  return CMOE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int cmoe_layer_create(const cmoe_config* cfg, const void* w_gate, const void* w_up,
+                      const void* w_down, const int32_t* neuron_perm, const int32_t* rep_idx,
+                      const float* gate_scale_u, const float* select_bias_b, void* stream,
+                      cmoe_layer** out_layer) {
+  if (!cfg || !w_gate || !w_up || !w_down || !neuron_perm || !out_layer)
+    return arg_fail(CMOE_ERR_INVALID_ARG, "null argument");
+  *out_layer = nullptr;
+  int rc = check_config(*cfg);
+  if (rc != CMOE_OK) return rc;
+  const int d = cfg->d_model, d_ff = cfg->d_ff, m = d_ff / cfg->n_experts;
+  const int n_r = cfg->n_experts - cfg->n_shared;
+  if (n_r > 0 && !rep_idx) return arg_fail(CMOE_ERR_INVALID_ARG, "rep_idx is null");
+  {
+    std::vector<int32_t> where(d_ff, -1);          // original neuron -> packed position
+    for (int i = 0; i < d_ff; ++i) {
+      const int32_t n = neuron_perm[i];
+      if (n < 0 || n >= d_ff || where[n] >= 0)
+        return arg_fail(CMOE_ERR_BAD_PARTITION, "neuron_perm is not a permutation of [0, d_ff)");
+      where[n] = i;
+    }
+    for (int j = 0; j < n_r; ++j) {
+      const int32_t r = rep_idx[j];
+      if (r < 0 || r >= d_ff || where[r] / m != cfg->n_shared + j)
+        return arg_fail(CMOE_ERR_BAD_REP, "representative outside its routed expert's slice");
+    }
+  }
+  rc = check_device();
+  if (rc != CMOE_OK) return rc;
+
+  cmoe_layer* L = new (std::nothrow) cmoe_layer();
+  if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "out of host memory");
+  L->cfg = *cfg; L->m = m; L->n_r = n_r; L->n_outer = 1; L->outer_k = 1; L->hier = false;
+  L->esz = cfg->dtype == CMOE_BF16 ? 2 : 4;
+  cudaGetDevice(&L->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t *perm_dev = nullptr, *rep_dev = nullptr;
+  auto fail = [&](int code) { cudaFree(perm_dev); cudaFree(rep_dev); free_layer(L); return code; };
+#define TRY_OR_FAIL(expr)                                                 \
+  do {                                                                    \
+    cudaError_t e_ = (expr);                                              \
+    if (e_ != cudaSuccess) return fail(cuda_fail(e_, #expr));             \
+  } while (0)
+  const size_t wbytes = (size_t)d_ff * d * L->esz;
+  TRY_OR_FAIL(cudaMalloc(&L->wg_p, wbytes));
+  TRY_OR_FAIL(cudaMalloc(&L->wu_p, wbytes));
+  TRY_OR_FAIL(cudaMalloc(&L->wd_p, wbytes));
+  TRY_OR_FAIL(cudaMalloc(&L->w_rep, (size_t)(n_r ? 2 * n_r : 1) * d * L->esz));
+  TRY_OR_FAIL(cudaMalloc(&L->u, (size_t)(n_r ? n_r : 1) * sizeof(float)));
+  TRY_OR_FAIL(cudaMalloc(&L->b, (size_t)(n_r ? n_r : 1) * sizeof(float)));
+  TRY_OR_FAIL(cudaMalloc(&perm_dev, (size_t)d_ff * sizeof(int32_t)));
+  TRY_OR_FAIL(cudaMalloc(&rep_dev, (size_t)(n_r ? n_r : 1) * sizeof(int32_t)));
+  TRY_OR_FAIL(cudaMemcpyAsync(perm_dev, neuron_perm, (size_t)d_ff * sizeof(int32_t),
+                              cudaMemcpyHostToDevice, st));
+  if (n_r)
+    TRY_OR_FAIL(cudaMemcpyAsync(rep_dev, rep_idx, (size_t)n_r * sizeof(int32_t),
+                                cudaMemcpyHostToDevice, st));
+  rc = cfg->dtype == CMOE_BF16 ? pack_weights<bf16>(L, w_gate, w_up, w_down, perm_dev, rep_dev, st)
+                               : pack_weights<float>(L, w_gate, w_up, w_down, perm_dev, rep_dev, st);
+  if (rc != CMOE_OK) return fail(rc);
+  rc = upload_gate_params(L, gate_scale_u, select_bias_b, st);
+  if (rc != CMOE_OK) return fail(rc);
+  rc = finish_layer(L, st);
+  if (rc != CMOE_OK) return fail(rc);
+  TRY_OR_FAIL(cudaStreamSynchronize(st));
+#undef TRY_OR_FAIL
+  cudaFree(perm_dev); cudaFree(rep_dev);
+  *out_layer = L;
+  return CMOE_OK;
+}
+
+int cmoe_hier_create(int32_t n_outer, int32_t outer_top_k, const void* w_router,
+                     cmoe_layer* const* inner, int32_t max_tokens, void* stream,
+                     cmoe_layer** out_layer) {
+  if (!w_router || !inner || !out_layer) return arg_fail(CMOE_ERR_INVALID_ARG, "null argument");
+  *out_layer = nullptr;
+  if (n_outer <= 0 || n_outer > kMaxOuter || outer_top_k <= 0 || outer_top_k > n_outer ||
+      outer_top_k > kMaxTopK || max_tokens <= 0)
+    return arg_fail(CMOE_ERR_INVALID_ARG, "outer expert count / top-k out of range");
+  for (int i = 0; i < n_outer; ++i) {
+    if (!inner[i] || inner[i]->hier) return arg_fail(CMOE_ERR_INVALID_ARG, "inner layer invalid");
+    const cmoe_config &a = inner[0]->cfg, &c = inner[i]->cfg;
+    if (a.d_model != c.d_model || a.d_ff != c.d_ff || a.n_experts != c.n_experts ||
+        a.n_shared != c.n_shared || a.top_k != c.top_k || a.dtype != c.dtype)
+      return arg_fail(CMOE_ERR_INVALID_ARG, "inner layers differ in configuration");
+    for (int k = 0; k < i; ++k)
+      if (inner[k] == inner[i]) return arg_fail(CMOE_ERR_INVALID_ARG, "inner layer listed twice");
+  }
+  int rc = check_device();
+  if (rc != CMOE_OK) return rc;
+  cmoe_layer* L = new (std::nothrow) cmoe_layer();
+  if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "out of host memory");
+  L->cfg = inner[0]->cfg; L->cfg.max_tokens = max_tokens;
+  L->m = inner[0]->m; L->n_r = inner[0]->n_r; L->esz = inner[0]->esz;
+  L->n_outer = n_outer; L->outer_k = outer_top_k; L->hier = true;
+  cudaGetDevice(&L->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t d = L->cfg.d_model, d_ff = L->cfg.d_ff, nr = L->n_r, esz = L->esz;
+  const size_t wbytes = d_ff * d * esz, rep_bytes = 2 * nr * d * esz;
+  auto fail = [&](int code) { free_layer(L); return code; };
+#define TRY_OR_FAIL(expr)                                                 \
+  do {                                                                    \
+    cudaError_t e_ = (expr);                                              \
+    if (e_ != cudaSuccess) return fail(cuda_fail(e_, #expr));             \
+  } while (0)
+  TRY_OR_FAIL(cudaMalloc(&L->wg_p, wbytes * n_outer));
+  TRY_OR_FAIL(cudaMalloc(&L->wu_p, wbytes * n_outer));
+  TRY_OR_FAIL(cudaMalloc(&L->wd_p, wbytes * n_outer));
+  TRY_OR_FAIL(cudaMalloc(&L->w_rep, (rep_bytes ? rep_bytes : 16) * n_outer));
+  TRY_OR_FAIL(cudaMalloc(&L->w_router, (size_t)n_outer * d * esz));
+  TRY_OR_FAIL(cudaMalloc(&L->u, (nr ? nr : 1) * n_outer * sizeof(float)));
+  TRY_OR_FAIL(cudaMalloc(&L->b, (nr ? nr : 1) * n_outer * sizeof(float)));
+  for (int i = 0; i < n_outer; ++i) {
+    const cmoe_layer* S = inner[i];
+    const auto D2D = cudaMemcpyDeviceToDevice;
+    TRY_OR_FAIL(cudaMemcpyAsync((char*)L->wg_p + i * wbytes, S->wg_p, wbytes, D2D, st));
+    TRY_OR_FAIL(cudaMemcpyAsync((char*)L->wu_p + i * wbytes, S->wu_p, wbytes, D2D, st));
+    TRY_OR_FAIL(cudaMemcpyAsync((char*)L->wd_p + i * wbytes, S->wd_p, wbytes, D2D, st));
+    if (nr) {
+      TRY_OR_FAIL(cudaMemcpyAsync((char*)L->w_rep + i * rep_bytes, S->w_rep, rep_bytes, D2D, st));
+      TRY_OR_FAIL(cudaMemcpyAsync(L->u + i * nr, S->u, nr * sizeof(float), D2D, st));
+      TRY_OR_FAIL(cudaMemcpyAsync(L->b + i * nr, S->b, nr * sizeof(float), D2D, st));
+    }
+  }
+  TRY_OR_FAIL(cudaMemcpyAsync(L->w_router, w_router, (size_t)n_outer * d * esz,
+                              cudaMemcpyDeviceToDevice, st));
+  rc = finish_layer(L, st);
+  if (rc != CMOE_OK) return fail(rc);
+  TRY_OR_FAIL(cudaStreamSynchronize(st));
+#undef TRY_OR_FAIL
+  for (int i = 0; i < n_outer; ++i) free_layer(inner[i]);
+  *out_layer = L;
+  return CMOE_OK;
+}
+
+int cmoe_ffn_forward(cmoe_layer* L, const void* x, int32_t T, void* out, void* stream) {
+  if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "null layer");
+  if (T < 0) return arg_fail(CMOE_ERR_INVALID_ARG, "negative token count");
+  if (T == 0) { L->last_T = 0; L->launches = 0; return CMOE_OK; }
+  if (!x || !out) return arg_fail(CMOE_ERR_INVALID_ARG, "null x / out");
+  if (T > L->cfg.max_tokens) return arg_fail(CMOE_ERR_CAPACITY, "T exceeds max_tokens");
+  if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(out)) & 15)
+    return arg_fail(CMOE_ERR_INVALID_ARG, "x / out must be 16-byte aligned");
+  {
+    const char *xa = (const char*)x, *oa = (const char*)out;
+    const size_t bytes = (size_t)T * L->cfg.d_model * L->esz;
+    if (xa < oa + bytes && oa < xa + bytes) return arg_fail(CMOE_ERR_INVALID_ARG, "x and out overlap");
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  L->last_stream = st;
+  L->last_T = T;
+  return L->cfg.dtype == CMOE_BF16 ? forward_impl<bf16>(L, (const bf16*)x, T, (bf16*)out, st)
+                                   : forward_impl<float>(L, (const float*)x, T, (float*)out, st);
+}
+
+int cmoe_layer_set_gate_params(cmoe_layer* L, const float* u, const float* b, void* stream) {
+  if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "null layer");
+  return upload_gate_params(L, u, b, static_cast<cudaStream_t>(stream));
+}
+
+int cmoe_layer_set_gemm_path(cmoe_layer* L, int32_t path) {
+  if (!L || path < 0 || path > 2) return arg_fail(CMOE_ERR_INVALID_ARG, "gemm path");
+  if (path == 2 && !L->umma_ok)
+    return arg_fail(CMOE_ERR_INVALID_ARG, "tensor-core path not available for this layer");
+  L->gemm_path = path;
+  return CMOE_OK;
+}
+
+int cmoe_layer_dims(const cmoe_layer* L, int32_t* n_routed_groups, int32_t* top_k, int32_t* n_outer,
+                    int32_t* outer_top_k) {
+  if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "null layer");
+  if (n_routed_groups) *n_routed_groups = L->n_outer * L->n_r;
+  if (top_k) *top_k = L->cfg.top_k;
+  if (n_outer) *n_outer = L->hier ? L->n_outer : 0;
+  if (outer_top_k) *outer_top_k = L->hier ? L->outer_k : 0;
+  return CMOE_OK;
+}
+
+int cmoe_get_routing(cmoe_layer* L, float* keys, float* scores, int32_t* topk_idx, float* topk_gate,
+                     int32_t* counts, int32_t* offsets, int32_t* row_token, int32_t* row_of,
+                     int32_t* outer_idx, float* outer_w, int32_t* outer_row_token) {
+  if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "null layer");
+  cudaStream_t st = L->last_stream;
+  const size_t T = L->last_T, R = T * (L->hier ? L->outer_k : 1), P = R * L->cfg.top_k;
+  const size_t nr = L->n_r, G = (size_t)L->n_outer * nr;
+  const auto D2H = cudaMemcpyDeviceToHost;
+  if (T > 0 && nr > 0) {
+    if (keys) CU_TRY(cudaMemcpyAsync(keys, L->keys, R * nr * 4, D2H, st));
+    if (scores) CU_TRY(cudaMemcpyAsync(scores, L->scores, R * nr * 4, D2H, st));
+    if (topk_idx && P) CU_TRY(cudaMemcpyAsync(topk_idx, L->topk_idx, P * 4, D2H, st));
+    if (topk_gate && P) CU_TRY(cudaMemcpyAsync(topk_gate, L->topk_gate, P * 4, D2H, st));
+    if (counts) CU_TRY(cudaMemcpyAsync(counts, L->counts, G * 4, D2H, st));
+    if (offsets) CU_TRY(cudaMemcpyAsync(offsets, L->offsets, (G + 1) * 4, D2H, st));
+    if (row_token && P) CU_TRY(cudaMemcpyAsync(row_token, L->row_token, P * 4, D2H, st));
+    if (row_of && P) CU_TRY(cudaMemcpyAsync(row_of, L->row_of, P * 4, D2H, st));
+  }
+  if (T > 0 && L->hier) {
+    if (outer_idx) CU_TRY(cudaMemcpyAsync(outer_idx, L->outer_idx, R * 4, D2H, st));
+    if (outer_w) CU_TRY(cudaMemcpyAsync(outer_w, L->outer_w, R * 4, D2H, st));
+    if (outer_row_token) CU_TRY(cudaMemcpyAsync(outer_row_token, L->outer_row_token, R * 4, D2H, st));
+  }
+  CU_TRY(cudaStreamSynchronize(st));
+  return CMOE_OK;
+}
+
+int cmoe_layer_status(cmoe_layer* L, int32_t* device_error_word) {
+  if (!L || !device_error_word) return arg_fail(CMOE_ERR_INVALID_ARG, "null argument");
+  CU_TRY(cudaMemcpyAsync(device_error_word, L->err_word, 4, cudaMemcpyDeviceToHost, L->last_stream));
+  CU_TRY(cudaStreamSynchronize(L->last_stream));
+  return *device_error_word ? CMOE_ERR_DEVICE_TIMEOUT : CMOE_OK;
+}
+
+int cmoe_layer_launch_count(const cmoe_layer* L, int32_t* n_launches) {
+  if (!L || !n_launches) return arg_fail(CMOE_ERR_INVALID_ARG, "null argument");
+  *n_launches = L->launches;
+  return CMOE_OK;
+}
+
+int cmoe_layer_destroy(cmoe_layer* L) {
+  if (!L) return CMOE_OK;
+  free_layer(L);
+  return CMOE_OK;
+}
+
+int64_t cmoe_token_permute_scratch_bytes(int32_t n_rows, int32_t n_groups) {
+  if (n_rows < 0 || n_groups <= 0) return 0;
+  return permute_scratch_bytes(n_rows, n_groups);
+}
+
+int cmoe_token_permute(const int32_t* topk_idx, int32_t n_rows, int32_t n_k, int32_t n_groups,
+                       int32_t* counts, int32_t* offsets, int32_t* row_token, int32_t* row_of,
+                       void* scratch, int64_t scratch_bytes, void* stream) {
+  if (n_rows < 0 || n_k < 0 || n_k > kMaxTopK || n_groups <= 0 || n_groups > kPermMaxGroups)
+    return arg_fail(CMOE_ERR_INVALID_ARG, "permute: size out of range");
+  if (!counts || !offsets || ((int64_t)n_rows * n_k > 0 && (!topk_idx || !row_token || !row_of)))
+    return arg_fail(CMOE_ERR_INVALID_ARG, "permute: null pointer");
+  if (n_rows > kPermChunk) {
+    if (!scratch || (reinterpret_cast<uintptr_t>(scratch) & 255))
+      return arg_fail(CMOE_ERR_INVALID_ARG, "permute: scratch null or not 256-byte aligned");
+    if (scratch_bytes < permute_scratch_bytes(n_rows, n_groups))
+      return arg_fail(CMOE_ERR_CAPACITY, "permute: scratch too small");
+  }
+  launch_token_permute(topk_idx, n_rows, n_k, n_groups, counts, offsets, row_token, row_of,
+                       static_cast<int32_t*>(scratch), static_cast<cudaStream_t>(stream));
+  CU_TRY(cudaGetLastError());
+  return CMOE_OK;
+}
+
+const char* cmoe_status_string(int status) {
+  switch (status) {
+    case CMOE_OK: return "ok";
+    case CMOE_ERR_INVALID_ARG: return "invalid argument";
+    case CMOE_ERR_BAD_PARTITION: return "neuron partition is not a permutation into equal experts";
+    case CMOE_ERR_BAD_REP: return "representative neuron outside its expert";
+    case CMOE_ERR_CAPACITY: return "capacity exceeded";
+    case CMOE_ERR_CUDA: return "CUDA error";
+    case CMOE_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case CMOE_ERR_UNSUPPORTED: return "unsupported device";
+    default: return "unknown status";
+  }
+}
+
+const char* cmoe_last_error(void) { return g_last_error; }
+
+}  // extern "C"
