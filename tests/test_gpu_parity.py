@@ -1,0 +1,139 @@
+"""-m gpu: the CUDA path, called through the C-ABI, against the CPU oracle on the
+same seeded inputs.  Small shapes keep each expert's ragged tile tails (m = 1376,
+448, 864 ...) and token counts that are not multiples of any tile."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+from oracle import cmoe_oracle as oracle
+from paper_2502_04416_b200 import binding, workloads as wl
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+PATHS = [binding.GEMM_SIMT, binding.GEMM_AUTO]
+PATH_IDS = ["simt", "auto"]
+
+
+def _inputs(name, d_model=None, tokens=None, m=None, n_outer=None, seed=None):
+    w = wl.WORKLOADS[name]
+    if d_model is not None:
+        w = wl.shrunk(w, d_model=d_model, tokens=tokens, m=m, n_outer=n_outer)
+    if seed is not None:
+        w = dataclasses.replace(w, seed=seed)
+    return wl.make_inputs(w)
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_c1_tiny_fp32(path):
+    inp = _inputs("c1_tiny_fp32")
+    lay = inp.layers[0]
+    layer = parity.gpu_layer(lay, 64)
+    layer.set_gemm_path(path)
+    st = parity.check_plain_layer(layer, lay, inp.x)
+    assert st["differing"] == 0
+    assert st["max_rel"] < 1e-4 and st["mean_rel"] < 1e-4      # fp32 end to end
+    layer.destroy()
+
+
+SMALL = [
+    ("c2_llama2_7b", 256, None, (1, 16, 77, 300)),
+    ("c3_llama3_8b", 256, None, (33, 517)),
+    ("c5_skew_13b", 320, None, (129, 700)),
+    ("c2_llama2_7b", 512, 200, (1000,)),       # m = 200: neither a multiple of 16 nor of 64
+]
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+@pytest.mark.parametrize("name,d,m,tokens", SMALL, ids=[f"{s[0]}-d{s[1]}-m{s[2]}" for s in SMALL])
+def test_small_shapes(name, d, m, tokens, path):
+    inp = _inputs(name, d_model=d, tokens=tokens, m=m)
+    lay = inp.layers[0]
+    if wl.WORKLOADS[name].zipf_s:
+        rng = np.random.default_rng(1)
+        lay.select_bias_b = rng.normal(scale=0.05, size=lay.shape.n_routed).astype(np.float32)
+        lay.gate_scale_u = rng.normal(scale=0.5, size=lay.shape.n_routed).astype(np.float32)
+    layer = parity.gpu_layer(lay, max(tokens))
+    layer.set_gemm_path(path)
+    for t in tokens:
+        st = parity.check_plain_layer(layer, lay, inp.x[:t])
+        assert st["differing"] <= st["near_tie"]
+    layer.destroy()
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_hierarchical_small(path):
+    inp = _inputs("c4_hier_8x7b", d_model=256, tokens=(257,), m=224)
+    inners = [parity.gpu_layer(lay, 8) for lay in inp.layers]
+    layer = binding.Layer.create_hier(parity.to_device(inp.w_router, "bf16"), inners, 2, 300)
+    layer.set_gemm_path(path)
+    st = parity.check_hier_layer(layer, inp, inp.x)
+    assert st["differing"] <= st["near_tie"]
+    st = parity.check_hier_layer(layer, inp, inp.x[:3])          # most outer experts empty
+    layer.destroy()
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_degenerate_structures(path):
+    base = wl.shrunk(wl.WORKLOADS["c2_llama2_7b"], d_model=128, tokens=(70,), m=80)
+    for n_shared, top_k in [(2, 0), (0, 2), (2, 6), (8, 0), (0, 8)]:
+        shape = dataclasses.replace(base.shape, n_shared=n_shared, top_k=top_k)
+        inp = wl.make_inputs(dataclasses.replace(base, shape=shape))
+        lay = inp.layers[0]
+        layer = parity.gpu_layer(lay, 70)
+        layer.set_gemm_path(path)
+        st = parity.check_plain_layer(layer, lay, inp.x)
+        if top_k == shape.n_routed:           # every expert on with unit gates: the dense FFN
+            import torch
+            got = parity.to_host(layer.forward(parity.to_device(inp.x, "bf16")))
+            torch.cuda.synchronize()
+            parity.check_output(got, oracle.dense_ffn(inp.x, lay.w_gate, lay.w_up, lay.w_down))
+        layer.destroy()
+
+
+def test_call_contract():
+    import torch
+    inp = _inputs("c2_llama2_7b", d_model=128, tokens=(40,), m=48)
+    lay = inp.layers[0]
+    layer = parity.gpu_layer(lay, 32)
+    x = parity.to_device(inp.x, "bf16")
+    out = torch.full_like(x, 7.0)
+    layer.forward(x[:0], out[:0])                                 # T = 0: no-op
+    torch.cuda.synchronize()
+    assert float(out.float().min()) == 7.0
+    with pytest.raises(binding.CmoeError) as e:
+        layer.forward(x, out)                                     # 40 > max_tokens
+    assert e.value.status == -4
+    with pytest.raises(binding.CmoeError) as e:
+        layer.forward(x[:8], x[:8])                               # aliasing
+    assert e.value.status == -1
+    a = layer.forward(x[:32]).clone()
+    b = layer.forward(x[:32]).clone()
+    torch.cuda.synchronize()
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))  # run-to-run bit identical
+    # gate parameters can be replaced after create
+    u = np.linspace(-1, 1, lay.shape.n_routed).astype(np.float32)
+    layer.set_gate_params(gate_scale_u=u)
+    lay.gate_scale_u = u
+    parity.check_plain_layer(layer, lay, inp.x[:32])
+    layer.destroy()
+
+
+@pytest.mark.parametrize("n_rows,n_k,n_groups", [(1, 2, 6), (255, 2, 6), (256, 4, 28), (257, 4, 28),
+                                                 (5000, 2, 56), (16384, 4, 14), (3000, 8, 1000),
+                                                 (700, 1, 3), (40, 0, 5)])
+def test_token_permute_standalone(n_rows, n_k, n_groups):
+    import torch
+    rng = np.random.default_rng(n_rows + n_groups)
+    sel = np.stack([rng.permutation(n_groups)[:n_k] for _ in range(n_rows)]).astype(np.int32)
+    if n_groups > 4 and n_k:
+        sel[sel == 2] = 3 if n_k == 1 else sel[sel == 2]          # an empty group when n_k == 1
+    dev = torch.from_numpy(sel).cuda() if n_k else torch.zeros((n_rows, 0), dtype=torch.int32).cuda()
+    cnt, off, row_token, row_of = binding.token_permute(dev, n_groups)
+    torch.cuda.synchronize()
+    w_cnt, w_off, w_row_token, w_row_of = oracle.token_permutation(sel, n_groups)
+    np.testing.assert_array_equal(cnt.cpu().numpy(), w_cnt)
+    np.testing.assert_array_equal(off.cpu().numpy(), w_off)
+    np.testing.assert_array_equal(row_token.cpu().numpy(), w_row_token)
+    np.testing.assert_array_equal(row_of.cpu().numpy(), w_row_of)
