@@ -1,0 +1,358 @@
+#!/usr/bin/env python
+"""Benchmark of the restructured-FFN MoE forward on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--workload NAME --tokens T]
+    python bench.py --impl reference ...        # the CPU oracle, as it stands, on host cores
+
+A step is one pass of the whole forward (router, histogram/permute, shared and
+routed SwiGLU expert GEMMs, combine) over one batch of T synthetic tokens.  The
+path shards by tokens with no exchange, so N GPUs run N independent replicas
+("replicas only"): value = N*T*K / max-over-ranks device time.  Prints ONE JSON
+line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2502_04416_b200 import workloads as wl  # noqa: E402
+
+METRIC = "moe_ffn_layer_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS if k in p} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS, source="fallback")
+
+
+# ------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.gpu = [], None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------- CPU oracle arm
+def host_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return len(os.sched_getaffinity(0))
+
+
+def oracle_step(inputs: wl.WorkloadInputs, x: np.ndarray):
+    """One oracle forward on x (the oracle as it stands: fp64 numpy)."""
+    from oracle import cmoe_oracle as oracle
+    w = inputs.workload
+    s = w.shape
+
+    def kw(lay):
+        return dict(w_gate=lay.w_gate, w_up=lay.w_up, w_down=lay.w_down,
+                    neuron_perm=lay.neuron_perm, rep_idx=lay.rep_idx, n_experts=s.n_experts,
+                    n_shared=s.n_shared, top_k=s.top_k, gate_scale_u=lay.gate_scale_u,
+                    select_bias_b=lay.select_bias_b)
+    if w.n_outer:
+        return oracle.hier_forward(x, inputs.w_router, w.outer_top_k, [kw(l) for l in inputs.layers])[0]
+    return oracle.cmoe_layer_forward(x, **kw(inputs.layers[0]))[0]
+
+
+def time_oracle(inputs, x, sample_tokens: int, repeats: int = 1):
+    xs = x[:sample_tokens]
+    oracle_step(inputs, xs[:min(8, len(xs))])              # import + BLAS warm-up
+    t0 = time.perf_counter()
+    for _ in range(repeats):
+        oracle_step(inputs, xs)
+    dt = (time.perf_counter() - t0) / repeats
+    return len(xs) / dt, dt
+
+
+def load_select_bias(name: str):
+    path = os.path.join(ROOT, "tests", "golden", f"{name}_select_bias.txt")
+    if not os.path.exists(path):
+        return None
+    return np.array([float(l) for l in open(path) if l.strip() and not l.startswith("#")],
+                    dtype=np.float32)
+
+
+def prepare_inputs(name: str):
+    w = wl.WORKLOADS[name]
+    inputs = wl.make_inputs(w)
+    if w.zipf_s:
+        b = load_select_bias(name)
+        if b is not None:
+            inputs.layers[0].select_bias_b = b
+    return inputs
+
+
+# ------------------------------------------------------------------ GPU arm
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2502_04416_b200 import binding
+    from paper_2502_04416_b200 import torch_io
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    binding.load()
+
+    inputs = prepare_inputs(args.workload)
+    w = inputs.workload
+    s = w.shape
+    T = args.tokens or w.t_max
+    x_host = inputs.x[:T]
+    layer = torch_io.layer_from_workload(inputs, T)
+    x = torch_io.to_device(x_host, s.dtype)
+    out = torch.empty_like(x)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        """K steps between CUDA events on the launching stream; max over ranks."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        barrier()
+        ms = torch.tensor([e0.elapsed_time(e1)], device="cuda")
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    # ---- device-resident throughput, with per-stage events for the roofline
+    layer.enable_stage_timing(min(args.steps, 4096))
+    for _ in range(args.warmup):
+        layer.forward(x, out)
+    layer.enable_stage_timing(min(args.steps, 4096))          # reset the ring after warm-up
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms_total = timed(lambda: layer.forward(x, out), args.steps)
+    clocks = sampler.stop()
+    stage_ms, n_cov = layer.stage_times()
+    launches = layer.launch_count() * args.steps
+    assert layer.status() == 0, "device-side wait timed out"
+    layer.enable_stage_timing(0)
+    value = world * T * args.steps / (ms_total * 1e-3)
+
+    # ---- end to end through the public call with host buffers
+    x_pin = torch.empty(x.shape, dtype=x.dtype).pin_memory()
+    x_pin.copy_(x.cpu())
+    out_pin = torch.empty(x.shape, dtype=x.dtype).pin_memory()
+
+    def e2e_step():
+        x.copy_(x_pin, non_blocking=True)
+        layer.forward(x, out)
+        out_pin.copy_(out, non_blocking=True)
+    for _ in range(max(args.warmup, 3)):
+        e2e_step()
+    e2e_ms = timed(e2e_step, args.steps)
+    io_bytes = T * s.d_model * s.elem_bytes
+
+    # ---- dense cuBLAS FFN of the same shape (comparison run, never the product path)
+    dense = None
+    if rank == 0 and not w.n_outer:
+        lay = inputs.layers[0]
+        wg, wu, wd = (torch_io.to_device(a, s.dtype) for a in (lay.w_gate, lay.w_up, lay.w_down))
+        F = torch.nn.functional
+
+        def dense_step():
+            return F.linear(F.silu(F.linear(x, wg)) * F.linear(x, wu), wd)
+        for _ in range(3):
+            dense_step()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(args.steps):
+            dense_step()
+        e1.record()
+        torch.cuda.synchronize()
+        dms = e0.elapsed_time(e1) / args.steps
+        dense = {"kind": "torch F.linear x3 + silu*mul (cuBLAS), same d and d_ff",
+                 "ms_per_step": dms, "value": T / (dms * 1e-3), "unit": UNIT}
+        del wg, wu, wd
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return None
+
+    # ---- roofline of the dominant kernel stage
+    peaks = load_peaks()
+    touched = s.n_routed
+    if not w.n_outer and T * s.top_k < 64 * s.n_routed:
+        r = layer.routing(T, s.n_routed)
+        touched = int((r["counts"] > 0).sum())
+    mult = w.outer_top_k if w.n_outer else 1
+    flops = mult * T * 6 * s.d_model * s.m * (s.n_shared + s.top_k)
+    w_bytes = (w.n_outer if w.n_outer else 1) * (s.n_shared + touched) * s.expert_weight_bytes()
+    alg_bytes = w_bytes + 2 * T * s.d_model * s.elem_bytes
+    gemm_ms = (stage_ms[2] + stage_ms[3]) / max(n_cov, 1)
+    step_ms = ms_total / args.steps
+    t_tensor = flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
+    if t_tensor >= t_hbm:
+        ach = flops / (gemm_ms * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": ach / peaks["bf16_tflops"],
+                "frac_of_sustained": ach / peaks["bf16_tflops_sustained"]}
+    else:
+        ach = alg_bytes / (gemm_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / peaks["hbm_gbs"]}
+    roof.update({"kernel": "expert GEMMs (gate/up + SwiGLU, down)", "kernel_ms": gemm_ms,
+                 "peak_source": peaks["source"], "traffic": None,
+                 "whole_step_frac": (t_tensor if t_tensor >= t_hbm else t_hbm) / (step_ms * 1e-3),
+                 "stage_ms": {n: v / max(n_cov, 1) for n, v in zip(binding.STAGE_NAMES, stage_ms)}})
+
+    # ---- CPU baseline: the oracle on a bounded sample, on this machine's host cores
+    sample = args.cpu_sample_tokens
+    cpu_v, cpu_dt = time_oracle(inputs, x_host, min(sample, T))
+    cpu = {"value": cpu_v, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+           "sample": f"first {min(sample, T)} tokens of the same workload, one pass, {cpu_dt:.2f} s"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": s.dtype, "data": "synthetic",
+        "config": {"workload": f"{w.name} T={T}", "note": w.note, "d_model": s.d_model,
+                   "d_ff": s.d_ff, "experts": f"S{s.n_shared}A{s.top_k}E{s.n_experts}",
+                   "tokens_per_step": T, "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": "weights (%.0f MB) exceed the 126 MB L2" % (w_bytes / 1e6)},
+        "e2e": {"value": world * T * args.steps / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": io_bytes, "d2h_bytes_per_step": io_bytes},
+        "gpu_launches": launches, "clocks": clocks, "roofline": roof, "cpu_baseline": cpu,
+        "dense_cublas": dense,
+    }
+    if world > 1:
+        dist.destroy_process_group()
+    return line
+
+
+# ------------------------------------------------------------ reference arm
+def run_reference(args):
+    """The CPU oracle, unmodified, timed on the host cores on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return None
+    inputs = prepare_inputs(args.workload)
+    w = inputs.workload
+    T = args.tokens or w.t_max
+    sample = min(args.cpu_sample_tokens, T)
+    xs = inputs.x[:sample]
+    for _ in range(args.warmup):
+        oracle_step(inputs, xs[:min(16, sample)])
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(inputs, xs)
+    dt = time.perf_counter() - t0
+    v = sample * args.steps / dt
+    s = w.shape
+    desc = f"first {sample} tokens of the workload per step"
+    return {
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{w.name} T={T}", "sample": desc, "d_model": s.d_model, "d_ff": s.d_ff,
+                   "experts": f"S{s.n_shared}A{s.top_k}E{s.n_experts}"},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+                         "sample": desc},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default="c2_llama2_7b", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--tokens", type=int, default=0, help="tokens per step (default: the workload's largest T)")
+    ap.add_argument("--cpu-sample-tokens", type=int, default=256)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        line = run_reference(args)
+    else:
+        args.warmup = max(args.warmup, 3)
+        line = run_gpu(args)
+    if line is not None:
+        print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    main()

@@ -145,6 +145,18 @@ int cmoe_layer_status(cmoe_layer* layer, int32_t* device_error_word);
 /* Number of this library's kernels the last forward launched. */
 int cmoe_layer_launch_count(const cmoe_layer* layer, int32_t* n_launches);
 
+/* Per-stage device timing with CUDA events on the forward's stream.  ring_steps > 0
+ * creates a ring of events covering that many forwards (0 switches timing off);
+ * while on, every forward records CMOE_N_STAGES+1 events and allocates nothing.
+ * Stages: 0 routing (top-level router and its permutation for hierarchical layers,
+ * analytical router + gates), 1 histogram/scan/permute + row gather, 2 gate/up GEMM
+ * with the SwiGLU epilogue, 3 down GEMM, 4 combine.
+ * cmoe_layer_stage_times synchronises the last stream and returns, per stage, the
+ * summed milliseconds over the last n_steps forwards held in the ring. */
+#define CMOE_N_STAGES 5
+int cmoe_layer_enable_stage_timing(cmoe_layer* layer, int32_t ring_steps);
+int cmoe_layer_stage_times(cmoe_layer* layer, float* ms_sum /*[CMOE_N_STAGES]*/, int32_t* n_steps);
+
 int cmoe_layer_destroy(cmoe_layer* layer);
 
 /* Stand-alone token histogram / exclusive scan / stable permutation: the

@@ -14,11 +14,14 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcmoe.so"
 
 CMOE_BF16, CMOE_FP32 = 0, 1
 GEMM_AUTO, GEMM_SIMT, GEMM_TENSOR = 0, 1, 2
+N_STAGES = 5
+STAGE_NAMES = ["route", "permute", "gemm1_swiglu", "gemm2_down", "combine"]
 
 EXPORTS = [
     "cmoe_layer_create", "cmoe_hier_create", "cmoe_ffn_forward", "cmoe_layer_set_gate_params",
     "cmoe_layer_set_gemm_path", "cmoe_layer_dims", "cmoe_get_routing", "cmoe_layer_status",
-    "cmoe_layer_launch_count", "cmoe_layer_destroy", "cmoe_token_permute_scratch_bytes",
+    "cmoe_layer_launch_count", "cmoe_layer_enable_stage_timing", "cmoe_layer_stage_times",
+    "cmoe_layer_destroy", "cmoe_token_permute_scratch_bytes",
     "cmoe_token_permute", "cmoe_status_string", "cmoe_last_error",
 ]
 
@@ -59,6 +62,8 @@ def load() -> C.CDLL:
     lib.cmoe_layer_status.argtypes = [vp, C.POINTER(i32)]
     lib.cmoe_layer_launch_count.argtypes = [vp, C.POINTER(i32)]
     lib.cmoe_layer_destroy.argtypes = [vp]
+    lib.cmoe_layer_enable_stage_timing.argtypes = [vp, i32]
+    lib.cmoe_layer_stage_times.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(i32)]
     lib.cmoe_token_permute_scratch_bytes.argtypes = [i32, i32]
     lib.cmoe_token_permute_scratch_bytes.restype = i64
     lib.cmoe_token_permute.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, i64, vp]
@@ -203,6 +208,17 @@ class Layer:
         w = C.c_int32()
         _check(load().cmoe_layer_launch_count(self._h, C.byref(w)), "cmoe_layer_launch_count")
         return w.value
+
+    def enable_stage_timing(self, ring_steps: int) -> None:
+        _check(load().cmoe_layer_enable_stage_timing(self._h, ring_steps),
+               "cmoe_layer_enable_stage_timing")
+
+    def stage_times(self):
+        """(per-stage summed milliseconds [N_STAGES], forwards covered)."""
+        ms = (C.c_float * N_STAGES)()
+        n = C.c_int32()
+        _check(load().cmoe_layer_stage_times(self._h, ms, C.byref(n)), "cmoe_layer_stage_times")
+        return [float(v) for v in ms], n.value
 
     def destroy(self) -> None:
         if self._h and self._h.value:

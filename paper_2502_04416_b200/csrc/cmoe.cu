@@ -95,6 +95,11 @@ struct cmoe_layer {
   int last_T = 0;
   int launches = 0;
 
+  // optional per-stage CUDA-event timing: ring of (kStages + 1) events per forward
+  std::vector<cudaEvent_t> ev;
+  int ev_ring = 0;
+  long long ev_count = 0;
+
   int n_groups_total() const { return n_outer + n_outer * n_r; }
   int shared_width() const { return cfg.n_shared * m; }
 };
@@ -103,6 +108,7 @@ namespace {
 
 void free_layer(cmoe_layer* L) {
   if (!L) return;
+  for (cudaEvent_t e : L->ev) cudaEventDestroy(e);
   umma_plan_destroy(&L->umma);
   cudaFree(L->wg_p); cudaFree(L->wu_p); cudaFree(L->wd_p); cudaFree(L->w_rep);
   cudaFree(L->w_router); cudaFree(L->u); cudaFree(L->b); cudaFree(L->gs); cudaFree(L->ws);
@@ -269,6 +275,9 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   const int row_vec = d * (int)sizeof(T) / 16;
   int launches = 0;
   const T* xo = x;
+  cudaEvent_t* ev = L->ev_ring ? &L->ev[(size_t)(L->ev_count % L->ev_ring) * (CMOE_N_STAGES + 1)] : nullptr;
+  auto mark = [&](int i) { if (ev) cudaEventRecord(ev[i], st); };
+  mark(0);
 
   if (L->hier) {
     outer_router_kernel<T><<<(n_tok + 7) / 8, 256, 0, st>>>(x, n_tok, d, L->n_outer, L->outer_k,
@@ -295,8 +304,11 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
     else CMOE_ROUTER(64);
 #undef CMOE_ROUTER
     ++launches;
+    mark(1);
     launches += launch_token_permute(L->topk_idx, R, n_k, G, L->counts, L->offsets, L->row_token,
                                      L->row_of, L->perm_scratch, st);
+  } else {
+    mark(1);
   }
   plan_groups_kernel<<<1, 256, 0, st>>>(L->n_outer, n_r, n_tok, L->hier ? L->outer_off : nullptr,
                                         L->counts, L->offsets, L->gr);
@@ -306,9 +318,10 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
     ++launches;
   }
 
+  mark(2);
   const bool use_umma = L->umma_ok && L->gemm_path != 1;
   if (use_umma) {
-    const int n = umma_forward(&L->umma, xo, R, P, L->gr, L->err_word, st);
+    const int n = umma_forward(&L->umma, xo, R, P, L->gr, L->err_word, st, ev ? ev[3] : nullptr);
     if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     launches += n;
   } else {
@@ -321,6 +334,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
     a.c_shared = (T*)L->h_s; a.c_routed = (T*)L->h_r;
     dim3 g1((R + kSimtTile - 1) / kSimtTile, (max_w + kSimtTile - 1) / kSimtTile, L->n_groups_total());
     simt_gemm1_kernel<T><<<g1, 256, 0, st>>>(a);
+    mark(3);
     a.a_shared = (const T*)L->h_s; a.a_routed = (const T*)L->h_r;
     a.w_gate = (const T*)L->wd_p; a.w_up = nullptr;
     a.c_shared = (T*)L->y_s; a.c_routed = (T*)L->y_r;
@@ -329,12 +343,15 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
     launches += 2;
   }
 
+  mark(4);
   const int threads = d / 8 < 256 ? ((d / 8 + 31) / 32 * 32) : 256;
   combine_kernel<T><<<n_tok, threads, 0, st>>>(
       L->cfg.n_shared > 0 ? (const T*)L->y_s : nullptr, (const T*)L->y_r, L->topk_idx, L->topk_gate,
       L->row_of, L->hier ? L->outer_row_of : nullptr, L->hier ? L->outer_w : nullptr,
       L->hier ? L->outer_k : 1, n_k, d, out);
   ++launches;
+  mark(5);
+  if (ev) ++L->ev_count;
   CU_TRY(cudaGetLastError());
   L->launches = launches;
   return CMOE_OK;
@@ -558,6 +575,40 @@ int cmoe_layer_status(cmoe_layer* L, int32_t* device_error_word) {
 int cmoe_layer_launch_count(const cmoe_layer* L, int32_t* n_launches) {
   if (!L || !n_launches) return arg_fail(CMOE_ERR_INVALID_ARG, "null argument");
   *n_launches = L->launches;
+  return CMOE_OK;
+}
+
+int cmoe_layer_enable_stage_timing(cmoe_layer* L, int32_t ring_steps) {
+  if (!L || ring_steps < 0 || ring_steps > 4096) return arg_fail(CMOE_ERR_INVALID_ARG, "stage timing ring");
+  for (cudaEvent_t e : L->ev) cudaEventDestroy(e);
+  L->ev.clear();
+  L->ev_ring = 0;
+  L->ev_count = 0;
+  for (int i = 0; i < ring_steps * (CMOE_N_STAGES + 1); ++i) {
+    cudaEvent_t e;
+    CU_TRY(cudaEventCreate(&e));
+    L->ev.push_back(e);
+  }
+  L->ev_ring = ring_steps;
+  return CMOE_OK;
+}
+
+int cmoe_layer_stage_times(cmoe_layer* L, float* ms_sum, int32_t* n_steps) {
+  if (!L || !ms_sum || !n_steps) return arg_fail(CMOE_ERR_INVALID_ARG, "null argument");
+  for (int s = 0; s < CMOE_N_STAGES; ++s) ms_sum[s] = 0.0f;
+  *n_steps = 0;
+  if (!L->ev_ring) return CMOE_OK;
+  CU_TRY(cudaStreamSynchronize(L->last_stream));
+  const long long n = L->ev_count < L->ev_ring ? L->ev_count : L->ev_ring;
+  for (long long i = 0; i < n; ++i) {
+    cudaEvent_t* ev = &L->ev[(size_t)i * (CMOE_N_STAGES + 1)];
+    for (int s = 0; s < CMOE_N_STAGES; ++s) {
+      float ms = 0.0f;
+      CU_TRY(cudaEventElapsedTime(&ms, ev[s], ev[s + 1]));
+      ms_sum[s] += ms;
+    }
+  }
+  *n_steps = (int32_t)n;
   return CMOE_OK;
 }
 

@@ -20,7 +20,8 @@ inline int umma_plan_create(UmmaPlan*, const UmmaShape&, const GroupStatic*, int
                             const void*, const void*, void*, void*, void*, void*, void*) { return 1; }
 inline void umma_plan_destroy(UmmaPlan*) {}
 // Enqueues both expert GEMMs; returns the number of kernels launched or -1.
-inline int umma_forward(UmmaPlan*, const void*, int, int, const GroupRows*, int32_t*, cudaStream_t) {
+inline int umma_forward(UmmaPlan*, const void*, int, int, const GroupRows*, int32_t*, cudaStream_t,
+                        cudaEvent_t /*recorded between GEMM-1 and GEMM-2, may be null*/) {
   return -1;
 }
 

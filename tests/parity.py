@@ -16,34 +16,14 @@ from typing import Optional
 import numpy as np
 
 from oracle import cmoe_oracle as oracle
-from paper_2502_04416_b200 import binding, workloads as wl
+from paper_2502_04416_b200 import binding, torch_io, workloads as wl
 
 MARGIN = 1e-3
 OUT_MAX_REL = 2e-2
 OUT_MEAN_REL = 5e-3
 
 
-def to_device(a: np.ndarray, dtype: str):
-    import torch
-    if dtype == "bf16":
-        bits = wl.f32_to_bf16_bits(a)
-        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
-    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
-
-
-def to_host(t) -> np.ndarray:
-    import torch
-    if t.dtype == torch.bfloat16:
-        return wl.bf16_bits_to_f32(t.view(torch.int16).cpu().numpy().view(np.uint16))
-    return t.cpu().numpy()
-
-
-def gpu_layer(lay: wl.LayerInputs, max_tokens: int) -> binding.Layer:
-    s = lay.shape
-    return binding.Layer.create(
-        to_device(lay.w_gate, s.dtype), to_device(lay.w_up, s.dtype), to_device(lay.w_down, s.dtype),
-        lay.neuron_perm, lay.rep_idx, s.n_experts, s.n_shared, s.top_k, max_tokens,
-        lay.gate_scale_u, lay.select_bias_b)
+to_device, to_host, gpu_layer = torch_io.to_device, torch_io.to_host, torch_io.layer_from_inputs
 
 
 def oracle_kwargs(lay: wl.LayerInputs) -> dict:
