@@ -176,6 +176,34 @@ int cmoe_token_permute(const int32_t* topk_idx, int32_t n_rows, int32_t n_k, int
                        int32_t* counts, int32_t* offsets, int32_t* row_token, int32_t* row_of,
                        void* scratch, int64_t scratch_bytes, void* stream);
 
+/* cmoe_token_permute for callers that cannot allocate device memory.  (The paper has
+ * no counterpart; this is a packaging variant of the call above.)
+ *
+ * Who needs it: code that runs where cudaMalloc is unavailable or forbidden — inside a
+ * serving loop whose memory pool is frozen after start-up, in a plug-in that was handed
+ * only its input and output buffers, or in a process that must not touch the allocator
+ * because another component owns all of the device's free memory.  Such a caller cannot
+ * provide the `scratch` buffer of cmoe_token_permute, so this variant keeps the
+ * chunk-count matrix in a fixed 1 MiB array that is part of the library image: every GPU
+ * that loads the library holds that 1 MiB from load until the process exits.
+ *
+ * Same inputs, outputs and result as cmoe_token_permute.  Differences:
+ *   - limit: ceil(n_rows / 256) * n_groups <= CMOE_STATIC_PERMUTE_MAX_CELLS when
+ *     n_rows > 256 (e.g. 65,536 rows with 1024 groups, or 4 M rows with 16 groups);
+ *     larger problems are refused with CMOE_ERR_CAPACITY and nothing is launched.
+ *   - it calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - the first call on each device looks up the array's device address (a one-off,
+ *     host-side query made with that device current); make that first call outside any
+ *     stream capture.
+ *   - all calls on one device share the array.  Its contents carry over from call to
+ *     call, which is harmless (each call overwrites every cell before reading it), but two
+ *     calls that overlap in time on the GPU — different streams, or the same call from
+ *     two threads — race on it and return garbage: serialise them. */
+#define CMOE_STATIC_PERMUTE_MAX_CELLS 262144
+int cmoe_token_permute_static(const int32_t* topk_idx, int32_t n_rows, int32_t n_k,
+                              int32_t n_groups, int32_t* counts, int32_t* offsets,
+                              int32_t* row_token, int32_t* row_of, void* stream);
+
 const char* cmoe_status_string(int status);
 /* Text of the most recent error seen by this library on the calling thread. */
 const char* cmoe_last_error(void);

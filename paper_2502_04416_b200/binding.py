@@ -22,7 +22,7 @@ EXPORTS = [
     "cmoe_layer_set_gemm_path", "cmoe_layer_dims", "cmoe_get_routing", "cmoe_layer_status",
     "cmoe_layer_launch_count", "cmoe_layer_enable_stage_timing", "cmoe_layer_stage_times",
     "cmoe_layer_destroy", "cmoe_token_permute_scratch_bytes",
-    "cmoe_token_permute", "cmoe_status_string", "cmoe_last_error",
+    "cmoe_token_permute", "cmoe_token_permute_static", "cmoe_status_string", "cmoe_last_error",
 ]
 
 
@@ -67,6 +67,7 @@ def load() -> C.CDLL:
     lib.cmoe_token_permute_scratch_bytes.argtypes = [i32, i32]
     lib.cmoe_token_permute_scratch_bytes.restype = i64
     lib.cmoe_token_permute.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, i64, vp]
+    lib.cmoe_token_permute_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.cmoe_status_string.argtypes = [C.c_int]
     lib.cmoe_status_string.restype = C.c_char_p
     lib.cmoe_last_error.restype = C.c_char_p
@@ -252,4 +253,30 @@ def token_permute(topk_idx, n_groups: int, stream=None):
                                    offsets.data_ptr(), row_token.data_ptr(), row_of.data_ptr(),
                                    scratch.data_ptr(), nbytes, _stream_ptr(stream))
     _check(st, "cmoe_token_permute")
+    return counts, offsets, row_token[:n_rows * n_k], row_of
+
+
+STATIC_PERMUTE_MAX_CELLS = 262144
+
+
+def token_permute_static(topk_idx, n_groups: int, out=None, stream=None):
+    """cmoe_token_permute_static: the same permutation, for callers that may not allocate
+    device memory.  The library's built-in 1 MiB scratch array replaces the scratch buffer;
+    pass ``out`` = (counts, offsets, row_token, row_of) preallocated CUDA int32 tensors to
+    keep the call itself free of allocations (this wrapper allocates them otherwise).
+    Calls on one device share that array and must not overlap on the GPU."""
+    import torch
+    n_rows, n_k = topk_idx.shape
+    dev = topk_idx.device
+    if out is None:
+        out = (torch.empty(n_groups, dtype=torch.int32, device=dev),
+               torch.empty(n_groups + 1, dtype=torch.int32, device=dev),
+               torch.empty(max(n_rows * n_k, 1), dtype=torch.int32, device=dev),
+               torch.empty((n_rows, n_k), dtype=torch.int32, device=dev))
+    counts, offsets, row_token, row_of = out
+    st = load().cmoe_token_permute_static(topk_idx.data_ptr(), n_rows, n_k, n_groups,
+                                          counts.data_ptr(), offsets.data_ptr(),
+                                          row_token.data_ptr(), row_of.data_ptr(),
+                                          _stream_ptr(stream))
+    _check(st, "cmoe_token_permute_static")
     return counts, offsets, row_token[:n_rows * n_k], row_of

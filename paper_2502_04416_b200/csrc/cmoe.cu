@@ -8,6 +8,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -638,6 +639,64 @@ int cmoe_token_permute(const int32_t* topk_idx, int32_t n_rows, int32_t n_k, int
   }
   launch_token_permute(topk_idx, n_rows, n_k, n_groups, counts, offsets, row_token, row_of,
                        static_cast<int32_t*>(scratch), static_cast<cudaStream_t>(stream));
+  CU_TRY(cudaGetLastError());
+  return CMOE_OK;
+}
+
+}  // extern "C" (re-opened below)
+
+// ---------------------------------------------------------------------------
+// Token permutation for callers that cannot allocate device memory.
+//
+// The chunk-count matrix of the permutation lives in this fixed array instead of
+// a caller-supplied buffer.  Every GPU that loads the library holds these
+// kStaticPermInts * 4 bytes (1 MiB) until the process exits.  The name below is
+// only meaningful to device code; the host obtains the array's device address
+// once per device through cudaGetSymbolAddress and passes that to the kernels.
+constexpr int64_t kStaticPermInts = 262144;   // n_chunks * n_groups may not exceed this
+static __device__ __align__(256) int32_t g_static_perm_scratch[kStaticPermInts];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_perm_mutex;
+int32_t* g_static_perm_addr[kMaxDevices] = {};   // device address of the array, per device
+
+// Device address of g_static_perm_scratch on the current device (looked up once).
+int static_perm_scratch(int32_t** out) {
+  int dev = 0;
+  CU_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return arg_fail(CMOE_ERR_INVALID_ARG, "device ordinal too large");
+  std::lock_guard<std::mutex> lock(g_static_perm_mutex);
+  if (!g_static_perm_addr[dev]) {
+    void* p = nullptr;
+    CU_TRY(cudaGetSymbolAddress(&p, g_static_perm_scratch));
+    g_static_perm_addr[dev] = static_cast<int32_t*>(p);
+  }
+  *out = g_static_perm_addr[dev];
+  return CMOE_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int cmoe_token_permute_static(const int32_t* topk_idx, int32_t n_rows, int32_t n_k,
+                              int32_t n_groups, int32_t* counts, int32_t* offsets,
+                              int32_t* row_token, int32_t* row_of, void* stream) {
+  if (n_rows < 0 || n_k < 0 || n_k > kMaxTopK || n_groups <= 0 || n_groups > kPermMaxGroups)
+    return arg_fail(CMOE_ERR_INVALID_ARG, "permute: size out of range");
+  if (!counts || !offsets || ((int64_t)n_rows * n_k > 0 && (!topk_idx || !row_token || !row_of)))
+    return arg_fail(CMOE_ERR_INVALID_ARG, "permute: null pointer");
+  const int64_t n_chunks = ((int64_t)n_rows + kPermChunk - 1) / kPermChunk;
+  if (n_rows > kPermChunk && n_chunks * n_groups > kStaticPermInts)
+    return arg_fail(CMOE_ERR_CAPACITY,
+                    "permute (static scratch): ceil(n_rows/256) * n_groups exceeds 262144 cells");
+  int32_t* scratch = nullptr;
+  const int rc = static_perm_scratch(&scratch);
+  if (rc != CMOE_OK) return rc;
+  // Every cell the scan and scatter kernels read is first written by the count kernel of
+  // the same call, so nothing left over from an earlier call needs clearing.
+  launch_token_permute(topk_idx, n_rows, n_k, n_groups, counts, offsets, row_token, row_of, scratch,
+                       static_cast<cudaStream_t>(stream));
   CU_TRY(cudaGetLastError());
   return CMOE_OK;
 }
