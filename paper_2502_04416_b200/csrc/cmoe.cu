@@ -66,8 +66,9 @@ struct cmoe_layer {
   bool umma_ok = false;
 
   // packed weights
-  void* wg_p = nullptr;     // [n_outer*d_ff, d]   neurons in expert order
-  void* wu_p = nullptr;     // [n_outer*d_ff, d]
+  void* w_gu = nullptr;     // one allocation [2][n_outer*d_ff, d]: gate plane, then up plane
+  void* wg_p = nullptr;     // [n_outer*d_ff, d]   neurons in expert order (view into w_gu)
+  void* wu_p = nullptr;     // [n_outer*d_ff, d]   (view into w_gu)
   void* wd_p = nullptr;     // per outer expert: shared block [d, N_s*m], then N_r blocks [d, m]
   void* w_rep = nullptr;    // [n_outer][2*N_r][d] representatives' gate rows, then up rows
   void* w_router = nullptr; // [n_outer, d] (hierarchical)
@@ -111,7 +112,7 @@ void free_layer(cmoe_layer* L) {
   if (!L) return;
   for (cudaEvent_t e : L->ev) cudaEventDestroy(e);
   umma_plan_destroy(&L->umma);
-  cudaFree(L->wg_p); cudaFree(L->wu_p); cudaFree(L->wd_p); cudaFree(L->w_rep);
+  cudaFree(L->w_gu); cudaFree(L->wd_p); cudaFree(L->w_rep);
   cudaFree(L->w_router); cudaFree(L->u); cudaFree(L->b); cudaFree(L->gs); cudaFree(L->ws);
   delete L;
 }
@@ -238,8 +239,8 @@ int finish_layer(cmoe_layer* L, cudaStream_t st) {
     s.n_outer = L->n_outer; s.n_r = L->n_r;
     s.max_outer_rows = (size_t)L->cfg.max_tokens * (L->hier ? L->outer_k : 1);
     s.max_routed_rows = s.max_outer_rows * L->cfg.top_k;
-    rc = umma_plan_create(&L->umma, s, L->gs_host.data(), L->n_groups_total(), L->wg_p, L->wu_p,
-                          L->wd_p, L->x_perm, L->h_s, L->h_r, L->y_s, L->y_r);
+    rc = umma_plan_create(&L->umma, s, L->gs, L->n_groups_total(), L->w_gu, L->wd_p, L->x_perm,
+                          L->h_s, L->h_r, L->y_s, L->y_r, L->hier ? L->xo : nullptr);
     if (rc == CMOE_ERR_CUDA) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     L->umma_ok = (rc == CMOE_OK);
   }
@@ -405,8 +406,9 @@ int cmoe_layer_create(const cmoe_config* cfg, const void* w_gate, const void* w_
     if (e_ != cudaSuccess) return fail(cuda_fail(e_, #expr));             \
   } while (0)
   const size_t wbytes = (size_t)d_ff * d * L->esz;
-  TRY_OR_FAIL(cudaMalloc(&L->wg_p, wbytes));
-  TRY_OR_FAIL(cudaMalloc(&L->wu_p, wbytes));
+  TRY_OR_FAIL(cudaMalloc(&L->w_gu, 2 * wbytes));
+  L->wg_p = L->w_gu;
+  L->wu_p = (char*)L->w_gu + wbytes;
   TRY_OR_FAIL(cudaMalloc(&L->wd_p, wbytes));
   TRY_OR_FAIL(cudaMalloc(&L->w_rep, (size_t)(n_r ? 2 * n_r : 1) * d * L->esz));
   TRY_OR_FAIL(cudaMalloc(&L->u, (size_t)(n_r ? n_r : 1) * sizeof(float)));
@@ -466,8 +468,9 @@ int cmoe_hier_create(int32_t n_outer, int32_t outer_top_k, const void* w_router,
     cudaError_t e_ = (expr);                                              \
     if (e_ != cudaSuccess) return fail(cuda_fail(e_, #expr));             \
   } while (0)
-  TRY_OR_FAIL(cudaMalloc(&L->wg_p, wbytes * n_outer));
-  TRY_OR_FAIL(cudaMalloc(&L->wu_p, wbytes * n_outer));
+  TRY_OR_FAIL(cudaMalloc(&L->w_gu, 2 * wbytes * n_outer));
+  L->wg_p = L->w_gu;
+  L->wu_p = (char*)L->w_gu + wbytes * n_outer;
   TRY_OR_FAIL(cudaMalloc(&L->wd_p, wbytes * n_outer));
   TRY_OR_FAIL(cudaMalloc(&L->w_rep, (rep_bytes ? rep_bytes : 16) * n_outer));
   TRY_OR_FAIL(cudaMalloc(&L->w_router, (size_t)n_outer * d * esz));

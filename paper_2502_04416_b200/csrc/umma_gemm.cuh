@@ -1,28 +1,549 @@
-// Tensor-core (tcgen05 / TMEM / TMA) grouped expert GEMMs.  Placeholder: plan creation
-// reports "shape not taken", so every layer runs the SIMT kernels.
+// Tensor-core grouped expert GEMMs for sm_100a: tcgen05.mma with the accumulator in
+// tensor memory (TMEM), operands staged in shared memory by TMA, one persistent CTA per
+// SM, warp-specialised (TMA producer / MMA issuer / 4 epilogue warps), TMEM accumulator
+// double-buffered so the epilogue of one tile overlaps the MMAs of the next.
+//
+//   GEMM-1 (MODE 1): H[r, n] = Swish(x_r . Wg[n]) * (x_r . Wu[n])          (Eq. ori_ffn_method)
+//       A tile  : 128 rows of x (shared groups: outer-row order; routed: permuted rows) x 64 k
+//       B tile  : bn gate rows + bn up rows of the group's neurons x 64 k (one 3-D TMA box)
+//       D (TMEM): 128 lanes x 2*bn fp32 columns; epilogue fuses SiLU(gate)*up -> bf16 H
+//   GEMM-2 (MODE 2): Y[r, c] = sum_n H[r, n] Wd[c, n]
+//       A tile  : 128 rows of H x 64 k ;  B tile: 256 rows (output channels) of the group's
+//       W_down block x 64 k ;  D: 128 x 256 fp32 ; epilogue rounds to bf16 Y.
+// All operands are K-major with the 128-byte swizzle; rows or k beyond a tensor's extent
+// are zero-filled by TMA, rows beyond a group's count are computed but never stored.
+//
+// Every mbarrier wait is bounded (about a second of SM clock); a wait that runs out sets
+// the layer's device error word, raises a CTA-wide abort flag that the other waits poll,
+// and the CTA falls through to the common teardown, which frees its TMEM.
 #pragma once
+
+#include <cuda.h>
+
+#include <cstdio>
 
 #include "common.cuh"
 
 namespace cmoe {
 
+constexpr int kUmmaBM = 128;          // rows per tile (UMMA M)
+constexpr int kUmmaBK = 64;           // k per stage: 64 bf16 = one 128-byte swizzle row
+constexpr int kUmmaStages = 4;
+constexpr int kUmmaABytes = kUmmaBM * kUmmaBK * 2;       // 16 KB
+constexpr int kUmmaBBytes = 256 * kUmmaBK * 2;           // 32 KB (up to 256 B rows)
+constexpr int kUmmaStageBytes = kUmmaABytes + kUmmaBBytes;
+constexpr int kUmmaMaxGroups = 1088;
+constexpr int kUmmaThreads = 192;     // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr int kUmmaTmemCols = 512;    // two accumulator buffers of 256 columns
+constexpr int kUmmaSmemBytes = 1024 /*alignment slack*/ + kUmmaStages * kUmmaStageBytes +
+                               256 /*barriers*/ + (kUmmaMaxGroups + 1) * 4;
+constexpr long long kUmmaWaitCycles = 2000000000LL;   // ~1 s at SM clock
+
+enum { kErrWaitFull = 1, kErrWaitEmpty = 2, kErrWaitAccFull = 3, kErrWaitAccEmpty = 4 };
+
+// ----------------------------------------------------------------------------- PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the wait ran out (error word + abort flag set) or another wait
+// of this CTA already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* err_word, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kUmmaWaitCycles) {
+      *abort_flag = 1;
+      atomicCAS(err_word, 0, code);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1,
+                                            int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1,
+                                            int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(cols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// D[tmem] (+)= A[smem desc] * B[smem desc]^T, bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// mbarrier arrives once all tcgen05 operations issued so far by this thread have completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 16 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major tile, 128-byte rows, 128-byte swizzle, 8-row
+// groups 1024 bytes apart; `addr` is the 1024-byte-aligned tile base plus the k offset.
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFF);
+  d |= (uint64_t)1 << 16;                 // leading-dimension offset (unused with swizzle)
+  d |= (uint64_t)(1024 >> 4) << 32;       // stride between 8-row groups
+  d |= (uint64_t)1 << 46;                 // descriptor version of sm_100
+  d |= (uint64_t)2 << 61;                 // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kUmmaBM >> 4) << 24);
+}
+
+// ----------------------------------------------------------------------------- kernel
+struct UmmaArgs {
+  const GroupStatic* gs;
+  const GroupRows* gr;
+  int n_groups, n_outer, n_r;
+  int d;                 // model width: K of GEMM-1, N of GEMM-2
+  int bn_s, bn_r;        // GEMM-1 neurons per tile for shared / routed groups
+  int d_ff, shared_width;
+  bf16* out_s;           // GEMM-1: H_s ; GEMM-2: Y_s
+  bf16* out_r;           // GEMM-1: H_r ; GEMM-2: Y_r
+  int ld_out_s, ld_out_r;
+  int32_t* err;
+};
+
+struct TileCoord { int g, mt, nt; };
+
+template <int MODE>
+__device__ __forceinline__ int umma_n_tiles(const UmmaArgs& p, const GroupStatic& g) {
+  if (MODE == 1) {
+    const int bn = g.is_shared ? p.bn_s : p.bn_r;
+    return (g.width + bn - 1) / bn;
+  }
+  return g.width > 0 ? (p.d + 255) / 256 : 0;
+}
+
+__device__ __forceinline__ TileCoord umma_decode(const int32_t* tile_start, int n_groups, int t,
+                                                 const GroupRows* gr) {
+  int lo = 0, hi = n_groups;                 // last g with tile_start[g] <= t
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (tile_start[mid] <= t) lo = mid; else hi = mid;
+  }
+  const int local = t - tile_start[lo];
+  const int m_tiles = (gr[lo].count + kUmmaBM - 1) / kUmmaBM;
+  TileCoord c;
+  c.g = lo; c.mt = local % m_tiles; c.nt = local / m_tiles;
+  return c;
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_constant__ CUtensorMap tm_a_r,
+                    const __grid_constant__ CUtensorMap tm_b_s, const __grid_constant__ CUtensorMap tm_b_r,
+                    const UmmaArgs p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - raw);                       // generic pointer to the aligned base
+  const uint32_t bars = base + kUmmaStages * kUmmaStageBytes;   // barrier block
+  uint8_t* bars_gen = gen + kUmmaStages * kUmmaStageBytes;
+  // barrier block: full[4] empty[4] acc_full[2] acc_empty[2] (8 B each), tmem slot, abort flag
+  const uint32_t full0 = bars, empty0 = bars + 32, accf0 = bars + 64, acce0 = bars + 80;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_gen + 96);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 100);
+  int32_t* tile_start = reinterpret_cast<int32_t*>(bars_gen + 256);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kUmmaStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), kUmmaTmemCols);
+    tmem_relinquish();
+  }
+  // tiles of every group, then their exclusive prefix
+  for (int g = threadIdx.x; g < p.n_groups; g += blockDim.x) {
+    const int m_tiles = (p.gr[g].count + kUmmaBM - 1) / kUmmaBM;
+    tile_start[g + 1] = m_tiles * umma_n_tiles<MODE>(p, p.gs[g]);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int run = 0;
+    tile_start[0] = 0;
+    for (int g = 0; g < p.n_groups; ++g) { run += tile_start[g + 1]; tile_start[g + 1] = run; }
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int total_tiles = tile_start[p.n_groups];
+  const int k_blocks_fixed = (p.d + kUmmaBK - 1) / kUmmaBK;      // GEMM-1: K = d
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        const TileCoord c = umma_decode(tile_start, p.n_groups, t, p.gr);
+        const GroupStatic g = p.gs[c.g];
+        const int row = p.gr[c.g].row0 + c.mt * kUmmaBM;
+        const CUtensorMap* ta = g.is_shared ? &tm_a_s : &tm_a_r;
+        const CUtensorMap* tb = g.is_shared ? &tm_b_s : &tm_b_r;
+        int k_blocks, b_bytes, b_row = 0, j = 0;
+        if (MODE == 1) {
+          const int bn = g.is_shared ? p.bn_s : p.bn_r;
+          k_blocks = k_blocks_fixed;
+          b_bytes = 2 * bn * kUmmaBK * 2;
+          b_row = g.w_row0 + c.nt * bn;
+        } else {
+          k_blocks = (g.width + kUmmaBK - 1) / kUmmaBK;
+          b_bytes = kUmmaBBytes;
+          b_row = c.nt * 256;
+          j = g.is_shared ? 0 : (c.g - p.n_outer) - g.outer * p.n_r;
+        }
+        for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+          const uint32_t s = it % kUmmaStages, n = it / kUmmaStages;
+          if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
+          const uint32_t fb = full0 + 8 * s;
+          const uint32_t sa = base + s * kUmmaStageBytes, sb = sa + kUmmaABytes;
+          mbar_expect_tx(fb, kUmmaABytes + b_bytes);
+          tma_load_2d(sa, ta, fb, kb * kUmmaBK, row);
+          if (MODE == 1) tma_load_3d(sb, tb, fb, kb * kUmmaBK, b_row, 0);
+          else if (g.is_shared) tma_load_3d(sb, tb, fb, kb * kUmmaBK, b_row, g.outer);
+          else tma_load_4d(sb, tb, fb, kb * kUmmaBK, b_row, j, g.outer);
+        }
+      }
+      if (!ok) for (int i = 0; i < 200; ++i) __nanosleep(1000);   // let copies in flight land
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t it = 0, tile_n = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_n) {
+        const TileCoord c = umma_decode(tile_start, p.n_groups, t, p.gr);
+        const GroupStatic g = p.gs[c.g];
+        int k_blocks, n_mma;
+        if (MODE == 1) { k_blocks = k_blocks_fixed; n_mma = 2 * (g.is_shared ? p.bn_s : p.bn_r); }
+        else { k_blocks = (g.width + kUmmaBK - 1) / kUmmaBK; n_mma = 256; }
+        const uint32_t idesc = umma_idesc(n_mma);
+        const uint32_t buf = tile_n & 1, use = tile_n >> 1;
+        if (!mbar_wait(acce0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.err, kErrWaitAccEmpty)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * 256;
+        for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+          const uint32_t s = it % kUmmaStages, n = it / kUmmaStages;
+          if (!mbar_wait(full0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = base + s * kUmmaStageBytes, sb = sa + kUmmaABytes;
+#pragma unroll
+          for (int k = 0; k < kUmmaBK / 16; ++k)
+            umma_bf16(d_tmem, umma_smem_desc(sa + k * 32), umma_smem_desc(sb + k * 32), idesc,
+                      (kb | k) != 0 ? 1u : 0u);
+          umma_commit(empty0 + 8 * s);         // stage reusable once these MMAs have read it
+        }
+        if (ok) umma_commit(accf0 + 8 * buf);  // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
+    uint32_t tile_n = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_n) {
+      const TileCoord c = umma_decode(tile_start, p.n_groups, t, p.gr);
+      const GroupStatic g = p.gs[c.g];
+      const GroupRows r = p.gr[c.g];
+      const uint32_t buf = tile_n & 1, use = tile_n >> 1;
+      if (!mbar_wait(accf0 + 8 * buf, use & 1, abort_flag, p.err, kErrWaitAccFull)) { ok = false; break; }
+      tc_fence_after();
+      const int row_in_group = c.mt * kUmmaBM + quad * 32 + lane;
+      const bool row_ok = row_in_group < r.count;
+      const uint32_t taddr = tmem_base + buf * 256 + ((uint32_t)(quad * 32) << 16);
+      if (MODE == 1) {
+        const int bn = g.is_shared ? p.bn_s : p.bn_r;
+        const int ld = g.is_shared ? p.ld_out_s : p.ld_out_r;
+        const int n0 = c.nt * bn;
+        const int n_valid = min(bn, g.width - n0);
+        bf16* dst = (g.is_shared ? p.out_s : p.out_r) + (size_t)(r.row0 + row_in_group) * ld + n0;
+        for (int c0 = 0; c0 < n_valid; c0 += 16) {
+          float gt[16], up[16];
+          tmem_ld16(taddr + c0, gt);
+          tmem_ld16(taddr + bn + c0, up);
+          tmem_ld_wait();
+          if (row_ok) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              if (c0 + h * 8 < n_valid) {
+                float v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                  const float a = gt[h * 8 + q];
+                  v[q] = a / (1.0f + __expf(-a)) * up[h * 8 + q];
+                }
+                store8(dst + c0 + h * 8, v);
+              }
+            }
+          }
+        }
+      } else {
+        const int n0 = c.nt * 256;
+        const int n_valid = min(256, p.d - n0);
+        bf16* dst = (g.is_shared ? p.out_s : p.out_r) + (size_t)(r.row0 + row_in_group) * p.d + n0;
+        for (int c0 = 0; c0 < n_valid; c0 += 16) {
+          float acc[16];
+          tmem_ld16(taddr + c0, acc);
+          tmem_ld_wait();
+          if (row_ok) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              if (c0 + h * 8 < n_valid) {
+                float v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) v[q] = acc[h * 8 + q];
+                store8(dst + c0 + h * 8, v);
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acce0 + 8 * buf);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kUmmaTmemCols);
+  }
+}
+
+// ----------------------------------------------------------------------------- host
 struct UmmaShape {
   int d = 0, m = 0, shared_width = 0, d_ff = 0, n_outer = 1, n_r = 0;
   size_t max_outer_rows = 0, max_routed_rows = 0;
 };
 
+typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                    CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                    CUtensorMapFloatOOBfill);
+
 struct UmmaPlan {
+  bool built = false;
   char error[256] = "";
+  UmmaShape shape;
+  int bn_s = 128, bn_r = 128, n_sms = 0, n_groups = 0;
+  const GroupStatic* gs_dev = nullptr;
+  PFN_encodeTiled encode = nullptr;
+  bool x_is_fixed = false;                 // hierarchical layers read x from their own buffer
+  CUtensorMap a1_s, a1_r, b1_s, b1_r;      // GEMM-1: x rows / permuted x rows / stacked gate+up rows
+  CUtensorMap a2_s, a2_r, b2_s, b2_r;      // GEMM-2: H_s / H_r / shared W_down / routed W_down blocks
+  bf16 *h_s = nullptr, *h_r = nullptr, *y_s = nullptr, *y_r = nullptr;
 };
 
-// 0: plan built; 1: shape not taken by this path; CMOE_ERR_CUDA (-5): a driver call failed.
-inline int umma_plan_create(UmmaPlan*, const UmmaShape&, const GroupStatic*, int, const void*,
-                            const void*, const void*, void*, void*, void*, void*, void*) { return 1; }
-inline void umma_plan_destroy(UmmaPlan*) {}
-// Enqueues both expert GEMMs; returns the number of kernels launched or -1.
-inline int umma_forward(UmmaPlan*, const void*, int, int, const GroupRows*, int32_t*, cudaStream_t,
-                        cudaEvent_t /*recorded between GEMM-1 and GEMM-2, may be null*/) {
-  return -1;
+// Neurons per GEMM-1 tile: the multiple of 8 in [96, 128] that wastes the least of the last tile.
+inline int umma_pick_bn(int width) {
+  if (width <= 0) return 128;
+  int best = 128, best_pad = (width + 127) / 128 * 128;
+  for (int bn = 120; bn >= 96; bn -= 8) {
+    const int pad = (width + bn - 1) / bn * bn;
+    if (pad < best_pad) { best = bn; best_pad = pad; }
+  }
+  return best;
+}
+
+inline bool umma_encode(UmmaPlan* P, CUtensorMap* tm, const void* base, int rank, const cuuint64_t* dims,
+                        const cuuint64_t* strides_bytes, const cuuint32_t* box, const char* what) {
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  for (int i = 0; i < rank; ++i)
+    if (dims[i] == 0) { snprintf(P->error, sizeof(P->error), "tensor map %s: zero extent", what); return false; }
+  const CUresult r = P->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base),
+                               dims, strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(P->error, sizeof(P->error), "cuTensorMapEncodeTiled(%s) failed with CUresult %d", what, (int)r);
+    return false;
+  }
+  return true;
+}
+
+// [rows, cols] row-major bf16 matrix, box 64 x 128.
+inline bool umma_encode_rows(UmmaPlan* P, CUtensorMap* tm, const void* base, size_t rows, size_t cols,
+                             const char* what) {
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t str[1] = {cols * 2};
+  const cuuint32_t box[2] = {kUmmaBK, kUmmaBM};
+  return umma_encode(P, tm, base, 2, dims, str, box, what);
+}
+
+// 0: plan built; 1: shape not taken by this path; -5: a driver call failed (P->error).
+inline int umma_plan_create(UmmaPlan* P, const UmmaShape& s, const GroupStatic* gs_dev, int n_groups,
+                            const void* w_gate_up /* [2][n_outer*d_ff][d] */, const void* w_down,
+                            const void* x_perm, void* h_s, void* h_r, void* y_s, void* y_r,
+                            const void* x_fixed /* hierarchical: the layer's own outer-row copy of x */) {
+  P->built = false;
+  const bool has_s = s.shared_width > 0 && s.max_outer_rows > 0;
+  const bool has_r = s.n_r > 0 && s.max_routed_rows > 0;
+  if (!has_s && !has_r) return 1;
+  if (s.d % 8 || s.m % 8 || s.shared_width % 8 || n_groups > kUmmaMaxGroups) return 1;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
+      q != cudaDriverEntryPointSuccess) {
+    snprintf(P->error, sizeof(P->error), "cuTensorMapEncodeTiled entry point not found");
+    return -5;
+  }
+  P->encode = reinterpret_cast<PFN_encodeTiled>(fn);
+  P->shape = s;
+  P->gs_dev = gs_dev;
+  P->n_groups = n_groups;
+  P->bn_s = umma_pick_bn(s.shared_width);
+  P->bn_r = umma_pick_bn(s.m);
+  P->h_s = (bf16*)h_s; P->h_r = (bf16*)h_r; P->y_s = (bf16*)y_s; P->y_r = (bf16*)y_r;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&P->n_sms, cudaDevAttrMultiProcessorCount, dev);
+
+  const size_t d = s.d, rows_w = (size_t)s.n_outer * s.d_ff;
+  bool ok = true;
+  // GEMM-1 B: gate and up stacked, [2][rows_w][d]; box = 64 k x bn rows x 2 planes
+  for (int shared = 0; shared < 2 && ok; ++shared) {
+    const int bn = shared ? P->bn_s : P->bn_r;
+    const cuuint64_t dims[3] = {d, rows_w, 2};
+    const cuuint64_t str[2] = {d * 2, rows_w * d * 2};
+    const cuuint32_t box[3] = {kUmmaBK, (cuuint32_t)bn, 2};
+    ok = umma_encode(P, shared ? &P->b1_s : &P->b1_r, w_gate_up, 3, dims, str, box, "gate/up weights");
+  }
+  // GEMM-1 A (routed): permuted rows of x; GEMM-2 A: H_s, H_r
+  if (ok && has_r) ok = umma_encode_rows(P, &P->a1_r, x_perm, s.max_routed_rows, d, "permuted x");
+  if (ok && has_r) ok = umma_encode_rows(P, &P->a2_r, h_r, s.max_routed_rows, s.m, "H routed");
+  if (ok && has_s) ok = umma_encode_rows(P, &P->a2_s, h_s, s.max_outer_rows, s.shared_width, "H shared");
+  // GEMM-2 B: shared block [d, W_s] of every outer expert; routed blocks [d, m] x N_r of every outer expert
+  if (ok && has_s) {
+    const cuuint64_t dims[3] = {(cuuint64_t)s.shared_width, d, (cuuint64_t)s.n_outer};
+    const cuuint64_t str[2] = {(cuuint64_t)s.shared_width * 2, d * s.d_ff * 2};
+    const cuuint32_t box[3] = {kUmmaBK, 256, 1};
+    ok = umma_encode(P, &P->b2_s, w_down, 3, dims, str, box, "shared W_down");
+  }
+  if (ok && has_r) {
+    const cuuint64_t dims[4] = {(cuuint64_t)s.m, d, (cuuint64_t)s.n_r, (cuuint64_t)s.n_outer};
+    const cuuint64_t str[3] = {(cuuint64_t)s.m * 2, d * s.m * 2, d * s.d_ff * 2};
+    const cuuint32_t box[4] = {kUmmaBK, 256, 1, 1};
+    ok = umma_encode(P, &P->b2_r, (const bf16*)w_down + (size_t)s.shared_width * d, 4, dims, str, box,
+                     "routed W_down");
+  }
+  P->x_is_fixed = x_fixed != nullptr;
+  if (ok && x_fixed && has_s) ok = umma_encode_rows(P, &P->a1_s, x_fixed, s.max_outer_rows, d, "outer rows of x");
+  if (!ok) return -5;
+  // placeholders for absent operand classes (never dereferenced: such groups have no tiles)
+  if (!has_r) { P->a1_r = P->a2_s; P->a2_r = P->a2_s; P->b2_r = P->b2_s; }
+  if (!has_s) { P->a2_s = P->a2_r; P->b2_s = P->b2_r; P->a1_s = P->a1_r; }
+  cudaError_t e = cudaFuncSetAttribute(umma_grouped_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kUmmaSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(umma_grouped_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kUmmaSmemBytes);
+  if (e != cudaSuccess) {
+    snprintf(P->error, sizeof(P->error), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+    return -5;
+  }
+  P->built = true;
+  return 0;
+}
+
+inline void umma_plan_destroy(UmmaPlan* P) { P->built = false; }
+
+// Enqueues GEMM-1 and GEMM-2 over all groups; returns the number of kernels launched, or -1
+// (P->error).  `x_rows` are the outer rows of x ([n_outer_rows, d]); for a plain layer this is
+// the caller's x, whose tensor map is encoded here (a host-side struct fill, no allocation).
+inline int umma_forward(UmmaPlan* P, const void* x_rows, int n_outer_rows, int n_routed_rows,
+                        const GroupRows* gr, int32_t* err_word, cudaStream_t st, cudaEvent_t mid) {
+  (void)n_routed_rows;
+  const UmmaShape& s = P->shape;
+  CUtensorMap a1_s = P->a1_s;
+  if (!P->x_is_fixed && s.shared_width > 0) {
+    if (!umma_encode_rows(P, &a1_s, x_rows, (size_t)n_outer_rows, (size_t)s.d, "x")) return -1;
+  }
+  UmmaArgs a;
+  a.gs = P->gs_dev; a.gr = gr; a.n_groups = P->n_groups; a.n_outer = s.n_outer; a.n_r = s.n_r;
+  a.d = s.d; a.bn_s = P->bn_s; a.bn_r = P->bn_r; a.d_ff = s.d_ff; a.shared_width = s.shared_width;
+  a.err = err_word;
+  a.out_s = P->h_s; a.out_r = P->h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
+  umma_grouped_kernel<1><<<P->n_sms, kUmmaThreads, kUmmaSmemBytes, st>>>(a1_s, P->a1_r, P->b1_s, P->b1_r, a);
+  if (mid) cudaEventRecord(mid, st);
+  a.out_s = P->y_s; a.out_r = P->y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
+  umma_grouped_kernel<2><<<P->n_sms, kUmmaThreads, kUmmaSmemBytes, st>>>(P->a2_s, P->a2_r, P->b2_s, P->b2_r, a);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    snprintf(P->error, sizeof(P->error), "tensor-core GEMM launch: %s", cudaGetErrorString(e));
+    return -1;
+  }
+  return 2;
 }
 
 }  // namespace cmoe
