@@ -52,6 +52,18 @@ class ClockSampler:
 
     def __init__(self, gpu_index: int):
         self.rows, self.proc, self.gpu = [], None, gpu_index
+        self.begin = self.end = None
+
+    def wait_first(self, timeout: float = 5.0):
+        t0 = time.time()
+        while not self.rows and time.time() - t0 < timeout and self.proc is not None:
+            time.sleep(0.02)
+
+    def mark_begin(self):
+        self.begin = len(self.rows)
+
+    def mark_end(self):
+        self.end = len(self.rows)
 
     def start(self):
         try:
@@ -76,7 +88,12 @@ class ClockSampler:
                 self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        rows, window = self.rows, "all samples while the process ran"
+        if self.begin is not None and self.end is not None and self.end > self.begin:
+            rows, window = self.rows[self.begin:self.end + 1], "timed region"
+        elif self.begin is not None:
+            rows, window = self.rows[max(self.begin - 1, 0):], "timed region shorter than one sample: nearest samples"
+        for r in rows:
             if len(r) < 7:
                 continue
             try:
@@ -88,7 +105,7 @@ class ClockSampler:
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None,
                 "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
-                "samples": len(sm)}
+                "samples": len(sm), "window": window}
 
 
 # ------------------------------------------------------------- CPU oracle arm
@@ -194,13 +211,17 @@ def run_gpu(args):
         return float(ms.item())
 
     # ---- device-resident throughput, with per-stage events for the roofline
+    sampler = ClockSampler(local)
+    sampler.start()
     layer.enable_stage_timing(min(args.steps, 4096))
     for _ in range(args.warmup):
         layer.forward(x, out)
     layer.enable_stage_timing(min(args.steps, 4096))          # reset the ring after warm-up
-    sampler = ClockSampler(local)
-    sampler.start()
+    sampler.wait_first()
+    sampler.mark_begin()
     ms_total = timed(lambda: layer.forward(x, out), args.steps)
+    sampler.mark_end()
+    time.sleep(0.12)                                          # let the sample that covers the end arrive
     clocks = sampler.stop()
     stage_ms, n_cov = layer.stage_times()
     launches = layer.launch_count() * args.steps
@@ -338,8 +359,8 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="c2_llama2_7b", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--tokens", type=int, default=0, help="tokens per step (default: the workload's largest T)")
