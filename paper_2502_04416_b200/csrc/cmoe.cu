@@ -10,12 +10,14 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <type_traits>
 #include <vector>
 
 #include "combine.cuh"
 #include "common.cuh"
 #include "permute.cuh"
 #include "router.cuh"
+#include "router_mma.cuh"
 #include "simt_gemm.cuh"
 #include "umma_gemm.cuh"
 
@@ -282,9 +284,20 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   mark(0);
 
   if (L->hier) {
-    outer_router_kernel<T><<<(n_tok + 7) / 8, 256, 0, st>>>(x, n_tok, d, L->n_outer, L->outer_k,
-                                                            (const T*)L->w_router, L->outer_logits,
-                                                            L->outer_idx, L->outer_w);
+    if constexpr (std::is_same<T, bf16>::value) {
+      if (n_tok >= 2048)
+        outer_router_mma_kernel<4, 2><<<(n_tok + 31) / 32, 128, 0, st>>>(
+            x, n_tok, d, L->n_outer, L->outer_k, (const bf16*)L->w_router, L->outer_logits, L->outer_idx,
+            L->outer_w);
+      else
+        outer_router_mma_kernel<8, 1><<<(n_tok + 15) / 16, 256, 0, st>>>(
+            x, n_tok, d, L->n_outer, L->outer_k, (const bf16*)L->w_router, L->outer_logits, L->outer_idx,
+            L->outer_w);
+    } else {
+      outer_router_kernel<T><<<(n_tok + 7) / 8, 256, 0, st>>>(x, n_tok, d, L->n_outer, L->outer_k,
+                                                              (const T*)L->w_router, L->outer_logits,
+                                                              L->outer_idx, L->outer_w);
+    }
     ++launches;
     launches += launch_token_permute(L->outer_idx, n_tok, L->outer_k, L->n_outer, L->outer_counts,
                                      L->outer_off, L->outer_row_token, L->outer_row_of,
@@ -301,9 +314,20 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   router_kernel<T, NACC><<<blocks, 256, 0, st>>>(xo, R, d, n_r, n_k, (const T*)L->w_rep, L->u,   \
                                                  L->b, ooff, L->n_outer, L->scores, L->keys,      \
                                                  L->topk_idx, L->topk_gate)
-    if (2 * n_r <= 16) CMOE_ROUTER(16);
-    else if (2 * n_r <= 32) CMOE_ROUTER(32);
-    else CMOE_ROUTER(64);
+    if constexpr (std::is_same<T, bf16>::value) {
+      if (R >= 2048)
+        router_mma_kernel<4, 2><<<(R + 31) / 32, 128, 0, st>>>(
+            xo, R, d, n_r, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->scores, L->keys,
+            L->topk_idx, L->topk_gate);
+      else
+        router_mma_kernel<8, 1><<<(R + 15) / 16, 256, 0, st>>>(
+            xo, R, d, n_r, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->scores, L->keys,
+            L->topk_idx, L->topk_gate);
+    } else {
+      if (2 * n_r <= 16) CMOE_ROUTER(16);
+      else if (2 * n_r <= 32) CMOE_ROUTER(32);
+      else CMOE_ROUTER(64);
+    }
 #undef CMOE_ROUTER
     ++launches;
     mark(1);
