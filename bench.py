@@ -229,6 +229,14 @@ def run_gpu(args):
     layer.enable_stage_timing(0)
     value = world * T * args.steps / (ms_total * 1e-3)
 
+    if args.forward_only:                     # profiling runs: nothing but the forward passes
+        if rank == 0:
+            print(json.dumps({"forward_only": True, "workload": f"{w.name} T={T}", "ms_per_step": ms_total / args.steps,
+                              "stage_ms": {n: v / max(n_cov, 1) for n, v in zip(binding.STAGE_NAMES, stage_ms)}}))
+        if world > 1:
+            dist.destroy_process_group()
+        return None
+
     # ---- end to end through the public call with host buffers
     x_pin = torch.empty(x.shape, dtype=x.dtype).pin_memory()
     x_pin.copy_(x.cpu())
@@ -365,6 +373,8 @@ def main():
     ap.add_argument("--workload", default="c2_llama2_7b", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--tokens", type=int, default=0, help="tokens per step (default: the workload's largest T)")
     ap.add_argument("--cpu-sample-tokens", type=int, default=256)
+    ap.add_argument("--forward-only", action="store_true",
+                    help="run only the timed forward passes (for profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         line = run_reference(args)

@@ -44,6 +44,8 @@ int arg_fail(int code, const char* what) {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+constexpr int kTmaGatherMaxRows = 512;   // routed rows up to which gather4 replaces the permuted copy of x
+
 // Bump allocator over one device allocation (base == nullptr: measure only).
 struct Arena {
   char* base = nullptr;
@@ -60,7 +62,7 @@ struct Arena {
 
 struct cmoe_layer {
   cmoe_config cfg{};
-  int m = 0, n_r = 0, n_outer = 1, outer_k = 1;
+  int m = 0, n_r = 0, n_rp = 0, n_outer = 1, outer_k = 1;   // n_rp: N_r rounded up to 8
   bool hier = false;
   int device = 0;
   size_t esz = 2;
@@ -72,7 +74,7 @@ struct cmoe_layer {
   void* wg_p = nullptr;     // [n_outer*d_ff, d]   neurons in expert order (view into w_gu)
   void* wu_p = nullptr;     // [n_outer*d_ff, d]   (view into w_gu)
   void* wd_p = nullptr;     // per outer expert: shared block [d, N_s*m], then N_r blocks [d, m]
-  void* w_rep = nullptr;    // [n_outer][2*N_r][d] representatives' gate rows, then up rows
+  void* w_rep = nullptr;    // [n_outer][2*n_rp][d]: gate rows of the representatives (zero-padded to n_rp), then up rows
   void* w_router = nullptr; // [n_outer, d] (hierarchical)
   float* u = nullptr;       // [n_outer*N_r]
   float* b = nullptr;
@@ -238,11 +240,18 @@ int finish_layer(cmoe_layer* L, cudaStream_t st) {
   if (L->cfg.dtype == CMOE_BF16) {
     UmmaShape s;
     s.d = L->cfg.d_model; s.m = L->m; s.shared_width = L->shared_width(); s.d_ff = L->cfg.d_ff;
-    s.n_outer = L->n_outer; s.n_r = L->n_r;
+    s.n_outer = L->n_outer; s.n_r = L->n_r; s.n_rp = L->n_rp; s.n_k = L->cfg.top_k;
     s.max_outer_rows = (size_t)L->cfg.max_tokens * (L->hier ? L->outer_k : 1);
     s.max_routed_rows = s.max_outer_rows * L->cfg.top_k;
-    rc = umma_plan_create(&L->umma, s, L->gs, L->n_groups_total(), L->w_gu, L->wd_p, L->x_perm,
-                          L->h_s, L->h_r, L->y_s, L->y_r, L->hier ? L->xo : nullptr);
+    UmmaBuffers ub;
+    ub.w_gate_up = L->w_gu; ub.w_down = L->wd_p; ub.w_rep = L->w_rep;
+    ub.x_fixed = L->hier ? L->xo : nullptr;
+    ub.x_perm = L->x_perm;
+    ub.h_s = L->h_s; ub.h_r = L->h_r; ub.y_s = L->y_s; ub.y_r = L->y_r;
+    ub.gs_dev = L->gs; ub.u = L->u; ub.b = L->b;
+    ub.scores = L->scores; ub.keys = L->keys; ub.topk_idx = L->topk_idx; ub.topk_gate = L->topk_gate;
+    ub.row_token = L->row_token;
+    rc = umma_plan_create(&L->umma, s, ub, L->n_groups_total());
     if (rc == CMOE_ERR_CUDA) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     L->umma_ok = (rc == CMOE_OK);
   }
@@ -261,7 +270,7 @@ int pack_weights(cmoe_layer* L, const void* w_gate, const void* w_up, const void
     gather_rows_kernel<<<L->n_r, 256, 0, st>>>((const uint4*)w_gate, rep_dev, L->n_r, row_vec,
                                                (uint4*)L->w_rep);
     gather_rows_kernel<<<L->n_r, 256, 0, st>>>((const uint4*)w_up, rep_dev, L->n_r, row_vec,
-                                               (uint4*)((char*)L->w_rep + (size_t)L->n_r * d * sizeof(T)));
+                                               (uint4*)((char*)L->w_rep + (size_t)L->n_rp * d * sizeof(T)));
   }
   dim3 grid((d_ff + 255) / 256, d);
   pack_down_kernel<T><<<grid, 256, 0, st>>>((const T*)w_down, perm_dev, d, d_ff, L->m, L->shared_width(),
@@ -279,6 +288,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   const int row_vec = d * (int)sizeof(T) / 16;
   int launches = 0;
   const T* xo = x;
+  const bool use_umma = L->umma_ok && L->gemm_path != 1;
   cudaEvent_t* ev = L->ev_ring ? &L->ev[(size_t)(L->ev_count % L->ev_ring) * (CMOE_N_STAGES + 1)] : nullptr;
   auto mark = [&](int i) { if (ev) cudaEventRecord(ev[i], st); };
   mark(0);
@@ -307,25 +317,26 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
     xo = (const T*)L->xo;
   }
 
+  if (use_umma && !umma_bind_x(&L->umma, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   if (n_r > 0) {
     const int warps = (R + 1) / 2, blocks = (warps + 7) / 8;
     const int32_t* ooff = L->hier ? L->outer_off : nullptr;
 #define CMOE_ROUTER(NACC)                                                                         \
-  router_kernel<T, NACC><<<blocks, 256, 0, st>>>(xo, R, d, n_r, n_k, (const T*)L->w_rep, L->u,   \
+  router_kernel<T, NACC><<<blocks, 256, 0, st>>>(xo, R, d, n_r, L->n_rp, n_k, (const T*)L->w_rep, L->u,   \
                                                  L->b, ooff, L->n_outer, L->scores, L->keys,      \
                                                  L->topk_idx, L->topk_gate)
     if constexpr (std::is_same<T, bf16>::value) {
-      if (R >= 2048)
-        router_mma_kernel<4, 2><<<(R + 31) / 32, 128, 0, st>>>(
-            xo, R, d, n_r, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->scores, L->keys,
-            L->topk_idx, L->topk_gate);
-      else
+      if (use_umma && R >= 512) {
+        if (umma_router_forward(&L->umma, R, ooff, L->err_word, st) < 0)
+          return arg_fail(CMOE_ERR_CUDA, L->umma.error);
+      } else {
         router_mma_kernel<8, 1><<<(R + 15) / 16, 256, 0, st>>>(
-            xo, R, d, n_r, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->scores, L->keys,
-            L->topk_idx, L->topk_gate);
+            xo, R, d, n_r, L->n_rp, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->scores,
+            L->keys, L->topk_idx, L->topk_gate);
+      }
     } else {
-      if (2 * n_r <= 16) CMOE_ROUTER(16);
-      else if (2 * n_r <= 32) CMOE_ROUTER(32);
+      if (2 * L->n_rp <= 16) CMOE_ROUTER(16);
+      else if (2 * L->n_rp <= 32) CMOE_ROUTER(32);
       else CMOE_ROUTER(64);
     }
 #undef CMOE_ROUTER
@@ -339,15 +350,16 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   plan_groups_kernel<<<1, 256, 0, st>>>(L->n_outer, n_r, n_tok, L->hier ? L->outer_off : nullptr,
                                         L->counts, L->offsets, L->gr);
   ++launches;
-  if (P > 0) {
+  // Small batches: the tensor path gathers routed rows inside its TMA producer instead.
+  const bool tma_gather = use_umma && P <= kTmaGatherMaxRows;
+  if (P > 0 && !tma_gather) {
     gather_rows_kernel<<<P, 256, 0, st>>>((const uint4*)xo, L->row_token, P, row_vec, (uint4*)L->x_perm);
     ++launches;
   }
 
   mark(2);
-  const bool use_umma = L->umma_ok && L->gemm_path != 1;
   if (use_umma) {
-    const int n = umma_forward(&L->umma, xo, R, P, L->gr, L->err_word, st, ev ? ev[3] : nullptr);
+    const int n = umma_forward(&L->umma, L->gr, tma_gather, L->err_word, st, ev ? ev[3] : nullptr);
     if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     launches += n;
   } else {
@@ -418,7 +430,7 @@ int cmoe_layer_create(const cmoe_config* cfg, const void* w_gate, const void* w_
 
   cmoe_layer* L = new (std::nothrow) cmoe_layer();
   if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "out of host memory");
-  L->cfg = *cfg; L->m = m; L->n_r = n_r; L->n_outer = 1; L->outer_k = 1; L->hier = false;
+  L->cfg = *cfg; L->m = m; L->n_r = n_r; L->n_rp = (n_r + 7) / 8 * 8; L->n_outer = 1; L->outer_k = 1; L->hier = false;
   L->esz = cfg->dtype == CMOE_BF16 ? 2 : 4;
   cudaGetDevice(&L->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -434,7 +446,8 @@ int cmoe_layer_create(const cmoe_config* cfg, const void* w_gate, const void* w_
   L->wg_p = L->w_gu;
   L->wu_p = (char*)L->w_gu + wbytes;
   TRY_OR_FAIL(cudaMalloc(&L->wd_p, wbytes));
-  TRY_OR_FAIL(cudaMalloc(&L->w_rep, (size_t)(n_r ? 2 * n_r : 1) * d * L->esz));
+  TRY_OR_FAIL(cudaMalloc(&L->w_rep, (size_t)(n_r ? 2 * L->n_rp : 1) * d * L->esz));
+  TRY_OR_FAIL(cudaMemsetAsync(L->w_rep, 0, (size_t)(n_r ? 2 * L->n_rp : 1) * d * L->esz, st));
   TRY_OR_FAIL(cudaMalloc(&L->u, (size_t)(n_r ? n_r : 1) * sizeof(float)));
   TRY_OR_FAIL(cudaMalloc(&L->b, (size_t)(n_r ? n_r : 1) * sizeof(float)));
   TRY_OR_FAIL(cudaMalloc(&perm_dev, (size_t)d_ff * sizeof(int32_t)));
@@ -480,12 +493,12 @@ int cmoe_hier_create(int32_t n_outer, int32_t outer_top_k, const void* w_router,
   cmoe_layer* L = new (std::nothrow) cmoe_layer();
   if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "out of host memory");
   L->cfg = inner[0]->cfg; L->cfg.max_tokens = max_tokens;
-  L->m = inner[0]->m; L->n_r = inner[0]->n_r; L->esz = inner[0]->esz;
+  L->m = inner[0]->m; L->n_r = inner[0]->n_r; L->n_rp = inner[0]->n_rp; L->esz = inner[0]->esz;
   L->n_outer = n_outer; L->outer_k = outer_top_k; L->hier = true;
   cudaGetDevice(&L->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t d = L->cfg.d_model, d_ff = L->cfg.d_ff, nr = L->n_r, esz = L->esz;
-  const size_t wbytes = d_ff * d * esz, rep_bytes = 2 * nr * d * esz;
+  const size_t wbytes = d_ff * d * esz, rep_bytes = 2 * (size_t)L->n_rp * d * esz;
   auto fail = [&](int code) { free_layer(L); return code; };
 #define TRY_OR_FAIL(expr)                                                 \
   do {                                                                    \

@@ -55,7 +55,7 @@ __device__ __forceinline__ void gate_row(int lane, int n_r, int n_k, float a, fl
 
 template <typename T, int NACC>
 __global__ void __launch_bounds__(256)
-router_kernel(const T* __restrict__ xo, int n_rows, int d, int n_r, int n_k,
+router_kernel(const T* __restrict__ xo, int n_rows, int d, int n_r, int n_rp, int n_k,
               const T* __restrict__ w_rep, const float* __restrict__ u, const float* __restrict__ b,
               const int32_t* __restrict__ outer_off, int n_outer,
               float* __restrict__ scores, float* __restrict__ keys,
@@ -68,7 +68,7 @@ router_kernel(const T* __restrict__ xo, int n_rows, int d, int n_r, int n_k,
   const int r1 = has1 ? r0 + 1 : r0;
   const int g0 = outer_off ? find_outer(outer_off, n_outer, r0) : 0;
   const int g1 = outer_off ? find_outer(outer_off, n_outer, r1) : 0;
-  const int n2 = 2 * n_r;
+  const int n2 = 2 * n_rp;      // W^R block: n_rp gate rows (zero-padded), then n_rp up rows
   const T* x0 = xo + (size_t)r0 * d;
   const T* x1 = xo + (size_t)r1 * d;
   const T* w0 = w_rep + (size_t)g0 * n2 * d;
@@ -108,7 +108,7 @@ router_kernel(const T* __restrict__ xo, int n_rows, int d, int n_r, int n_k,
       const float t0 = warp_sum(acc0[j]);
       const float t1 = warp_sum(acc1[j]);
       if (lane == j) { a0 = t0; a1 = t1; }
-      if (lane == j - n_r) { v0 = t0; v1 = t1; }
+      if (lane == j - n_rp) { v0 = t0; v1 = t1; }
     }
   }
   gate_row(lane, n_r, n_k, a0, v0, u + g0 * n_r, b + g0 * n_r, g0 * n_r,

@@ -101,7 +101,7 @@ __device__ __forceinline__ void block_dot_tile(const bf16* __restrict__ x, int n
 
 template <int WARPS, int MT>
 __global__ void __launch_bounds__(WARPS * 32)
-router_mma_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, int n_k,
+router_mma_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, int n_rp, int n_k,
                   const bf16* __restrict__ w_rep, const float* __restrict__ u, const float* __restrict__ b,
                   const int32_t* __restrict__ outer_off, int n_outer,
                   float* __restrict__ scores, float* __restrict__ keys,
@@ -112,7 +112,7 @@ router_mma_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, int n
   __shared__ int row_group[ROWS];
   const int row0 = blockIdx.x * ROWS;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n2 = 2 * n_r;
+  const int n2 = 2 * n_rp;      // W^R block: n_rp gate rows (zero-padded), then n_rp up rows
   if (threadIdx.x < ROWS)
     row_group[threadIdx.x] = outer_off ? find_outer(outer_off, n_outer, min(row0 + (int)threadIdx.x, n_rows - 1)) : 0;
   __syncthreads();
@@ -125,7 +125,7 @@ router_mma_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, int n
     if (row >= n_rows) break;
     const int go = row_group[r];
     const float a = lane < n_r ? fin[r][lane] : 0.0f;
-    const float v = lane < n_r ? fin[r][n_r + lane] : 0.0f;
+    const float v = lane < n_r ? fin[r][n_rp + lane] : 0.0f;
     gate_row(lane, n_r, n_k, a, v, u + go * n_r, b + go * n_r, go * n_r, scores + (size_t)row * n_r,
              keys + (size_t)row * n_r, topk_idx + (size_t)row * n_k, topk_gate + (size_t)row * n_k);
   }

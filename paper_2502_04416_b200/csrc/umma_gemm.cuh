@@ -1,15 +1,24 @@
-// Tensor-core grouped expert GEMMs for sm_100a: tcgen05.mma with the accumulator in
-// tensor memory (TMEM), operands staged in shared memory by TMA, one persistent CTA per
-// SM, warp-specialised (TMA producer / MMA issuer / 4 epilogue warps), TMEM accumulator
+// Tensor-core kernels for sm_100a: tcgen05.mma with the accumulator in tensor memory
+// (TMEM), operands staged in shared memory by TMA, one persistent CTA per SM,
+// warp-specialised (TMA producer warp / MMA issuer / 4 epilogue warps), TMEM accumulator
 // double-buffered so the epilogue of one tile overlaps the MMAs of the next.
 //
-//   GEMM-1 (MODE 1): H[r, n] = Swish(x_r . Wg[n]) * (x_r . Wu[n])          (Eq. ori_ffn_method)
-//       A tile  : 128 rows of x (shared groups: outer-row order; routed: permuted rows) x 64 k
+//   MODE 1, gate/up GEMM: H[r, n] = Swish(x_r . Wg[n]) * (x_r . Wu[n])      (Eq. ori_ffn_method)
+//       A tile  : 128 rows of x x 64 k.  Shared groups read consecutive outer rows.  Routed
+//                 groups read a permuted copy of x, or, when the batch is small, gather
+//                 their rows straight from x with TMA tile::gather4 (4 rows per copy, one
+//                 copy per producer lane, only as many copies as the tile has rows): a
+//                 full 128-row tile needs 32 gather copies per stage, which the TMA unit
+//                 issues far slower than one tiled box, so large batches use the copy.
 //       B tile  : bn gate rows + bn up rows of the group's neurons x 64 k (one 3-D TMA box)
 //       D (TMEM): 128 lanes x 2*bn fp32 columns; epilogue fuses SiLU(gate)*up -> bf16 H
-//   GEMM-2 (MODE 2): Y[r, c] = sum_n H[r, n] Wd[c, n]
-//       A tile  : 128 rows of H x 64 k ;  B tile: 256 rows (output channels) of the group's
-//       W_down block x 64 k ;  D: 128 x 256 fp32 ; epilogue rounds to bf16 Y.
+//   MODE 2, down GEMM: Y[r, c] = sum_n H[r, n] Wd[c, n]
+//       A tile  : 128 rows of H x 64 k ;  B tile: 256 output channels of the group's W_down
+//       block x 64 k ;  D: 128 x 256 fp32 ; epilogue rounds to bf16 Y.
+//   MODE 3, router: a_j = x_r . w_gate^{R_j}, v_j = x_r . w_up^{R_j}          (Eq. router)
+//       B tile  : the (outer) layer's padded representative rows, gate block then up block;
+//       epilogue: one thread per row does Swish(a)*v, the softmax over all N_r scores, the
+//       biased top-N_k and the gates 1 + s'u                                 (Eq. final_gate).
 // All operands are K-major with the 128-byte swizzle; rows or k beyond a tensor's extent
 // are zero-filled by TMA, rows beyond a group's count are computed but never stored.
 //
@@ -98,6 +107,14 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm,
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
       ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
+// Four rows r0..r3 of a 2-D tensor (box: 64 columns x 1 row) to four consecutive 128-byte rows.
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int r0,
+                                            int r1, int r2, int r3) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(cols)
                : "memory");
@@ -124,7 +141,7 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 // 16 consecutive fp32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
   uint32_t r[16];
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
@@ -157,38 +174,113 @@ struct UmmaArgs {
   const GroupStatic* gs;
   const GroupRows* gr;
   int n_groups, n_outer, n_r;
-  int d;                 // model width: K of GEMM-1, N of GEMM-2
-  int bn_s, bn_r;        // GEMM-1 neurons per tile for shared / routed groups
-  int d_ff, shared_width;
-  bf16* out_s;           // GEMM-1: H_s ; GEMM-2: Y_s
-  bf16* out_r;           // GEMM-1: H_r ; GEMM-2: Y_r
+  int d;                 // model width: K of modes 1 and 3, N of mode 2
+  int bn_s, bn_r;        // mode 1: neurons per tile for shared / routed groups
+  bf16* out_s;           // mode 1: H_s ; mode 2: Y_s
+  bf16* out_r;           // mode 1: H_r ; mode 2: Y_r
   int ld_out_s, ld_out_r;
+  const int32_t* row_token;   // mode 1: outer row held by each routed row (gather source)
+  int use_gather;             // mode 1: routed A rows via gather4 from x instead of the permuted copy
   int32_t* err;
+  // mode 3 (router)
+  const int32_t* outer_off;   // row ranges of the outer experts, or null (one range [0, n_rows))
+  int n_rows, n_rp, n_k;      // n_rp: N_r rounded up to 8 (rows per block of the padded W^R)
+  const float* u;
+  const float* b;
+  float* scores;
+  float* keys;
+  int32_t* topk_idx;
+  float* topk_gate;
 };
 
-struct TileCoord { int g, mt, nt; };
+struct TileCoord { int g, mt, nt, row0, count; };
 
 template <int MODE>
-__device__ __forceinline__ int umma_n_tiles(const UmmaArgs& p, const GroupStatic& g) {
-  if (MODE == 1) {
-    const int bn = g.is_shared ? p.bn_s : p.bn_r;
-    return (g.width + bn - 1) / bn;
+__device__ __forceinline__ GroupRows umma_rows(const UmmaArgs& p, int g) {
+  if (MODE == 3) {
+    GroupRows r;
+    r.row0 = p.outer_off ? p.outer_off[g] : 0;
+    r.count = p.outer_off ? p.outer_off[g + 1] - p.outer_off[g] : p.n_rows;
+    return r;
   }
-  return g.width > 0 ? (p.d + 255) / 256 : 0;
+  return p.gr[g];
 }
 
-__device__ __forceinline__ TileCoord umma_decode(const int32_t* tile_start, int n_groups, int t,
-                                                 const GroupRows* gr) {
+template <int MODE>
+__device__ __forceinline__ int umma_n_tiles(const UmmaArgs& p, int g) {
+  if (MODE == 3) return 1;
+  const GroupStatic gs = p.gs[g];
+  if (MODE == 1) {
+    const int bn = gs.is_shared ? p.bn_s : p.bn_r;
+    return (gs.width + bn - 1) / bn;
+  }
+  return gs.width > 0 ? (p.d + 255) / 256 : 0;
+}
+
+template <int MODE>
+__device__ __forceinline__ TileCoord umma_decode(const UmmaArgs& p, const int32_t* tile_start, int n_groups,
+                                                 int t) {
   int lo = 0, hi = n_groups;                 // last g with tile_start[g] <= t
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
     if (tile_start[mid] <= t) lo = mid; else hi = mid;
   }
   const int local = t - tile_start[lo];
-  const int m_tiles = (gr[lo].count + kUmmaBM - 1) / kUmmaBM;
+  const GroupRows r = umma_rows<MODE>(p, lo);
+  const int m_tiles = (r.count + kUmmaBM - 1) / kUmmaBM;
   TileCoord c;
-  c.g = lo; c.mt = local % m_tiles; c.nt = local / m_tiles;
+  c.g = lo; c.mt = local % m_tiles; c.nt = local / m_tiles; c.row0 = r.row0; c.count = r.count;
   return c;
+}
+
+// Router epilogue for one row (Eq. router, Eq. final_gate): a[j], v[j] are the gate / up
+// pre-activations of routed expert j's representative neuron, j < n_r <= 32.
+__device__ __forceinline__ void router_row_epilogue(const float (&a)[32], const float (&v)[32], int n_r, int n_k,
+                                                    const float* __restrict__ u, const float* __restrict__ b,
+                                                    int group_base, float* __restrict__ scores_row,
+                                                    float* __restrict__ keys_row, int32_t* __restrict__ idx_row,
+                                                    float* __restrict__ gates_row) {
+  float s[32];
+  float s_max = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    s[j] = j < n_r ? silu_accurate(a[j]) * v[j] : -INFINITY;
+    s_max = fmaxf(s_max, s[j]);
+  }
+  float sum = 0.0f;
+  float e[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    e[j] = j < n_r ? expf(s[j] - s_max) : 0.0f;
+    sum += e[j];
+  }
+  float key[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    if (j < n_r) {
+      e[j] = e[j] / sum;                              // s'_j
+      const float k = e[j] + __ldg(b + j);
+      scores_row[j] = s[j];
+      keys_row[j] = k;
+      key[j] = (k != k) ? -INFINITY : k;              // NaN ranks last
+    } else {
+      key[j] = -INFINITY;
+    }
+  }
+  uint32_t taken = 0;
+  for (int i = 0; i < n_k; ++i) {
+    int who = -1;
+    float best = 0.0f, best_sp = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      if (j < n_r && !((taken >> j) & 1u) && (who < 0 || key[j] > best)) {   // ties: lower index
+        who = j; best = key[j]; best_sp = e[j];
+      }
+    }
+    taken |= 1u << who;
+    idx_row[i] = group_base + who;
+    gates_row[i] = 1.0f + best_sp * __ldg(u + who);
+  }
 }
 
 template <int MODE>
@@ -209,6 +301,7 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
   int32_t* tile_start = reinterpret_cast<int32_t*>(bars_gen + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_groups = MODE == 3 ? p.n_outer : p.n_groups;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kUmmaStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
@@ -222,71 +315,99 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
     tmem_relinquish();
   }
   // tiles of every group, then their exclusive prefix
-  for (int g = threadIdx.x; g < p.n_groups; g += blockDim.x) {
-    const int m_tiles = (p.gr[g].count + kUmmaBM - 1) / kUmmaBM;
-    tile_start[g + 1] = m_tiles * umma_n_tiles<MODE>(p, p.gs[g]);
+  for (int g = threadIdx.x; g < n_groups; g += blockDim.x) {
+    const int m_tiles = (umma_rows<MODE>(p, g).count + kUmmaBM - 1) / kUmmaBM;
+    tile_start[g + 1] = m_tiles * umma_n_tiles<MODE>(p, g);
   }
   __syncthreads();
   if (threadIdx.x == 0) {
     int run = 0;
     tile_start[0] = 0;
-    for (int g = 0; g < p.n_groups; ++g) { run += tile_start[g + 1]; tile_start[g + 1] = run; }
+    for (int g = 0; g < n_groups; ++g) { run += tile_start[g + 1]; tile_start[g + 1] = run; }
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int total_tiles = tile_start[p.n_groups];
-  const int k_blocks_fixed = (p.d + kUmmaBK - 1) / kUmmaBK;      // GEMM-1: K = d
+  const int total_tiles = tile_start[n_groups];
+  const int k_blocks_fixed = (p.d + kUmmaBK - 1) / kUmmaBK;      // modes 1 and 3: K = d
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      uint32_t it = 0;
-      bool ok = true;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-        const TileCoord c = umma_decode(tile_start, p.n_groups, t, p.gr);
-        const GroupStatic g = p.gs[c.g];
-        const int row = p.gr[c.g].row0 + c.mt * kUmmaBM;
-        const CUtensorMap* ta = g.is_shared ? &tm_a_s : &tm_a_r;
-        const CUtensorMap* tb = g.is_shared ? &tm_b_s : &tm_b_r;
-        int k_blocks, b_bytes, b_row = 0, j = 0;
-        if (MODE == 1) {
-          const int bn = g.is_shared ? p.bn_s : p.bn_r;
-          k_blocks = k_blocks_fixed;
-          b_bytes = 2 * bn * kUmmaBK * 2;
-          b_row = g.w_row0 + c.nt * bn;
-        } else {
-          k_blocks = (g.width + kUmmaBK - 1) / kUmmaBK;
-          b_bytes = kUmmaBBytes;
-          b_row = c.nt * 256;
-          j = g.is_shared ? 0 : (c.g - p.n_outer) - g.outer * p.n_r;
+    // ------------------------------------------------------------ TMA producer (whole warp)
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      const TileCoord c = umma_decode<MODE>(p, tile_start, n_groups, t);
+      GroupStatic g;
+      if (MODE != 3) g = p.gs[c.g]; else { g.is_shared = 1; g.outer = c.g; g.width = 0; g.w_row0 = 0; }
+      const int row = c.row0 + c.mt * kUmmaBM;
+      const bool gather = MODE == 1 && !g.is_shared && p.use_gather;
+      const CUtensorMap* ta = g.is_shared ? &tm_a_s : &tm_a_r;
+      const CUtensorMap* tb = g.is_shared ? &tm_b_s : &tm_b_r;
+      int k_blocks, b_bytes, b_row = 0, j = 0;
+      int a_bytes = kUmmaABytes, n_issue = 0;
+      int gr0 = 0, gr1 = 0, gr2 = 0, gr3 = 0;
+      if (MODE == 1) {
+        const int bn = g.is_shared ? p.bn_s : p.bn_r;
+        k_blocks = k_blocks_fixed;
+        b_bytes = 2 * bn * kUmmaBK * 2;
+        b_row = g.w_row0 + c.nt * bn;
+        if (gather) {                          // this lane's four rows; rows past the group repeat its last row
+          n_issue = (min(kUmmaBM, c.count - c.mt * kUmmaBM) + 3) >> 2;    // copies that carry valid rows
+          a_bytes = n_issue * 512;
+          const int last = c.row0 + c.count - 1;
+          const int r = row + 4 * lane;
+          gr0 = __ldg(p.row_token + min(r, last));
+          gr1 = __ldg(p.row_token + min(r + 1, last));
+          gr2 = __ldg(p.row_token + min(r + 2, last));
+          gr3 = __ldg(p.row_token + min(r + 3, last));
         }
-        for (int kb = 0; kb < k_blocks; ++kb, ++it) {
-          const uint32_t s = it % kUmmaStages, n = it / kUmmaStages;
-          if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
-          const uint32_t fb = full0 + 8 * s;
-          const uint32_t sa = base + s * kUmmaStageBytes, sb = sa + kUmmaABytes;
-          mbar_expect_tx(fb, kUmmaABytes + b_bytes);
+      } else if (MODE == 2) {
+        k_blocks = (g.width + kUmmaBK - 1) / kUmmaBK;
+        b_bytes = kUmmaBBytes;
+        b_row = c.nt * 256;
+        j = g.is_shared ? 0 : (c.g - p.n_outer) - g.outer * p.n_r;
+      } else {
+        k_blocks = k_blocks_fixed;
+        b_bytes = 2 * p.n_rp * kUmmaBK * 2;
+      }
+      for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+        const uint32_t s = it % kUmmaStages, n = it / kUmmaStages;
+        if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
+        const uint32_t fb = full0 + 8 * s;
+        const uint32_t sa = base + s * kUmmaStageBytes, sb = sa + kUmmaABytes;
+        if (lane == 0) mbar_expect_tx(fb, a_bytes + b_bytes);
+        __syncwarp();
+        if (gather) {
+          if (lane < n_issue) tma_gather4(sa + lane * 512, ta, fb, kb * kUmmaBK, gr0, gr1, gr2, gr3);
+        } else if (lane == 0) {
           tma_load_2d(sa, ta, fb, kb * kUmmaBK, row);
+        }
+        if (lane == 0) {
           if (MODE == 1) tma_load_3d(sb, tb, fb, kb * kUmmaBK, b_row, 0);
+          else if (MODE == 3) tma_load_3d(sb, tb, fb, kb * kUmmaBK, 0, c.g);
           else if (g.is_shared) tma_load_3d(sb, tb, fb, kb * kUmmaBK, b_row, g.outer);
           else tma_load_4d(sb, tb, fb, kb * kUmmaBK, b_row, j, g.outer);
         }
       }
-      if (!ok) for (int i = 0; i < 200; ++i) __nanosleep(1000);   // let copies in flight land
     }
+    if (!ok) for (int i = 0; i < 200; ++i) __nanosleep(1000);   // let copies in flight land
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       uint32_t it = 0, tile_n = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_n) {
-        const TileCoord c = umma_decode(tile_start, p.n_groups, t, p.gr);
-        const GroupStatic g = p.gs[c.g];
+        const TileCoord c = umma_decode<MODE>(p, tile_start, n_groups, t);
         int k_blocks, n_mma;
-        if (MODE == 1) { k_blocks = k_blocks_fixed; n_mma = 2 * (g.is_shared ? p.bn_s : p.bn_r); }
-        else { k_blocks = (g.width + kUmmaBK - 1) / kUmmaBK; n_mma = 256; }
+        if (MODE == 1) {
+          const GroupStatic g = p.gs[c.g];
+          k_blocks = k_blocks_fixed; n_mma = 2 * (g.is_shared ? p.bn_s : p.bn_r);
+        } else if (MODE == 2) {
+          k_blocks = (p.gs[c.g].width + kUmmaBK - 1) / kUmmaBK; n_mma = 256;
+        } else {
+          k_blocks = k_blocks_fixed; n_mma = 2 * p.n_rp;
+        }
         const uint32_t idesc = umma_idesc(n_mma);
         const uint32_t buf = tile_n & 1, use = tile_n >> 1;
         if (!mbar_wait(acce0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.err, kErrWaitAccEmpty)) { ok = false; break; }
@@ -312,21 +433,20 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
     uint32_t tile_n = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_n) {
-      const TileCoord c = umma_decode(tile_start, p.n_groups, t, p.gr);
-      const GroupStatic g = p.gs[c.g];
-      const GroupRows r = p.gr[c.g];
+      const TileCoord c = umma_decode<MODE>(p, tile_start, n_groups, t);
       const uint32_t buf = tile_n & 1, use = tile_n >> 1;
       if (!mbar_wait(accf0 + 8 * buf, use & 1, abort_flag, p.err, kErrWaitAccFull)) { ok = false; break; }
       tc_fence_after();
       const int row_in_group = c.mt * kUmmaBM + quad * 32 + lane;
-      const bool row_ok = row_in_group < r.count;
+      const bool row_ok = row_in_group < c.count;
       const uint32_t taddr = tmem_base + buf * 256 + ((uint32_t)(quad * 32) << 16);
       if (MODE == 1) {
+        const GroupStatic g = p.gs[c.g];
         const int bn = g.is_shared ? p.bn_s : p.bn_r;
         const int ld = g.is_shared ? p.ld_out_s : p.ld_out_r;
         const int n0 = c.nt * bn;
         const int n_valid = min(bn, g.width - n0);
-        bf16* dst = (g.is_shared ? p.out_s : p.out_r) + (size_t)(r.row0 + row_in_group) * ld + n0;
+        bf16* dst = (g.is_shared ? p.out_s : p.out_r) + (size_t)(c.row0 + row_in_group) * ld + n0;
         for (int c0 = 0; c0 < n_valid; c0 += 16) {
           float gt[16], up[16];
           tmem_ld16(taddr + c0, gt);
@@ -347,10 +467,11 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
             }
           }
         }
-      } else {
+      } else if (MODE == 2) {
+        const GroupStatic g = p.gs[c.g];
         const int n0 = c.nt * 256;
         const int n_valid = min(256, p.d - n0);
-        bf16* dst = (g.is_shared ? p.out_s : p.out_r) + (size_t)(r.row0 + row_in_group) * p.d + n0;
+        bf16* dst = (g.is_shared ? p.out_s : p.out_r) + (size_t)(c.row0 + row_in_group) * p.d + n0;
         for (int c0 = 0; c0 < n_valid; c0 += 16) {
           float acc[16];
           tmem_ld16(taddr + c0, acc);
@@ -366,6 +487,21 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
               }
             }
           }
+        }
+      } else {
+        float a[32], v[32];
+        tmem_ld16(taddr, a);
+        tmem_ld16(taddr + p.n_rp, v);
+        if (p.n_rp > 16) {                     // warp-uniform
+          tmem_ld16(taddr + 16, a + 16);
+          tmem_ld16(taddr + p.n_rp + 16, v + 16);
+        }
+        tmem_ld_wait();
+        if (row_ok) {
+          const size_t row = (size_t)(c.row0 + row_in_group);
+          router_row_epilogue(a, v, p.n_r, p.n_k, p.u + c.g * p.n_r, p.b + c.g * p.n_r, c.g * p.n_r,
+                              p.scores + row * p.n_r, p.keys + row * p.n_r, p.topk_idx + row * p.n_k,
+                              p.topk_gate + row * p.n_k);
         }
       }
       tc_fence_before();
@@ -383,8 +519,22 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
 
 // ----------------------------------------------------------------------------- host
 struct UmmaShape {
-  int d = 0, m = 0, shared_width = 0, d_ff = 0, n_outer = 1, n_r = 0;
+  int d = 0, m = 0, shared_width = 0, d_ff = 0, n_outer = 1, n_r = 0, n_rp = 0, n_k = 0;
   size_t max_outer_rows = 0, max_routed_rows = 0;
+};
+
+struct UmmaBuffers {
+  const void* w_gate_up = nullptr;   // [2][n_outer*d_ff][d]
+  const void* w_down = nullptr;      // packed W_down
+  const void* w_rep = nullptr;       // [n_outer][2*n_rp][d] padded representative rows
+  const void* x_fixed = nullptr;     // hierarchical: the layer's own outer-row copy of x
+  const void* x_perm = nullptr;      // routed rows of x in expert-contiguous order
+  void *h_s = nullptr, *h_r = nullptr, *y_s = nullptr, *y_r = nullptr;
+  const GroupStatic* gs_dev = nullptr;
+  const float *u = nullptr, *b = nullptr;
+  float *scores = nullptr, *keys = nullptr, *topk_gate = nullptr;
+  int32_t* topk_idx = nullptr;
+  const int32_t* row_token = nullptr;
 };
 
 typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -396,16 +546,18 @@ struct UmmaPlan {
   bool built = false;
   char error[256] = "";
   UmmaShape shape;
+  UmmaBuffers buf;
   int bn_s = 128, bn_r = 128, n_sms = 0, n_groups = 0;
-  const GroupStatic* gs_dev = nullptr;
+  bool has_s = false, has_r = false;
   PFN_encodeTiled encode = nullptr;
-  bool x_is_fixed = false;                 // hierarchical layers read x from their own buffer
-  CUtensorMap a1_s, a1_r, b1_s, b1_r;      // GEMM-1: x rows / permuted x rows / stacked gate+up rows
-  CUtensorMap a2_s, a2_r, b2_s, b2_r;      // GEMM-2: H_s / H_r / shared W_down / routed W_down blocks
-  bf16 *h_s = nullptr, *h_r = nullptr, *y_s = nullptr, *y_r = nullptr;
+  CUtensorMap x_rows, x_gather;            // x: 64 x 128 boxes for consecutive rows, 64 x 1 for gather4
+  CUtensorMap x_perm;                      // permuted copy of x
+  CUtensorMap b1_s, b1_r;                  // stacked gate+up rows, box heights bn_s / bn_r
+  CUtensorMap a2_s, a2_r, b2_s, b2_r;      // H_s / H_r / shared W_down / routed W_down blocks
+  CUtensorMap w_rep;                       // padded representative rows
 };
 
-// Neurons per GEMM-1 tile: the multiple of 8 in [96, 128] that wastes the least of the last tile.
+// Neurons per gate/up tile: the multiple of 8 in [96, 128] that wastes the least of the last tile.
 inline int umma_pick_bn(int width) {
   if (width <= 0) return 128;
   int best = 128, best_pad = (width + 127) / 128 * 128;
@@ -432,23 +584,29 @@ inline bool umma_encode(UmmaPlan* P, CUtensorMap* tm, const void* base, int rank
   return true;
 }
 
-// [rows, cols] row-major bf16 matrix, box 64 x 128.
+// [rows, cols] row-major bf16 matrix, box 64 columns x box_rows.
 inline bool umma_encode_rows(UmmaPlan* P, CUtensorMap* tm, const void* base, size_t rows, size_t cols,
-                             const char* what) {
+                             int box_rows, const char* what) {
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t str[1] = {cols * 2};
-  const cuuint32_t box[2] = {kUmmaBK, kUmmaBM};
+  const cuuint32_t box[2] = {kUmmaBK, (cuuint32_t)box_rows};
   return umma_encode(P, tm, base, 2, dims, str, box, what);
 }
 
+// Tensor maps of x for this forward: the caller's buffer for a plain layer (a host-side
+// struct fill, no allocation), fixed at plan creation for a hierarchical layer.
+inline bool umma_bind_x(UmmaPlan* P, const void* x_rows, int n_rows) {
+  if (P->buf.x_fixed) return true;
+  return umma_encode_rows(P, &P->x_rows, x_rows, (size_t)n_rows, (size_t)P->shape.d, kUmmaBM, "x") &&
+         umma_encode_rows(P, &P->x_gather, x_rows, (size_t)n_rows, (size_t)P->shape.d, 1, "x (gather)");
+}
+
 // 0: plan built; 1: shape not taken by this path; -5: a driver call failed (P->error).
-inline int umma_plan_create(UmmaPlan* P, const UmmaShape& s, const GroupStatic* gs_dev, int n_groups,
-                            const void* w_gate_up /* [2][n_outer*d_ff][d] */, const void* w_down,
-                            const void* x_perm, void* h_s, void* h_r, void* y_s, void* y_r,
-                            const void* x_fixed /* hierarchical: the layer's own outer-row copy of x */) {
+inline int umma_plan_create(UmmaPlan* P, const UmmaShape& s, const UmmaBuffers& buf, int n_groups) {
   P->built = false;
-  const bool has_s = s.shared_width > 0 && s.max_outer_rows > 0;
-  const bool has_r = s.n_r > 0 && s.max_routed_rows > 0;
+  P->has_s = s.shared_width > 0 && s.max_outer_rows > 0;
+  P->has_r = s.n_r > 0 && s.n_k > 0 && s.max_routed_rows > 0;
+  const bool has_s = P->has_s, has_r = P->has_r;
   if (!has_s && !has_r) return 1;
   if (s.d % 8 || s.m % 8 || s.shared_width % 8 || n_groups > kUmmaMaxGroups) return 1;
   void* fn = nullptr;
@@ -460,54 +618,59 @@ inline int umma_plan_create(UmmaPlan* P, const UmmaShape& s, const GroupStatic* 
   }
   P->encode = reinterpret_cast<PFN_encodeTiled>(fn);
   P->shape = s;
-  P->gs_dev = gs_dev;
+  P->buf = buf;
   P->n_groups = n_groups;
   P->bn_s = umma_pick_bn(s.shared_width);
   P->bn_r = umma_pick_bn(s.m);
-  P->h_s = (bf16*)h_s; P->h_r = (bf16*)h_r; P->y_s = (bf16*)y_s; P->y_r = (bf16*)y_r;
   int dev = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&P->n_sms, cudaDevAttrMultiProcessorCount, dev);
 
   const size_t d = s.d, rows_w = (size_t)s.n_outer * s.d_ff;
   bool ok = true;
-  // GEMM-1 B: gate and up stacked, [2][rows_w][d]; box = 64 k x bn rows x 2 planes
+  // gate/up weights stacked, [2][rows_w][d]; box = 64 k x bn rows x 2 planes
   for (int shared = 0; shared < 2 && ok; ++shared) {
     const int bn = shared ? P->bn_s : P->bn_r;
     const cuuint64_t dims[3] = {d, rows_w, 2};
     const cuuint64_t str[2] = {d * 2, rows_w * d * 2};
     const cuuint32_t box[3] = {kUmmaBK, (cuuint32_t)bn, 2};
-    ok = umma_encode(P, shared ? &P->b1_s : &P->b1_r, w_gate_up, 3, dims, str, box, "gate/up weights");
+    ok = umma_encode(P, shared ? &P->b1_s : &P->b1_r, buf.w_gate_up, 3, dims, str, box, "gate/up weights");
   }
-  // GEMM-1 A (routed): permuted rows of x; GEMM-2 A: H_s, H_r
-  if (ok && has_r) ok = umma_encode_rows(P, &P->a1_r, x_perm, s.max_routed_rows, d, "permuted x");
-  if (ok && has_r) ok = umma_encode_rows(P, &P->a2_r, h_r, s.max_routed_rows, s.m, "H routed");
-  if (ok && has_s) ok = umma_encode_rows(P, &P->a2_s, h_s, s.max_outer_rows, s.shared_width, "H shared");
-  // GEMM-2 B: shared block [d, W_s] of every outer expert; routed blocks [d, m] x N_r of every outer expert
+  if (ok && has_r) ok = umma_encode_rows(P, &P->a2_r, buf.h_r, s.max_routed_rows, s.m, kUmmaBM, "H routed");
+  if (ok && has_r) ok = umma_encode_rows(P, &P->x_perm, buf.x_perm, s.max_routed_rows, d, kUmmaBM, "permuted x");
+  if (ok && has_s) ok = umma_encode_rows(P, &P->a2_s, buf.h_s, s.max_outer_rows, s.shared_width, kUmmaBM, "H shared");
+  // W_down: shared block [d, W_s] of every outer expert; routed blocks [d, m] x N_r of every outer expert
   if (ok && has_s) {
     const cuuint64_t dims[3] = {(cuuint64_t)s.shared_width, d, (cuuint64_t)s.n_outer};
     const cuuint64_t str[2] = {(cuuint64_t)s.shared_width * 2, d * s.d_ff * 2};
     const cuuint32_t box[3] = {kUmmaBK, 256, 1};
-    ok = umma_encode(P, &P->b2_s, w_down, 3, dims, str, box, "shared W_down");
+    ok = umma_encode(P, &P->b2_s, buf.w_down, 3, dims, str, box, "shared W_down");
   }
   if (ok && has_r) {
     const cuuint64_t dims[4] = {(cuuint64_t)s.m, d, (cuuint64_t)s.n_r, (cuuint64_t)s.n_outer};
     const cuuint64_t str[3] = {(cuuint64_t)s.m * 2, d * s.m * 2, d * s.d_ff * 2};
     const cuuint32_t box[4] = {kUmmaBK, 256, 1, 1};
-    ok = umma_encode(P, &P->b2_r, (const bf16*)w_down + (size_t)s.shared_width * d, 4, dims, str, box,
+    ok = umma_encode(P, &P->b2_r, (const bf16*)buf.w_down + (size_t)s.shared_width * d, 4, dims, str, box,
                      "routed W_down");
   }
-  P->x_is_fixed = x_fixed != nullptr;
-  if (ok && x_fixed && has_s) ok = umma_encode_rows(P, &P->a1_s, x_fixed, s.max_outer_rows, d, "outer rows of x");
+  if (ok && s.n_r > 0) {
+    const cuuint64_t dims[3] = {d, (cuuint64_t)2 * s.n_rp, (cuuint64_t)s.n_outer};
+    const cuuint64_t str[2] = {d * 2, (cuuint64_t)2 * s.n_rp * d * 2};
+    const cuuint32_t box[3] = {kUmmaBK, (cuuint32_t)(2 * s.n_rp), 1};
+    ok = umma_encode(P, &P->w_rep, buf.w_rep, 3, dims, str, box, "representative rows");
+  }
+  if (ok && buf.x_fixed)
+    ok = umma_encode_rows(P, &P->x_rows, buf.x_fixed, s.max_outer_rows, d, kUmmaBM, "outer rows of x") &&
+         umma_encode_rows(P, &P->x_gather, buf.x_fixed, s.max_outer_rows, d, 1, "outer rows of x (gather)");
   if (!ok) return -5;
   // placeholders for absent operand classes (never dereferenced: such groups have no tiles)
-  if (!has_r) { P->a1_r = P->a2_s; P->a2_r = P->a2_s; P->b2_r = P->b2_s; }
-  if (!has_s) { P->a2_s = P->a2_r; P->b2_s = P->b2_r; P->a1_s = P->a1_r; }
-  cudaError_t e = cudaFuncSetAttribute(umma_grouped_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kUmmaSmemBytes);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(umma_grouped_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kUmmaSmemBytes);
+  if (!has_r) { P->a2_r = P->a2_s; P->b2_r = P->b2_s; }
+  if (!has_s) { P->a2_s = P->a2_r; P->b2_s = P->b2_r; }
+  if (s.n_r == 0) P->w_rep = P->b1_s;
+  cudaError_t e = cudaSuccess;
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(umma_grouped_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(umma_grouped_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(umma_grouped_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmemBytes);
   if (e != cudaSuccess) {
     snprintf(P->error, sizeof(P->error), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     return -5;
@@ -518,25 +681,45 @@ inline int umma_plan_create(UmmaPlan* P, const UmmaShape& s, const GroupStatic* 
 
 inline void umma_plan_destroy(UmmaPlan* P) { P->built = false; }
 
-// Enqueues GEMM-1 and GEMM-2 over all groups; returns the number of kernels launched, or -1
-// (P->error).  `x_rows` are the outer rows of x ([n_outer_rows, d]); for a plain layer this is
-// the caller's x, whose tensor map is encoded here (a host-side struct fill, no allocation).
-inline int umma_forward(UmmaPlan* P, const void* x_rows, int n_outer_rows, int n_routed_rows,
-                        const GroupRows* gr, int32_t* err_word, cudaStream_t st, cudaEvent_t mid) {
-  (void)n_routed_rows;
+inline UmmaArgs umma_base_args(const UmmaPlan* P, const GroupRows* gr, int32_t* err_word) {
   const UmmaShape& s = P->shape;
-  CUtensorMap a1_s = P->a1_s;
-  if (!P->x_is_fixed && s.shared_width > 0) {
-    if (!umma_encode_rows(P, &a1_s, x_rows, (size_t)n_outer_rows, (size_t)s.d, "x")) return -1;
+  UmmaArgs a{};
+  a.gs = P->buf.gs_dev; a.gr = gr; a.n_groups = P->n_groups; a.n_outer = s.n_outer; a.n_r = s.n_r;
+  a.d = s.d; a.bn_s = P->bn_s; a.bn_r = P->bn_r; a.err = err_word;
+  a.row_token = P->buf.row_token;
+  a.n_rp = s.n_rp; a.n_k = s.n_k; a.u = P->buf.u; a.b = P->buf.b;
+  a.scores = P->buf.scores; a.keys = P->buf.keys; a.topk_idx = P->buf.topk_idx; a.topk_gate = P->buf.topk_gate;
+  return a;
+}
+
+// Router on the tensor path (mode 3).  Requires umma_bind_x for this forward.  Returns launches or -1.
+inline int umma_router_forward(UmmaPlan* P, int n_rows, const int32_t* outer_off, int32_t* err_word,
+                               cudaStream_t st) {
+  UmmaArgs a = umma_base_args(P, nullptr, err_word);
+  a.outer_off = outer_off; a.n_rows = n_rows;
+  const int tiles = (n_rows + kUmmaBM - 1) / kUmmaBM + P->shape.n_outer;
+  const int grid = tiles < P->n_sms ? tiles : P->n_sms;
+  umma_grouped_kernel<3><<<grid, kUmmaThreads, kUmmaSmemBytes, st>>>(P->x_rows, P->x_rows, P->w_rep, P->w_rep, a);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    snprintf(P->error, sizeof(P->error), "tensor-core router launch: %s", cudaGetErrorString(e));
+    return -1;
   }
-  UmmaArgs a;
-  a.gs = P->gs_dev; a.gr = gr; a.n_groups = P->n_groups; a.n_outer = s.n_outer; a.n_r = s.n_r;
-  a.d = s.d; a.bn_s = P->bn_s; a.bn_r = P->bn_r; a.d_ff = s.d_ff; a.shared_width = s.shared_width;
-  a.err = err_word;
-  a.out_s = P->h_s; a.out_r = P->h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
-  umma_grouped_kernel<1><<<P->n_sms, kUmmaThreads, kUmmaSmemBytes, st>>>(a1_s, P->a1_r, P->b1_s, P->b1_r, a);
+  return 1;
+}
+
+// Enqueues the gate/up and the down GEMM over all groups.  Requires umma_bind_x for this
+// forward.  Returns the number of kernels launched, or -1 (P->error).
+inline int umma_forward(UmmaPlan* P, const GroupRows* gr, bool gather_rows, int32_t* err_word, cudaStream_t st,
+                        cudaEvent_t mid) {
+  const UmmaShape& s = P->shape;
+  UmmaArgs a = umma_base_args(P, gr, err_word);
+  a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
+  a.use_gather = gather_rows ? 1 : 0;
+  umma_grouped_kernel<1><<<P->n_sms, kUmmaThreads, kUmmaSmemBytes, st>>>(
+      P->x_rows, (gather_rows || !P->has_r) ? P->x_gather : P->x_perm, P->b1_s, P->b1_r, a);
   if (mid) cudaEventRecord(mid, st);
-  a.out_s = P->y_s; a.out_r = P->y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
+  a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
   umma_grouped_kernel<2><<<P->n_sms, kUmmaThreads, kUmmaSmemBytes, st>>>(P->a2_s, P->a2_r, P->b2_s, P->b2_r, a);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {

@@ -63,8 +63,10 @@ def check_routing(gpu_idx: np.ndarray, gpu_gate: np.ndarray, gpu_keys: np.ndarra
         return RoutingCheck(sel, gates, 0, 0)
     local = gpu_idx - (0 if group_base is None else group_base[:, None])
     assert local.min() >= 0 and local.max() < n_r, "selected expert index out of range"
-    np.testing.assert_allclose(gpu_scores, s, rtol=2e-4, atol=2e-5)
-    np.testing.assert_allclose(gpu_keys, keys, rtol=2e-4, atol=2e-5)
+    # fp32 (tensor-core) accumulation over d <= 8192 terms against fp64: ~4e-5 absolute seen
+    # on scores of magnitude ~3; 1e-4 keeps a 10x distance to the 1e-3 near-tie margin.
+    np.testing.assert_allclose(gpu_scores, s, rtol=2e-4, atol=1e-4)
+    np.testing.assert_allclose(gpu_keys, keys, rtol=2e-4, atol=1e-4)
     margin = oracle.logit_margin(s_prime, keys, top_k)
     near = margin < MARGIN
     same = np.sort(local, axis=1) == np.sort(sel, axis=1)
