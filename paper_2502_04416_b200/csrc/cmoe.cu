@@ -382,7 +382,8 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   }
 
   mark(4);
-  const int threads = d / 8 < 256 ? ((d / 8 + 31) / 32 * 32) : 256;
+  const int per_thread = (sizeof(T) == 2 && d % 16 == 0) ? 16 : 8;
+  const int threads = d / per_thread < 256 ? ((d / per_thread + 31) / 32 * 32) : 256;
   combine_kernel<T><<<n_tok, threads, 0, st>>>(
       L->cfg.n_shared > 0 ? (const T*)L->y_s : nullptr, (const T*)L->y_r, L->topk_idx, L->topk_gate,
       L->row_of, L->hier ? L->outer_row_of : nullptr, L->hier ? L->outer_w : nullptr,

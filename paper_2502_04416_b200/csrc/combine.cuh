@@ -73,6 +73,34 @@ combine_kernel(const T* __restrict__ y_s, const T* __restrict__ y_r,
     }
   }
   __syncthreads();
+  if (sizeof(T) == 2 && (d & 15) == 0) {            // bf16 rows in 32-byte pieces
+    const bf16* ys = reinterpret_cast<const bf16*>(y_s);
+    const bf16* yr = reinterpret_cast<const bf16*>(y_r);
+    bf16* o = reinterpret_cast<bf16*>(out);
+    for (int c = threadIdx.x * 16; c < d; c += blockDim.x * 16) {
+      float acc[16];
+#pragma unroll
+      for (int q = 0; q < 16; ++q) acc[q] = 0.0f;
+      for (int slot = 0; slot < outer_k; ++slot) {
+        float inner[16];
+#pragma unroll
+        for (int q = 0; q < 16; ++q) inner[q] = 0.0f;
+        if (ys) load16(ys + (size_t)s_orow[slot] * d + c, inner);
+        for (int j = 0; j < n_k; ++j) {
+          float v[16];
+          load16(yr + (size_t)s_row[slot][j] * d + c, v);
+          const float g = s_gate[slot][j];
+#pragma unroll
+          for (int q = 0; q < 16; ++q) inner[q] = fmaf(g, v[q], inner[q]);
+        }
+        const float w = s_w[slot];
+#pragma unroll
+        for (int q = 0; q < 16; ++q) acc[q] = fmaf(w, inner[q], acc[q]);
+      }
+      store16(o + (size_t)t * d + c, acc);
+    }
+    return;
+  }
   for (int c = threadIdx.x * 8; c < d; c += blockDim.x * 8) {
     float acc[8];
 #pragma unroll

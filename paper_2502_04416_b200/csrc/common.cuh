@@ -56,6 +56,26 @@ __device__ __forceinline__ void store8(float* p, const float (&v)[8]) {
   reinterpret_cast<float4*>(p)[1] = make_float4(v[4], v[5], v[6], v[7]);
 }
 
+// Sixteen consecutive bf16 elements with one 32-byte access (p 32-byte aligned).
+__device__ __forceinline__ void store16(bf16* p, const float* v) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"l"(p), "r"(pack_bf16x2(v[0], v[1])), "r"(pack_bf16x2(v[2], v[3])),
+                 "r"(pack_bf16x2(v[4], v[5])), "r"(pack_bf16x2(v[6], v[7])), "r"(pack_bf16x2(v[8], v[9])),
+                 "r"(pack_bf16x2(v[10], v[11])), "r"(pack_bf16x2(v[12], v[13])), "r"(pack_bf16x2(v[14], v[15]))
+               : "memory");
+}
+__device__ __forceinline__ void load16(const bf16* p, float* v) {
+  uint32_t w[8];
+  asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+               : "l"(p));
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

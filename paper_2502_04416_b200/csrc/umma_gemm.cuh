@@ -447,22 +447,27 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
         const int n0 = c.nt * bn;
         const int n_valid = min(bn, g.width - n0);
         bf16* dst = (g.is_shared ? p.out_s : p.out_r) + (size_t)(c.row0 + row_in_group) * ld + n0;
+        const bool wide = ((ld | n0) & 15) == 0;          // 32-byte aligned row segments
         for (int c0 = 0; c0 < n_valid; c0 += 16) {
           float gt[16], up[16];
           tmem_ld16(taddr + c0, gt);
           tmem_ld16(taddr + bn + c0, up);
           tmem_ld_wait();
           if (row_ok) {
+            float h16[16];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              if (c0 + h * 8 < n_valid) {
-                float v[8];
+            for (int q = 0; q < 16; ++q) h16[q] = gt[q] / (1.0f + __expf(-gt[q])) * up[q];
+            if (wide && c0 + 16 <= n_valid) {
+              store16(dst + c0, h16);
+            } else {
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                  const float a = gt[h * 8 + q];
-                  v[q] = a / (1.0f + __expf(-a)) * up[h * 8 + q];
+              for (int h = 0; h < 2; ++h) {
+                if (c0 + h * 8 < n_valid) {
+                  float v[8];
+#pragma unroll
+                  for (int q = 0; q < 8; ++q) v[q] = h16[h * 8 + q];
+                  store8(dst + c0 + h * 8, v);
                 }
-                store8(dst + c0 + h * 8, v);
               }
             }
           }
@@ -472,11 +477,14 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
         const int n0 = c.nt * 256;
         const int n_valid = min(256, p.d - n0);
         bf16* dst = (g.is_shared ? p.out_s : p.out_r) + (size_t)(c.row0 + row_in_group) * p.d + n0;
+        const bool wide = (p.d & 15) == 0;
         for (int c0 = 0; c0 < n_valid; c0 += 16) {
           float acc[16];
           tmem_ld16(taddr + c0, acc);
           tmem_ld_wait();
-          if (row_ok) {
+          if (row_ok && wide && c0 + 16 <= n_valid) {
+            store16(dst + c0, acc);
+          } else if (row_ok) {
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
               if (c0 + h * 8 < n_valid) {
