@@ -210,20 +210,38 @@ def run_gpu(args):
             dist.all_reduce(ms, op=dist.ReduceOp.MAX)
         return float(ms.item())
 
-    # ---- device-resident throughput, with per-stage events for the roofline
+    # ---- device-resident throughput.  Large batches: direct launches with per-stage events for
+    # the roofline.  Small batches are launch-bound, so the forward (same C-ABI call, same
+    # kernels) is captured once into a CUDA graph and replayed; stage events are off there.
+    use_graph = args.graph == "on" or (args.graph == "auto" and T <= 512)
     sampler = ClockSampler(local)
     sampler.start()
-    layer.enable_stage_timing(min(args.steps, 4096))
+    if use_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for _ in range(3):
+                layer.forward(x, out)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            layer.forward(x, out)
+        step = graph.replay
+    else:
+        layer.enable_stage_timing(min(args.steps, 4096))
+        step = lambda: layer.forward(x, out)
     for _ in range(args.warmup):
-        layer.forward(x, out)
-    layer.enable_stage_timing(min(args.steps, 4096))          # reset the ring after warm-up
+        step()
+    if not use_graph:
+        layer.enable_stage_timing(min(args.steps, 4096))      # reset the ring after warm-up
     sampler.wait_first()
     sampler.mark_begin()
-    ms_total = timed(lambda: layer.forward(x, out), args.steps)
+    ms_total = timed(step, args.steps)
     sampler.mark_end()
     time.sleep(0.12)                                          # let the sample that covers the end arrive
     clocks = sampler.stop()
-    stage_ms, n_cov = layer.stage_times()
+    stage_ms, n_cov = layer.stage_times() if not use_graph else ([0.0] * binding.N_STAGES, 0)
     launches = layer.launch_count() * args.steps
     assert layer.status() == 0, "device-side wait timed out"
     layer.enable_stage_timing(0)
@@ -244,7 +262,7 @@ def run_gpu(args):
 
     def e2e_step():
         x.copy_(x_pin, non_blocking=True)
-        layer.forward(x, out)
+        step()
         out_pin.copy_(out, non_blocking=True)
     for _ in range(max(args.warmup, 3)):
         e2e_step()
@@ -289,8 +307,8 @@ def run_gpu(args):
     flops = mult * T * 6 * s.d_model * s.m * (s.n_shared + s.top_k)
     w_bytes = (w.n_outer if w.n_outer else 1) * (s.n_shared + touched) * s.expert_weight_bytes()
     alg_bytes = w_bytes + 2 * T * s.d_model * s.elem_bytes
-    gemm_ms = (stage_ms[2] + stage_ms[3]) / max(n_cov, 1)
     step_ms = ms_total / args.steps
+    gemm_ms = (stage_ms[2] + stage_ms[3]) / max(n_cov, 1) if not use_graph else step_ms
     t_tensor = flops / (peaks["bf16_tflops"] * 1e12)
     t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
     if t_tensor >= t_hbm:
@@ -302,7 +320,9 @@ def run_gpu(args):
         ach = alg_bytes / (gemm_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": ach / peaks["hbm_gbs"]}
-    roof.update({"kernel": "expert GEMMs (gate/up + SwiGLU, down)", "kernel_ms": gemm_ms,
+    roof.update({"kernel": ("expert GEMMs (gate/up + SwiGLU, down)" if not use_graph else
+                            "whole forward, all kernels (CUDA graph replay; no per-stage events)"),
+                 "kernel_ms": gemm_ms,
                  "peak_source": peaks["source"], "traffic": None,
                  "whole_step_frac": (t_tensor if t_tensor >= t_hbm else t_hbm) / (step_ms * 1e-3),
                  "stage_ms": {n: v / max(n_cov, 1) for n, v in zip(binding.STAGE_NAMES, stage_ms)}})
@@ -320,7 +340,8 @@ def run_gpu(args):
         "config": {"workload": f"{w.name} T={T}", "note": w.note, "d_model": s.d_model,
                    "d_ff": s.d_ff, "experts": f"S{s.n_shared}A{s.top_k}E{s.n_experts}",
                    "tokens_per_step": T, "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "l2": "weights (%.0f MB) exceed the 126 MB L2" % (w_bytes / 1e6)},
+                   "l2": "weights (%.0f MB) exceed the 126 MB L2" % (w_bytes / 1e6),
+                   "launch": "CUDA graph replay" if use_graph else "direct launches"},
         "e2e": {"value": world * T * args.steps / (e2e_ms * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": io_bytes, "d2h_bytes_per_step": io_bytes},
         "gpu_launches": launches, "clocks": clocks, "roofline": roof, "cpu_baseline": cpu,
@@ -373,6 +394,8 @@ def main():
     ap.add_argument("--workload", default="c2_llama2_7b", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--tokens", type=int, default=0, help="tokens per step (default: the workload's largest T)")
     ap.add_argument("--cpu-sample-tokens", type=int, default=256)
+    ap.add_argument("--graph", choices=["auto", "on", "off"], default="auto",
+                    help="replay the forward from a CUDA graph (auto: batches of at most 512 tokens)")
     ap.add_argument("--forward-only", action="store_true",
                     help="run only the timed forward passes (for profiler captures)")
     args = ap.parse_args()

@@ -19,6 +19,7 @@
 #include "router.cuh"
 #include "router_mma.cuh"
 #include "simt_gemm.cuh"
+#include "umma_decode.cuh"
 #include "umma_gemm.cuh"
 
 using namespace cmoe;
@@ -96,6 +97,9 @@ struct cmoe_layer {
   void* xo = nullptr;
   int32_t* err_word = nullptr;
   UmmaPlan umma;
+  DecodePlan decode;
+  float* rsk_part = nullptr;    // split-K router partial sums [slices][64 rows][64]
+  int32_t* rsk_ticket = nullptr;
 
   cudaStream_t last_stream = nullptr;
   int last_T = 0;
@@ -192,6 +196,8 @@ void carve_workspace(cmoe_layer* L, char* base) {
   L->perm_scratch = a.take<int32_t>(permute_scratch_bytes((int)R, (int)(G ? G : 1)) / 4);
   L->gr = a.take<GroupRows>(L->n_groups_total());
   L->err_word = a.take<int32_t>(1);
+  L->rsk_ticket = a.take<int32_t>(1);
+  L->rsk_part = a.take<float>((size_t)kRskMaxSlices * kRskMaxRows * 64);
   L->x_perm = a.take<char>(P * d * esz);
   L->h_s = a.take<char>(R * L->shared_width() * esz);
   L->h_r = a.take<char>(P * L->m * esz);
@@ -254,6 +260,7 @@ int finish_layer(cmoe_layer* L, cudaStream_t st) {
     rc = umma_plan_create(&L->umma, s, ub, L->n_groups_total());
     if (rc == CMOE_ERR_CUDA) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     L->umma_ok = (rc == CMOE_OK);
+    if (L->umma_ok && !decode_plan_create(&L->umma, &L->decode)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   }
   CU_TRY(cudaStreamSynchronize(st));
   return CMOE_OK;
@@ -317,7 +324,9 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
     xo = (const T*)L->xo;
   }
 
+  const bool decode = use_umma && R <= kDecMaxRows;      // weights-on-M streaming kernels
   if (use_umma && !umma_bind_x(&L->umma, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
+  if (decode && !decode_bind_x(&L->umma, &L->decode, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   if (n_r > 0) {
     const int warps = (R + 1) / 2, blocks = (warps + 7) / 8;
     const int32_t* ooff = L->hier ? L->outer_off : nullptr;
@@ -329,6 +338,10 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
       if (use_umma && R >= 512) {
         if (umma_router_forward(&L->umma, R, ooff, L->err_word, st) < 0)
           return arg_fail(CMOE_ERR_CUDA, L->umma.error);
+      } else if (R <= kRskMaxRows && d <= kRskMaxSlices * kRskSliceK) {
+        router_splitk_kernel<<<(d + kRskSliceK - 1) / kRskSliceK, kRskThreads, 0, st>>>(
+            xo, R, d, n_r, L->n_rp, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->rsk_part,
+            L->rsk_ticket, L->scores, L->keys, L->topk_idx, L->topk_gate);
       } else {
         router_mma_kernel<8, 1><<<(R + 15) / 16, 256, 0, st>>>(
             xo, R, d, n_r, L->n_rp, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->scores,
@@ -351,7 +364,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
                                         L->counts, L->offsets, L->gr);
   ++launches;
   // Small batches: the tensor path gathers routed rows inside its TMA producer instead.
-  const bool tma_gather = use_umma && P <= kTmaGatherMaxRows;
+  const bool tma_gather = use_umma && (decode || P <= kTmaGatherMaxRows);
   if (P > 0 && !tma_gather) {
     gather_rows_kernel<<<P, 256, 0, st>>>((const uint4*)xo, L->row_token, P, row_vec, (uint4*)L->x_perm);
     ++launches;
@@ -359,7 +372,8 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
 
   mark(2);
   if (use_umma) {
-    const int n = umma_forward(&L->umma, L->gr, tma_gather, L->err_word, st, ev ? ev[3] : nullptr);
+    const int n = decode ? decode_forward(&L->umma, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
+                         : umma_forward(&L->umma, L->gr, tma_gather, L->err_word, st, ev ? ev[3] : nullptr);
     if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     launches += n;
   } else {

@@ -172,3 +172,107 @@ outer_router_mma_kernel(const bf16* __restrict__ x, int n_tokens, int d, int n_o
 }
 
 }  // namespace cmoe
+
+namespace cmoe {
+
+// ---------------------------------------------------------------------------------------
+// Router for at most kRskMaxRows rows (decode): the dot products are split over K across
+// the grid so that every 16-byte load of x and W^R is in flight at once instead of in a
+// per-warp sequence.  Block s owns the k slice [128 s, 128 s + 128); a warp takes one
+// (16-row tile, 64-wide half slice) unit; the block adds its two halves in a fixed order
+// and writes the slice's partial sums to scratch [slice][row][64]; the block that takes
+// the last ticket adds the slices in ascending order (deterministic) and runs the gate
+// logic, then resets the ticket for the next call.
+constexpr int kRskMaxRows = 64;
+constexpr int kRskSliceK = 128;
+constexpr int kRskMaxSlices = 64;           // d <= 8192
+constexpr int kRskThreads = 256;
+
+__global__ void __launch_bounds__(kRskThreads)
+router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, int n_rp, int n_k,
+                     const bf16* __restrict__ w_rep, const float* __restrict__ u, const float* __restrict__ b,
+                     const int32_t* __restrict__ outer_off, int n_outer,
+                     float* __restrict__ part /*[slices][kRskMaxRows][64]*/, int32_t* __restrict__ ticket,
+                     float* __restrict__ scores, float* __restrict__ keys,
+                     int32_t* __restrict__ topk_idx, float* __restrict__ topk_gate) {
+  __shared__ float unit[8][16][kRmStride];       // [unit = half*m_tiles + m-tile][row in tile][n]
+  __shared__ int row_group[kRskMaxRows];
+  __shared__ int is_last;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int n2 = 2 * n_rp, n_tiles = n2 >> 3;
+  const int m_tiles = (n_rows + 15) >> 4;
+  const int k_base = blockIdx.x * kRskSliceK;
+  for (int r = threadIdx.x; r < kRskMaxRows; r += kRskThreads)
+    row_group[r] = (outer_off && r < n_rows) ? find_outer(outer_off, n_outer, r) : 0;
+  __syncthreads();
+  const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+  const int un = warp;                           // at most 2 * 4 units for 8 warps
+  if (un < 2 * m_tiles) {
+    const int mt = un % m_tiles, half = un / m_tiles;
+    const int r_lo = min(mt * 16 + g, n_rows - 1), r_hi = min(mt * 16 + g + 8, n_rows - 1);
+    const int k0 = k_base + half * 64 + 8 * t, k1 = k0 + 32;
+    const bool in0 = k0 < d, in1 = k1 < d;
+    const uint4 a0_lo = in0 ? __ldg(reinterpret_cast<const uint4*>(xo + (size_t)r_lo * d + k0)) : zero;
+    const uint4 a0_hi = in0 ? __ldg(reinterpret_cast<const uint4*>(xo + (size_t)r_hi * d + k0)) : zero;
+    const uint4 a1_lo = in1 ? __ldg(reinterpret_cast<const uint4*>(xo + (size_t)r_lo * d + k1)) : zero;
+    const uint4 a1_hi = in1 ? __ldg(reinterpret_cast<const uint4*>(xo + (size_t)r_hi * d + k1)) : zero;
+    const int g_first = row_group[mt * 16], g_last = row_group[min(mt * 16 + 15, n_rows - 1)];
+    for (int go = g_first; go <= g_last; ++go) {       // one pass unless the tile straddles outer experts
+      const bf16* w = w_rep + (size_t)go * n2 * d;
+      uint4 b0[8], b1[8];
+#pragma unroll
+      for (int nt = 0; nt < 8; ++nt) {
+        const bf16* wr = w + (size_t)(nt * 8 + g) * d;
+        b0[nt] = (nt < n_tiles && in0) ? __ldg(reinterpret_cast<const uint4*>(wr + k0)) : zero;
+        b1[nt] = (nt < n_tiles && in1) ? __ldg(reinterpret_cast<const uint4*>(wr + k1)) : zero;
+      }
+      const bool take_lo = row_group[r_lo] == go, take_hi = row_group[r_hi] == go;
+#pragma unroll
+      for (int nt = 0; nt < 8; ++nt) {
+        if (nt < n_tiles) {
+          float acc[4] = {0.f, 0.f, 0.f, 0.f};
+          mma_bf16_16816(acc, a0_lo.x, a0_hi.x, a0_lo.y, a0_hi.y, b0[nt].x, b0[nt].y);
+          mma_bf16_16816(acc, a0_lo.z, a0_hi.z, a0_lo.w, a0_hi.w, b0[nt].z, b0[nt].w);
+          mma_bf16_16816(acc, a1_lo.x, a1_hi.x, a1_lo.y, a1_hi.y, b1[nt].x, b1[nt].y);
+          mma_bf16_16816(acc, a1_lo.z, a1_hi.z, a1_lo.w, a1_hi.w, b1[nt].z, b1[nt].w);
+          const int col = nt * 8 + 2 * t;
+          if (take_lo) { unit[un][g][col] = acc[0]; unit[un][g][col + 1] = acc[1]; }
+          if (take_hi) { unit[un][g + 8][col] = acc[2]; unit[un][g + 8][col + 1] = acc[3]; }
+        }
+      }
+    }
+  }
+  __syncthreads();
+  // slice partial = first half + second half
+  float* mine = part + (size_t)blockIdx.x * kRskMaxRows * 64;
+  for (int i = threadIdx.x; i < m_tiles * 16 * 64; i += kRskThreads) {
+    const int r = i >> 6, n = i & 63;
+    if (n < n2 && r < n_rows) {
+      const int mt = r >> 4, rr = r & 15;
+      mine[r * 64 + n] = unit[mt][rr][n] + unit[m_tiles + mt][rr][n];
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1) == (int)gridDim.x - 1);
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  for (int r = warp; r < n_rows; r += kRskThreads / 32) {
+    float a = 0.0f, v = 0.0f;
+    if (lane < n_r) {
+      for (int s = 0; s < (int)gridDim.x; ++s) {           // ascending slices: deterministic
+        const float* ps = part + ((size_t)s * kRskMaxRows + r) * 64;
+        a += __ldcg(ps + lane);
+        v += __ldcg(ps + n_rp + lane);
+      }
+    }
+    const int go = row_group[r];
+    gate_row(lane, n_r, n_k, a, v, u + go * n_r, b + go * n_r, go * n_r, scores + (size_t)r * n_r,
+             keys + (size_t)r * n_r, topk_idx + (size_t)r * n_k, topk_gate + (size_t)r * n_k);
+  }
+  if (threadIdx.x == 0) *ticket = 0;
+}
+
+}  // namespace cmoe

@@ -1,0 +1,322 @@
+// Decode-shaped expert GEMMs (at most 64 rows per group): the contraction is turned
+// around so that the WEIGHTS sit on the 128-row M side of the tcgen05 MMA and the few
+// tokens on the N side (N = row count rounded up to 16).  The tensor-core time per
+// 64-wide k block is then a few dozen cycles instead of the 512 a 128-row token tile
+// costs, so a CTA can stream its weight rows as fast as TMA delivers them: the regime is
+// HBM-bound on the active experts' weight bytes and the kernel is a weight streamer with
+// deep TMA pipelines (5 x 40 KB or 8 x 24 KB in flight per SM).
+//
+//   MODE 4, gate/up:  Dg[n, t] = Wg[n] . x_t ,  Du[n, t] = Wu[n] . x_t  (two MMAs sharing
+//       the token tile), epilogue H[t, n] = Swish(Dg) * Du           (Eq. ori_ffn_method)
+//       tile = 128 neurons of one group; routed groups gather their token rows from x
+//       with TMA tile::gather4 (ceil(count/4) copies per stage).
+//   MODE 5, down:     D[c, t] = Wd[c] . H_t ,  epilogue Y[t, c] = D
+//       tile = 128 output channels of one group.
+// Tiles are dealt to the persistent CTAs in snake order (left to right, then right to
+// left), which balances the long shared-expert tiles against the short routed ones.
+// Same warp roles, bounded waits and teardown as the token-major kernels.
+#pragma once
+
+#include "umma_gemm.cuh"
+
+namespace cmoe {
+
+constexpr int kDecMaxRows = 64;            // rows per group this path takes
+constexpr int kDecXBytes = kDecMaxRows * kUmmaBK * 2;      // 8 KB token tile
+constexpr int kDecTmemCols = 256;          // two buffers of (64 gate + 64 up) columns
+
+template <int MODE> struct DecodeCfg;
+template <> struct DecodeCfg<4> { static constexpr int kWBytes = 2 * 128 * kUmmaBK * 2, kStages = 5; };
+template <> struct DecodeCfg<5> { static constexpr int kWBytes = 128 * kUmmaBK * 2, kStages = 8; };
+
+template <int MODE>
+constexpr int decode_smem_bytes() {
+  return 1024 + DecodeCfg<MODE>::kStages * (DecodeCfg<MODE>::kWBytes + kDecXBytes) + 256 +
+         (kUmmaMaxGroups + 1) * 4;
+}
+
+struct DecodeArgs {
+  const GroupStatic* gs;
+  const GroupRows* gr;
+  int n_groups, n_outer, n_r;
+  int d;
+  bf16* out_s;           // mode 4: H_s ; mode 5: Y_s
+  bf16* out_r;           // mode 4: H_r ; mode 5: Y_r
+  int ld_out_s, ld_out_r;
+  const int32_t* row_token;
+  int32_t* err;
+};
+
+// Tile handled by CTA `cta` in its `round`-th turn: even rounds run left to right, odd
+// rounds right to left.  Returns -1 past the end.
+__device__ __forceinline__ int snake_tile(int round, int cta, int n_ctas, int total) {
+  const int t = round * n_ctas + ((round & 1) ? n_ctas - 1 - cta : cta);
+  return t < total ? t : -1;
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_constant__ CUtensorMap tm_w_r,
+                   const __grid_constant__ CUtensorMap tm_x_s, const __grid_constant__ CUtensorMap tm_x_r,
+                   const DecodeArgs p) {
+  constexpr int kStages = DecodeCfg<MODE>::kStages;
+  constexpr int kWBytes = DecodeCfg<MODE>::kWBytes;
+  constexpr int kStageBytes = kWBytes + kDecXBytes;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - raw);
+  const uint32_t bars = base + kStages * kStageBytes;
+  uint8_t* bars_gen = gen + kStages * kStageBytes;
+  // barrier block: full[8] empty[8] acc_full[2] acc_empty[2], tmem slot, abort flag
+  const uint32_t full0 = bars, empty0 = bars + 64, accf0 = bars + 128, acce0 = bars + 144;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_gen + 160);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
+  int32_t* tile_start = reinterpret_cast<int32_t*>(bars_gen + 256);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), kDecTmemCols);
+    tmem_relinquish();
+  }
+  for (int g = threadIdx.x; g < p.n_groups; g += blockDim.x) {
+    const int span = MODE == 4 ? p.gs[g].width : (p.gs[g].width > 0 ? p.d : 0);
+    tile_start[g + 1] = p.gr[g].count > 0 ? (span + 127) / 128 : 0;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int run = 0;
+    tile_start[0] = 0;
+    for (int g = 0; g < p.n_groups; ++g) { run += tile_start[g + 1]; tile_start[g + 1] = run; }
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int total_tiles = tile_start[p.n_groups];
+  const int cta = blockIdx.x, n_ctas = gridDim.x;
+
+  auto find_group = [&](int t) {
+    int lo = 0, hi = p.n_groups;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (tile_start[mid] <= t) lo = mid; else hi = mid;
+    }
+    return lo;
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (whole warp)
+    uint32_t it = 0;
+    bool ok = true;
+    for (int round = 0; ok; ++round) {
+      const int t = snake_tile(round, cta, n_ctas, total_tiles);
+      if (t < 0) break;
+      const int gi = find_group(t), nt = t - tile_start[gi];
+      const GroupStatic g = p.gs[gi];
+      const GroupRows r = p.gr[gi];
+      const bool gather = MODE == 4 && !g.is_shared;
+      const CUtensorMap* tw = g.is_shared ? &tm_w_s : &tm_w_r;
+      const CUtensorMap* tx = g.is_shared ? &tm_x_s : &tm_x_r;
+      const int k_blocks = ((MODE == 4 ? p.d : g.width) + kUmmaBK - 1) / kUmmaBK;
+      const int j = g.is_shared ? 0 : (gi - p.n_outer) - g.outer * p.n_r;
+      int x_bytes = kDecXBytes, n_issue = 0, gr0 = 0, gr1 = 0, gr2 = 0, gr3 = 0;
+      if (gather) {
+        n_issue = (r.count + 3) >> 2;
+        x_bytes = n_issue * 512;
+        const int last = r.row0 + r.count - 1, rr = r.row0 + 4 * lane;
+        gr0 = __ldg(p.row_token + min(rr, last));
+        gr1 = __ldg(p.row_token + min(rr + 1, last));
+        gr2 = __ldg(p.row_token + min(rr + 2, last));
+        gr3 = __ldg(p.row_token + min(rr + 3, last));
+      }
+      for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+        const uint32_t s = it % kStages, n = it / kStages;
+        if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
+        const uint32_t fb = full0 + 8 * s;
+        const uint32_t sw = base + s * kStageBytes, sx = sw + kWBytes;
+        if (lane == 0) mbar_expect_tx(fb, kWBytes + x_bytes);
+        __syncwarp();
+        if (lane == 0) {
+          if (MODE == 4) tma_load_3d(sw, tw, fb, kb * kUmmaBK, g.w_row0 + nt * 128, 0);
+          else if (g.is_shared) tma_load_3d(sw, tw, fb, kb * kUmmaBK, nt * 128, g.outer);
+          else tma_load_4d(sw, tw, fb, kb * kUmmaBK, nt * 128, j, g.outer);
+        }
+        if (gather) {
+          if (lane < n_issue) tma_gather4(sx + lane * 512, tx, fb, kb * kUmmaBK, gr0, gr1, gr2, gr3);
+        } else if (lane == 0) {
+          tma_load_2d(sx, tx, fb, kb * kUmmaBK, r.row0);
+        }
+      }
+    }
+    if (!ok) for (int i = 0; i < 200; ++i) __nanosleep(1000);
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int round = 0; ok; ++round) {
+        const int t = snake_tile(round, cta, n_ctas, total_tiles);
+        if (t < 0) break;
+        const int gi = find_group(t);
+        const GroupStatic g = p.gs[gi];
+        const int k_blocks = ((MODE == 4 ? p.d : g.width) + kUmmaBK - 1) / kUmmaBK;
+        const int n_mma = (p.gr[gi].count + 15) & ~15;               // tokens rounded up to 16
+        const uint32_t idesc = umma_idesc(n_mma);
+        const uint32_t buf = round & 1, use = round >> 1;
+        if (!mbar_wait(acce0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.err, kErrWaitAccEmpty)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * 128;
+        for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+          const uint32_t s = it % kStages, n = it / kStages;
+          if (!mbar_wait(full0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sw = base + s * kStageBytes, sx = sw + kWBytes;
+#pragma unroll
+          for (int k = 0; k < kUmmaBK / 16; ++k) {
+            const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
+            umma_bf16(d_tmem, umma_smem_desc(sw + k * 32), umma_smem_desc(sx + k * 32), idesc, acc);
+            if (MODE == 4)
+              umma_bf16(d_tmem + 64, umma_smem_desc(sw + 128 * kUmmaBK * 2 + k * 32),
+                        umma_smem_desc(sx + k * 32), idesc, acc);
+          }
+          umma_commit(empty0 + 8 * s);
+        }
+        if (ok) umma_commit(accf0 + 8 * buf);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int quad = warp & 3;
+    bool ok = true;
+    for (int round = 0; ok; ++round) {
+      const int t = snake_tile(round, cta, n_ctas, total_tiles);
+      if (t < 0) break;
+      const int gi = find_group(t), nt = t - tile_start[gi];
+      const GroupStatic g = p.gs[gi];
+      const GroupRows r = p.gr[gi];
+      const uint32_t buf = round & 1, use = round >> 1;
+      if (!mbar_wait(accf0 + 8 * buf, use & 1, abort_flag, p.err, kErrWaitAccFull)) { ok = false; break; }
+      tc_fence_after();
+      const int wr = nt * 128 + quad * 32 + lane;                 // neuron (mode 4) / channel (mode 5)
+      const int span = MODE == 4 ? g.width : p.d;
+      const int ld = MODE == 4 ? (g.is_shared ? p.ld_out_s : p.ld_out_r) : p.d;
+      bf16* dst = (g.is_shared ? p.out_s : p.out_r) + (size_t)r.row0 * ld + wr;
+      const uint32_t taddr = tmem_base + buf * 128 + ((uint32_t)(quad * 32) << 16);
+      for (int c0 = 0; c0 < r.count; c0 += 16) {
+        float a[16], b[16];
+        tmem_ld16(taddr + c0, a);
+        if (MODE == 4) tmem_ld16(taddr + 64 + c0, b);
+        tmem_ld_wait();
+        if (wr < span) {
+#pragma unroll
+          for (int q = 0; q < 16; ++q) {
+            if (c0 + q < r.count) {
+              const float v = MODE == 4 ? a[q] / (1.0f + __expf(-a[q])) * b[q] : a[q];
+              dst[(size_t)(c0 + q) * ld] = __float2bfloat16_rn(v);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acce0 + 8 * buf);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kDecTmemCols);
+  }
+}
+
+// ----------------------------------------------------------------------------- host
+struct DecodePlan {
+  bool built = false;
+  CUtensorMap w_gu;                 // stacked gate/up rows, box 64 k x 128 rows x 2 planes
+  CUtensorMap wd_s, wd_r;           // W_down blocks, 128-channel boxes
+  CUtensorMap x_rows64;             // x, 64-row boxes (bound per forward for a plain layer)
+  CUtensorMap h_s, h_r;             // H, 64-row boxes
+};
+
+inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
+  const UmmaShape& s = P->shape;
+  const UmmaBuffers& buf = P->buf;
+  const size_t d = s.d, rows_w = (size_t)s.n_outer * s.d_ff;
+  bool ok = true;
+  {
+    const cuuint64_t dims[3] = {d, rows_w, 2};
+    const cuuint64_t str[2] = {d * 2, rows_w * d * 2};
+    const cuuint32_t box[3] = {kUmmaBK, 128, 2};
+    ok = umma_encode(P, &D->w_gu, buf.w_gate_up, 3, dims, str, box, "gate/up weights (decode)");
+  }
+  if (ok && P->has_s) {
+    const cuuint64_t dims[3] = {(cuuint64_t)s.shared_width, d, (cuuint64_t)s.n_outer};
+    const cuuint64_t str[2] = {(cuuint64_t)s.shared_width * 2, d * s.d_ff * 2};
+    const cuuint32_t box[3] = {kUmmaBK, 128, 1};
+    ok = umma_encode(P, &D->wd_s, buf.w_down, 3, dims, str, box, "shared W_down (decode)") &&
+         umma_encode_rows(P, &D->h_s, buf.h_s, s.max_outer_rows, s.shared_width, kDecMaxRows, "H shared (decode)");
+  }
+  if (ok && P->has_r) {
+    const cuuint64_t dims[4] = {(cuuint64_t)s.m, d, (cuuint64_t)s.n_r, (cuuint64_t)s.n_outer};
+    const cuuint64_t str[3] = {(cuuint64_t)s.m * 2, d * s.m * 2, d * s.d_ff * 2};
+    const cuuint32_t box[4] = {kUmmaBK, 128, 1, 1};
+    ok = umma_encode(P, &D->wd_r, (const bf16*)buf.w_down + (size_t)s.shared_width * d, 4, dims, str, box,
+                     "routed W_down (decode)") &&
+         umma_encode_rows(P, &D->h_r, buf.h_r, s.max_routed_rows, s.m, kDecMaxRows, "H routed (decode)");
+  }
+  if (ok && buf.x_fixed)
+    ok = umma_encode_rows(P, &D->x_rows64, buf.x_fixed, s.max_outer_rows, d, kDecMaxRows, "outer rows of x (decode)");
+  if (!ok) return false;
+  if (!P->has_r) { D->wd_r = D->wd_s; D->h_r = D->h_s; }
+  if (!P->has_s) { D->wd_s = D->wd_r; D->h_s = D->h_r; }
+  cudaError_t e = cudaFuncSetAttribute(umma_decode_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       decode_smem_bytes<4>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(umma_decode_kernel<5>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             decode_smem_bytes<5>());
+  if (e != cudaSuccess) {
+    snprintf(P->error, sizeof(P->error), "cudaFuncSetAttribute (decode): %s", cudaGetErrorString(e));
+    return false;
+  }
+  D->built = true;
+  return true;
+}
+
+inline bool decode_bind_x(UmmaPlan* P, DecodePlan* D, const void* x_rows, int n_rows) {
+  if (P->buf.x_fixed) return true;
+  return umma_encode_rows(P, &D->x_rows64, x_rows, (size_t)n_rows, (size_t)P->shape.d, kDecMaxRows, "x (decode)");
+}
+
+// Both decode GEMMs; requires umma_bind_x and decode_bind_x for this forward and at most
+// kDecMaxRows outer rows.  Returns launches or -1.
+inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int32_t* err_word, cudaStream_t st,
+                          cudaEvent_t mid) {
+  const UmmaShape& s = P->shape;
+  DecodeArgs a{};
+  a.gs = P->buf.gs_dev; a.gr = gr; a.n_groups = P->n_groups; a.n_outer = s.n_outer; a.n_r = s.n_r;
+  a.d = s.d; a.row_token = P->buf.row_token; a.err = err_word;
+  a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
+  umma_decode_kernel<4><<<P->n_sms, kUmmaThreads, decode_smem_bytes<4>(), st>>>(D->w_gu, D->w_gu, D->x_rows64,
+                                                                             P->x_gather, a);
+  if (mid) cudaEventRecord(mid, st);
+  a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
+  umma_decode_kernel<5><<<P->n_sms, kUmmaThreads, decode_smem_bytes<5>(), st>>>(D->wd_s, D->wd_r, D->h_s, D->h_r, a);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    snprintf(P->error, sizeof(P->error), "decode GEMM launch: %s", cudaGetErrorString(e));
+    return -1;
+  }
+  return 2;
+}
+
+}  // namespace cmoe
