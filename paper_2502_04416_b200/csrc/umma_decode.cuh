@@ -8,8 +8,10 @@
 //
 //   MODE 4, gate/up:  Dg[n, t] = Wg[n] . x_t ,  Du[n, t] = Wu[n] . x_t  (two MMAs sharing
 //       the token tile), epilogue H[t, n] = Swish(Dg) * Du           (Eq. ori_ffn_method)
-//       tile = 128 neurons of one group; routed groups gather their token rows from x
-//       with TMA tile::gather4 (ceil(count/4) copies per stage).
+//       tile = 128 neurons of one group.  The token tile is ALL rows of the group's outer
+//       expert (the whole batch for a plain layer): with tokens on the N side the extra
+//       columns cost almost nothing, every group shares one tiled TMA box, and a routed
+//       group's epilogue simply stores the columns of the tokens that selected it.
 //   MODE 5, down:     D[c, t] = Wd[c] . H_t ,  epilogue Y[t, c] = D
 //       tile = 128 output channels of one group.
 // Tiles are dealt to the persistent CTAs in snake order (left to right, then right to
@@ -25,14 +27,15 @@ constexpr int kDecMaxRows = 64;            // rows per group this path takes
 constexpr int kDecXBytes = kDecMaxRows * kUmmaBK * 2;      // 8 KB token tile
 constexpr int kDecTmemCols = 256;          // two buffers of (64 gate + 64 up) columns
 
+constexpr int kDecInvOff = 256 + ((kUmmaMaxGroups + 1) * 4 + 15) / 16 * 16;   // per-warp token tables
+
 template <int MODE> struct DecodeCfg;
 template <> struct DecodeCfg<4> { static constexpr int kWBytes = 2 * 128 * kUmmaBK * 2, kStages = 5; };
 template <> struct DecodeCfg<5> { static constexpr int kWBytes = 128 * kUmmaBK * 2, kStages = 8; };
 
 template <int MODE>
 constexpr int decode_smem_bytes() {
-  return 1024 + DecodeCfg<MODE>::kStages * (DecodeCfg<MODE>::kWBytes + kDecXBytes) + 256 +
-         (kUmmaMaxGroups + 1) * 4;
+  return 1024 + DecodeCfg<MODE>::kStages * (DecodeCfg<MODE>::kWBytes + kDecXBytes) + kDecInvOff + 4 * 64 * 4;
 }
 
 struct DecodeArgs {
@@ -73,6 +76,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_gen + 160);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
   int32_t* tile_start = reinterpret_cast<int32_t*>(bars_gen + 256);
+  int32_t* inv_tables = reinterpret_cast<int32_t*>(bars_gen + kDecInvOff);     // [4 warps][64]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -122,39 +126,25 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
       if (t < 0) break;
       const int gi = find_group(t), nt = t - tile_start[gi];
       const GroupStatic g = p.gs[gi];
-      const GroupRows r = p.gr[gi];
-      const bool gather = MODE == 4 && !g.is_shared;
+      // mode 4: token rows of the group's outer expert; mode 5: the group's own H rows
+      const GroupRows r = MODE == 4 ? p.gr[g.outer] : p.gr[gi];
       const CUtensorMap* tw = g.is_shared ? &tm_w_s : &tm_w_r;
       const CUtensorMap* tx = g.is_shared ? &tm_x_s : &tm_x_r;
       const int k_blocks = ((MODE == 4 ? p.d : g.width) + kUmmaBK - 1) / kUmmaBK;
       const int j = g.is_shared ? 0 : (gi - p.n_outer) - g.outer * p.n_r;
-      int x_bytes = kDecXBytes, n_issue = 0, gr0 = 0, gr1 = 0, gr2 = 0, gr3 = 0;
-      if (gather) {
-        n_issue = (r.count + 3) >> 2;
-        x_bytes = n_issue * 512;
-        const int last = r.row0 + r.count - 1, rr = r.row0 + 4 * lane;
-        gr0 = __ldg(p.row_token + min(rr, last));
-        gr1 = __ldg(p.row_token + min(rr + 1, last));
-        gr2 = __ldg(p.row_token + min(rr + 2, last));
-        gr3 = __ldg(p.row_token + min(rr + 3, last));
-      }
       for (int kb = 0; kb < k_blocks; ++kb, ++it) {
         const uint32_t s = it % kStages, n = it / kStages;
         if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
         const uint32_t fb = full0 + 8 * s;
         const uint32_t sw = base + s * kStageBytes, sx = sw + kWBytes;
-        if (lane == 0) mbar_expect_tx(fb, kWBytes + x_bytes);
-        __syncwarp();
         if (lane == 0) {
+          mbar_expect_tx(fb, kWBytes + kDecXBytes);
           if (MODE == 4) tma_load_3d(sw, tw, fb, kb * kUmmaBK, g.w_row0 + nt * 128, 0);
           else if (g.is_shared) tma_load_3d(sw, tw, fb, kb * kUmmaBK, nt * 128, g.outer);
           else tma_load_4d(sw, tw, fb, kb * kUmmaBK, nt * 128, j, g.outer);
-        }
-        if (gather) {
-          if (lane < n_issue) tma_gather4(sx + lane * 512, tx, fb, kb * kUmmaBK, gr0, gr1, gr2, gr3);
-        } else if (lane == 0) {
           tma_load_2d(sx, tx, fb, kb * kUmmaBK, r.row0);
         }
+        __syncwarp();
       }
     }
     if (!ok) for (int i = 0; i < 200; ++i) __nanosleep(1000);
@@ -169,7 +159,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         const int gi = find_group(t);
         const GroupStatic g = p.gs[gi];
         const int k_blocks = ((MODE == 4 ? p.d : g.width) + kUmmaBK - 1) / kUmmaBK;
-        const int n_mma = (p.gr[gi].count + 15) & ~15;               // tokens rounded up to 16
+        const int n_mma = ((MODE == 4 ? p.gr[g.outer].count : p.gr[gi].count) + 15) & ~15;   // columns, rounded to 16
         const uint32_t idesc = umma_idesc(n_mma);
         const uint32_t buf = round & 1, use = round >> 1;
         if (!mbar_wait(acce0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.err, kErrWaitAccEmpty)) { ok = false; break; }
@@ -211,7 +201,21 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
       const int ld = MODE == 4 ? (g.is_shared ? p.ld_out_s : p.ld_out_r) : p.d;
       bf16* dst = (g.is_shared ? p.out_s : p.out_r) + (size_t)r.row0 * ld + wr;
       const uint32_t taddr = tmem_base + buf * 128 + ((uint32_t)(quad * 32) << 16);
-      for (int c0 = 0; c0 < r.count; c0 += 16) {
+      // Columns of the accumulator: mode 5 and shared groups, the group's own rows in order;
+      // routed groups in mode 4, every row of the outer expert -> position in the group or -1.
+      const bool lookup = MODE == 4 && !g.is_shared;
+      int32_t* inv = inv_tables + quad * 64;
+      int n_cols = r.count;
+      if (lookup) {
+        const GroupRows rs = p.gr[g.outer];
+        n_cols = rs.count;
+        __syncwarp();
+        inv[lane] = -1; inv[lane + 32] = -1;
+        __syncwarp();
+        for (int c = lane; c < r.count; c += 32) inv[__ldg(p.row_token + r.row0 + c) - rs.row0] = c;
+        __syncwarp();
+      }
+      for (int c0 = 0; c0 < n_cols; c0 += 16) {
         float a[16], b[16];
         tmem_ld16(taddr + c0, a);
         if (MODE == 4) tmem_ld16(taddr + 64 + c0, b);
@@ -219,9 +223,12 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         if (wr < span) {
 #pragma unroll
           for (int q = 0; q < 16; ++q) {
-            if (c0 + q < r.count) {
-              const float v = MODE == 4 ? a[q] / (1.0f + __expf(-a[q])) * b[q] : a[q];
-              dst[(size_t)(c0 + q) * ld] = __float2bfloat16_rn(v);
+            if (c0 + q < n_cols) {
+              const int pos = lookup ? inv[c0 + q] : c0 + q;
+              if (pos >= 0) {
+                const float v = MODE == 4 ? a[q] / (1.0f + __expf(-a[q])) * b[q] : a[q];
+                dst[(size_t)pos * ld] = __float2bfloat16_rn(v);
+              }
             }
           }
         }
@@ -307,7 +314,7 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int32
   a.d = s.d; a.row_token = P->buf.row_token; a.err = err_word;
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
   umma_decode_kernel<4><<<P->n_sms, kUmmaThreads, decode_smem_bytes<4>(), st>>>(D->w_gu, D->w_gu, D->x_rows64,
-                                                                             P->x_gather, a);
+                                                                             D->x_rows64, a);
   if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
   umma_decode_kernel<5><<<P->n_sms, kUmmaThreads, decode_smem_bytes<5>(), st>>>(D->wd_s, D->wd_r, D->h_s, D->h_r, a);
