@@ -164,6 +164,21 @@ def prepare_inputs(name: str):
     return inputs
 
 
+# DRAM bytes (read + write) per forward of the dominant kernels from the ncu captures summarised
+# under profiles/ (taken on this kernel version); None where no capture exists.
+NCU_TRAFFIC = {
+    ("c2_llama2_7b", 4096): {"bytes": 287.3e6 + 38.6e6 + 135.4e6 + 68.4e6,
+                             "source": "profiles/umma_grouped_gemm_c2_llama2_7b_T4096.md"},
+}
+
+
+def traffic_note(name, tokens, use_graph):
+    rec = NCU_TRAFFIC.get((name, tokens))
+    if rec is None or use_graph:
+        return None
+    return rec["bytes"]
+
+
 # ------------------------------------------------------------------ GPU arm
 def run_gpu(args):
     import torch
@@ -323,7 +338,7 @@ def run_gpu(args):
     roof.update({"kernel": ("expert GEMMs (gate/up + SwiGLU, down)" if not use_graph else
                             "whole forward, all kernels (CUDA graph replay; no per-stage events)"),
                  "kernel_ms": gemm_ms,
-                 "peak_source": peaks["source"], "traffic": None,
+                 "peak_source": peaks["source"], "traffic": traffic_note(w.name, T, use_graph),
                  "whole_step_frac": (t_tensor if t_tensor >= t_hbm else t_hbm) / (step_ms * 1e-3),
                  "stage_ms": {n: v / max(n_cov, 1) for n, v in zip(binding.STAGE_NAMES, stage_ms)}})
 
