@@ -179,6 +179,21 @@ def traffic_note(name, tokens, use_graph):
     return rec["bytes"]
 
 
+def max_over_ranks(ms_local: float, device: str) -> float:
+    """Slowest rank's device time: the job's time when every rank runs its own replica."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(world: int, tokens_per_step: int, steps: int, ms_max: float) -> float:
+    """Whole-job tokens/s of `world` independent replicas (tokens shard with no exchange)."""
+    return world * tokens_per_step * steps / (ms_max * 1e-3)
+
+
 # ------------------------------------------------------------------ GPU arm
 def run_gpu(args):
     import torch
@@ -220,10 +235,7 @@ def run_gpu(args):
             fn()
         e1.record(stream)
         barrier()
-        ms = torch.tensor([e0.elapsed_time(e1)], device="cuda")
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
+        return max_over_ranks(e0.elapsed_time(e1), "cuda")
 
     # ---- device-resident throughput.  Large batches: direct launches with per-stage events for
     # the roofline.  Small batches are launch-bound, so the forward (same C-ABI call, same
@@ -260,7 +272,7 @@ def run_gpu(args):
     launches = layer.launch_count() * args.steps
     assert layer.status() == 0, "device-side wait timed out"
     layer.enable_stage_timing(0)
-    value = world * T * args.steps / (ms_total * 1e-3)
+    value = replica_throughput(world, T, args.steps, ms_total)
 
     if args.forward_only:                     # profiling runs: nothing but the forward passes
         if rank == 0:
