@@ -19,6 +19,7 @@
 #include "router.cuh"
 #include "router_mma.cuh"
 #include "simt_gemm.cuh"
+#include "umma2_gemm.cuh"
 #include "umma_decode.cuh"
 #include "umma_gemm.cuh"
 
@@ -45,6 +46,7 @@ int arg_fail(int code, const char* what) {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+constexpr int kPairMinRows = 1024;       // outer rows from which the expert GEMMs run on CTA pairs
 constexpr int kTmaGatherMaxRows = 512;   // routed rows up to which gather4 replaces the permuted copy of x
 
 // Bump allocator over one device allocation (base == nullptr: measure only).
@@ -98,6 +100,7 @@ struct cmoe_layer {
   int32_t* err_word = nullptr;
   UmmaPlan umma;
   DecodePlan decode;
+  Umma2Plan pair;
   float* rsk_part = nullptr;    // split-K router partial sums [slices][64 rows][64]
   int32_t* rsk_ticket = nullptr;
 
@@ -261,6 +264,7 @@ int finish_layer(cmoe_layer* L, cudaStream_t st) {
     if (rc == CMOE_ERR_CUDA) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     L->umma_ok = (rc == CMOE_OK);
     if (L->umma_ok && !decode_plan_create(&L->umma, &L->decode)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
+    if (L->umma_ok && !umma2_plan_create(&L->umma, &L->pair)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   }
   CU_TRY(cudaStreamSynchronize(st));
   return CMOE_OK;
@@ -295,7 +299,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   const int row_vec = d * (int)sizeof(T) / 16;
   int launches = 0;
   const T* xo = x;
-  const bool use_umma = L->umma_ok && L->gemm_path != 1;
+  const bool use_umma = L->umma_ok && L->gemm_path != 1;     // 2: tensor, 3: tensor without CTA pairs
   cudaEvent_t* ev = L->ev_ring ? &L->ev[(size_t)(L->ev_count % L->ev_ring) * (CMOE_N_STAGES + 1)] : nullptr;
   auto mark = [&](int i) { if (ev) cudaEventRecord(ev[i], st); };
   mark(0);
@@ -372,7 +376,10 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
 
   mark(2);
   if (use_umma) {
+    // CTA pairs (256-row tiles) once the batch is large enough to fill them
+    const bool pairs = !decode && !tma_gather && R >= kPairMinRows && L->gemm_path != 3;
     const int n = decode ? decode_forward(&L->umma, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
+                : pairs  ? umma2_forward(&L->umma, &L->pair, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
                          : umma_forward(&L->umma, L->gr, tma_gather, L->err_word, st, ev ? ev[3] : nullptr);
     if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     launches += n;
@@ -577,8 +584,8 @@ int cmoe_layer_set_gate_params(cmoe_layer* L, const float* u, const float* b, vo
 }
 
 int cmoe_layer_set_gemm_path(cmoe_layer* L, int32_t path) {
-  if (!L || path < 0 || path > 2) return arg_fail(CMOE_ERR_INVALID_ARG, "gemm path");
-  if (path == 2 && !L->umma_ok)
+  if (!L || path < 0 || path > 3) return arg_fail(CMOE_ERR_INVALID_ARG, "gemm path");
+  if (path >= 2 && !L->umma_ok)
     return arg_fail(CMOE_ERR_INVALID_ARG, "tensor-core path not available for this layer");
   L->gemm_path = path;
   return CMOE_OK;
