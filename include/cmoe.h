@@ -111,7 +111,8 @@ int cmoe_layer_set_gate_params(cmoe_layer* layer, const float* gate_scale_u,
 
 /* Choose the expert-GEMM implementation: 0 = automatic (tensor-core path when the
  * dtype is bf16 and the shape allows, else the plain SIMT path), 1 = always SIMT,
- * 2 = tensor-core, 3 = tensor-core restricted to single-CTA tiles (no cta_group::2 pairs);
+ * 2 = tensor-core (single-CTA tiles), 3 = tensor-core on CTA pairs (cta_group::2) for batches
+ * of at least 1024 rows;
  * 2 and 3 return CMOE_ERR_INVALID_ARG if the layer cannot take the tensor-core path. */
 int cmoe_layer_set_gemm_path(cmoe_layer* layer, int32_t path);
 

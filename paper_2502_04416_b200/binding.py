@@ -13,7 +13,7 @@ import numpy as np
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcmoe.so")
 
 CMOE_BF16, CMOE_FP32 = 0, 1
-GEMM_AUTO, GEMM_SIMT, GEMM_TENSOR, GEMM_TENSOR_1CTA = 0, 1, 2, 3
+GEMM_AUTO, GEMM_SIMT, GEMM_TENSOR, GEMM_TENSOR_PAIRS = 0, 1, 2, 3
 N_STAGES = 5
 STAGE_NAMES = ["route", "permute", "gemm1_swiglu", "gemm2_down", "combine"]
 

@@ -299,7 +299,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   const int row_vec = d * (int)sizeof(T) / 16;
   int launches = 0;
   const T* xo = x;
-  const bool use_umma = L->umma_ok && L->gemm_path != 1;     // 2: tensor, 3: tensor without CTA pairs
+  const bool use_umma = L->umma_ok && L->gemm_path != 1;     // 2: tensor, 3: tensor on CTA pairs
   cudaEvent_t* ev = L->ev_ring ? &L->ev[(size_t)(L->ev_count % L->ev_ring) * (CMOE_N_STAGES + 1)] : nullptr;
   auto mark = [&](int i) { if (ev) cudaEventRecord(ev[i], st); };
   mark(0);
@@ -376,8 +376,9 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
 
   mark(2);
   if (use_umma) {
-    // CTA pairs (256-row tiles) once the batch is large enough to fill them
-    const bool pairs = !decode && !tma_gather && R >= kPairMinRows && L->gemm_path != 3;
+    // CTA pairs (cta_group::2, 256-row tiles) on request: measured equal to single-CTA tiles on
+    // even groups and slower on ragged ones (an odd m-tile count idles half a pair)
+    const bool pairs = !decode && !tma_gather && R >= kPairMinRows && L->gemm_path == 3;
     const int n = decode ? decode_forward(&L->umma, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
                 : pairs  ? umma2_forward(&L->umma, &L->pair, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
                          : umma_forward(&L->umma, L->gr, tma_gather, L->err_word, st, ev ? ev[3] : nullptr);
@@ -403,7 +404,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   }
 
   mark(4);
-  const int per_thread = (sizeof(T) == 2 && d % 16 == 0) ? 16 : 8;
+  const int per_thread = sizeof(T) == 2 ? 16 : 8;
   const int threads = d / per_thread < 256 ? ((d / per_thread + 31) / 32 * 32) : 256;
   combine_kernel<T><<<n_tok, threads, 0, st>>>(
       L->cfg.n_shared > 0 ? (const T*)L->y_s : nullptr, (const T*)L->y_r, L->topk_idx, L->topk_gate,

@@ -40,88 +40,101 @@ __global__ void plan_groups_kernel(int n_outer, int n_r, int n_tokens,
 
 // out[t] = sum_slot w[t,slot] * ( Y_s[orow] + sum_j g[orow,j] * Y_r[row_of[orow,j]] ),
 // orow = outer_row_of[t,slot] (plain layer: one slot, orow = t, w = 1).  Routed terms are
-// added in ascending group index; fp32 accumulation, one rounding to the output type.
+// added in the order of the selection (descending key), a fixed order, so results are
+// reproducible run to run; fp32 accumulation, one rounding to the output type.  Every
+// thread reads the token's few routing words itself (same addresses across the block, so
+// they broadcast from L1) and then streams its 16 (bf16) or 8 columns of every row.
 template <typename T>
 __global__ void __launch_bounds__(256)
 combine_kernel(const T* __restrict__ y_s, const T* __restrict__ y_r,
                const int32_t* __restrict__ topk_idx, const float* __restrict__ topk_gate,
                const int32_t* __restrict__ row_of, const int32_t* __restrict__ outer_row_of,
                const float* __restrict__ outer_w, int outer_k, int n_k, int d, T* __restrict__ out) {
-  __shared__ int32_t s_row[kMaxTopK][kMaxTopK];
-  __shared__ float s_gate[kMaxTopK][kMaxTopK];
-  __shared__ int32_t s_orow[kMaxTopK];
-  __shared__ float s_w[kMaxTopK];
+  (void)topk_idx;
   const int t = blockIdx.x;
-  if ((int)threadIdx.x < outer_k) {
-    const int slot = threadIdx.x;
-    const int orow = outer_row_of ? outer_row_of[(size_t)t * outer_k + slot] : t;
-    s_orow[slot] = orow;
-    s_w[slot] = outer_w ? outer_w[(size_t)t * outer_k + slot] : 1.0f;
-    int idx[kMaxTopK];
-    for (int j = 0; j < n_k; ++j) {                    // insertion sort by group index
-      const int e = topk_idx[(size_t)orow * n_k + j];
-      int p = j;
-      while (p > 0 && idx[p - 1] > e) {
-        idx[p] = idx[p - 1];
-        s_row[slot][p] = s_row[slot][p - 1];
-        s_gate[slot][p] = s_gate[slot][p - 1];
-        --p;
-      }
-      idx[p] = e;
-      s_row[slot][p] = row_of[(size_t)orow * n_k + j];
-      s_gate[slot][p] = topk_gate[(size_t)orow * n_k + j];
-    }
-  }
-  __syncthreads();
-  if (sizeof(T) == 2 && (d & 15) == 0) {            // bf16 rows in 32-byte pieces
-    const bf16* ys = reinterpret_cast<const bf16*>(y_s);
-    const bf16* yr = reinterpret_cast<const bf16*>(y_r);
-    bf16* o = reinterpret_cast<bf16*>(out);
-    for (int c = threadIdx.x * 16; c < d; c += blockDim.x * 16) {
-      float acc[16];
+  constexpr bool kWide = sizeof(T) == 2;
+  constexpr int kCols = kWide ? 16 : 8;
+  const bool wide_ok = (d % kCols) == 0;
+  for (int c = threadIdx.x * kCols; c < d; c += blockDim.x * kCols) {
+    float acc[kCols];
 #pragma unroll
-      for (int q = 0; q < 16; ++q) acc[q] = 0.0f;
-      for (int slot = 0; slot < outer_k; ++slot) {
-        float inner[16];
-#pragma unroll
-        for (int q = 0; q < 16; ++q) inner[q] = 0.0f;
-        if (ys) load16(ys + (size_t)s_orow[slot] * d + c, inner);
-        for (int j = 0; j < n_k; ++j) {
-          float v[16];
-          load16(yr + (size_t)s_row[slot][j] * d + c, v);
-          const float g = s_gate[slot][j];
-#pragma unroll
-          for (int q = 0; q < 16; ++q) inner[q] = fmaf(g, v[q], inner[q]);
-        }
-        const float w = s_w[slot];
-#pragma unroll
-        for (int q = 0; q < 16; ++q) acc[q] = fmaf(w, inner[q], acc[q]);
-      }
-      store16(o + (size_t)t * d + c, acc);
-    }
-    return;
-  }
-  for (int c = threadIdx.x * 8; c < d; c += blockDim.x * 8) {
-    float acc[8];
-#pragma unroll
-    for (int q = 0; q < 8; ++q) acc[q] = 0.0f;
+    for (int q = 0; q < kCols; ++q) acc[q] = 0.0f;
     for (int slot = 0; slot < outer_k; ++slot) {
-      float inner[8];
+      const int orow = outer_row_of ? __ldg(outer_row_of + (size_t)t * outer_k + slot) : t;
+      const float w = outer_w ? __ldg(outer_w + (size_t)t * outer_k + slot) : 1.0f;
+      float inner[kCols];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) inner[q] = 0.0f;
-      if (y_s) load8(y_s + (size_t)s_orow[slot] * d + c, inner);
-      for (int j = 0; j < n_k; ++j) {
+      for (int q = 0; q < kCols; ++q) inner[q] = 0.0f;
+      if constexpr (kWide) {
+        const bf16* ys = reinterpret_cast<const bf16*>(y_s);
+        const bf16* yr = reinterpret_cast<const bf16*>(y_r);
+        if (wide_ok) {
+          if (ys) load16(ys + (size_t)orow * d + c, inner);
+          for (int j = 0; j < n_k; ++j) {
+            const int row = __ldg(row_of + (size_t)orow * n_k + j);
+            const float g = __ldg(topk_gate + (size_t)orow * n_k + j);
+            float v[16];
+            load16(yr + (size_t)row * d + c, v);
+#pragma unroll
+            for (int q = 0; q < 16; ++q) inner[q] = fmaf(g, v[q], inner[q]);
+          }
+        } else {                                    // d % 16 == 8: two 8-column halves
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            if (c + h * 8 < d) {
+              float v[8], part[8];
+#pragma unroll
+              for (int q = 0; q < 8; ++q) part[q] = 0.0f;
+              if (ys) load8(ys + (size_t)orow * d + c + h * 8, part);
+              for (int j = 0; j < n_k; ++j) {
+                const int row = __ldg(row_of + (size_t)orow * n_k + j);
+                const float g = __ldg(topk_gate + (size_t)orow * n_k + j);
+                load8(yr + (size_t)row * d + c + h * 8, v);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) part[q] = fmaf(g, v[q], part[q]);
+              }
+#pragma unroll
+              for (int q = 0; q < 8; ++q) inner[h * 8 + q] = part[q];
+            }
+          }
+        }
+      } else {
         float v[8];
-        load8(y_r + (size_t)s_row[slot][j] * d + c, v);
-        const float g = s_gate[slot][j];
+        if (y_s) { load8(y_s + (size_t)orow * d + c, v);
 #pragma unroll
-        for (int q = 0; q < 8; ++q) inner[q] = fmaf(g, v[q], inner[q]);
+          for (int q = 0; q < 8; ++q) inner[q] = v[q]; }
+        for (int j = 0; j < n_k; ++j) {
+          const int row = __ldg(row_of + (size_t)orow * n_k + j);
+          const float g = __ldg(topk_gate + (size_t)orow * n_k + j);
+          load8(y_r + (size_t)row * d + c, v);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) inner[q] = fmaf(g, v[q], inner[q]);
+        }
       }
-      const float w = s_w[slot];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) acc[q] = fmaf(w, inner[q], acc[q]);
+      for (int q = 0; q < kCols; ++q) acc[q] = fmaf(w, inner[q], acc[q]);
     }
-    store8(out + (size_t)t * d + c, acc);
+    if constexpr (kWide) {
+      bf16* o = reinterpret_cast<bf16*>(out) + (size_t)t * d + c;
+      if (wide_ok) {
+        store16(o, acc);
+      } else {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (c + h * 8 < d) {
+            float v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v[q] = acc[h * 8 + q];
+            store8(o + h * 8, v);
+          }
+        }
+      }
+    } else {
+      float v[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) v[q] = acc[q];
+      store8(reinterpret_cast<float*>(out) + (size_t)t * d + c, v);
+    }
   }
 }
 

@@ -292,19 +292,21 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);                       // generic pointer to the aligned base
-  const uint32_t bars = base + kUmmaStages * kUmmaStageBytes;   // barrier block
-  uint8_t* bars_gen = gen + kUmmaStages * kUmmaStageBytes;
-  // barrier block: full[4] empty[4] acc_full[2] acc_empty[2] (8 B each), tmem slot, abort flag
-  const uint32_t full0 = bars, empty0 = bars + 32, accf0 = bars + 64, acce0 = bars + 80;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_gen + 96);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 100);
+  constexpr int kStages = MODE == 3 ? 8 : kUmmaStages;             // the router's B tile is at most 8 KB
+  constexpr int kStageBytes = MODE == 3 ? kUmmaABytes + 8192 : kUmmaStageBytes;
+  const uint32_t bars = base + kStages * kStageBytes;   // barrier block
+  uint8_t* bars_gen = gen + kStages * kStageBytes;
+  // barrier block: full[8] empty[8] acc_full[2] acc_empty[2] (8 B each), tmem slot, abort flag
+  const uint32_t full0 = bars, empty0 = bars + 64, accf0 = bars + 128, acce0 = bars + 144;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_gen + 160);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
   int32_t* tile_start = reinterpret_cast<int32_t*>(bars_gen + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_groups = MODE == 3 ? p.n_outer : p.n_groups;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kUmmaStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -372,10 +374,10 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
         b_bytes = 2 * p.n_rp * kUmmaBK * 2;
       }
       for (int kb = 0; kb < k_blocks; ++kb, ++it) {
-        const uint32_t s = it % kUmmaStages, n = it / kUmmaStages;
+        const uint32_t s = it % kStages, n = it / kStages;
         if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
         const uint32_t fb = full0 + 8 * s;
-        const uint32_t sa = base + s * kUmmaStageBytes, sb = sa + kUmmaABytes;
+        const uint32_t sa = base + s * kStageBytes, sb = sa + kUmmaABytes;
         if (lane == 0) mbar_expect_tx(fb, a_bytes + b_bytes);
         __syncwarp();
         if (gather) {
@@ -414,10 +416,10 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * 256;
         for (int kb = 0; kb < k_blocks; ++kb, ++it) {
-          const uint32_t s = it % kUmmaStages, n = it / kUmmaStages;
+          const uint32_t s = it % kStages, n = it / kStages;
           if (!mbar_wait(full0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = base + s * kUmmaStageBytes, sb = sa + kUmmaABytes;
+          const uint32_t sa = base + s * kStageBytes, sb = sa + kUmmaABytes;
 #pragma unroll
           for (int k = 0; k < kUmmaBK / 16; ++k)
             umma_bf16(d_tmem, umma_smem_desc(sa + k * 32), umma_smem_desc(sb + k * 32), idesc,

@@ -62,6 +62,18 @@ def test_small_shapes(name, d, m, tokens, path):
     layer.destroy()
 
 
+def test_cta_pair_gemms():
+    """Expert GEMMs on tcgen05 CTA pairs (cta_group::2): groups with odd and even m-tile counts."""
+    inp = _inputs("c2_llama2_7b", d_model=256, tokens=(1300, 1027), m=1376 // 4 * 4)
+    lay = inp.layers[0]
+    layer = parity.gpu_layer(lay, 1300)
+    layer.set_gemm_path(binding.GEMM_TENSOR_PAIRS)
+    for t in (1300, 1027):
+        st = parity.check_plain_layer(layer, lay, inp.x[:t])
+        assert st["differing"] <= st["near_tie"]
+    layer.destroy()
+
+
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
 def test_hierarchical_small(path):
     inp = _inputs("c4_hier_8x7b", d_model=256, tokens=(257,), m=224)
