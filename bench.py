@@ -335,7 +335,7 @@ def run_gpu(args):
     w_bytes = (w.n_outer if w.n_outer else 1) * (s.n_shared + touched) * s.expert_weight_bytes()
     alg_bytes = w_bytes + 2 * T * s.d_model * s.elem_bytes
     step_ms = ms_total / args.steps
-    gemm_ms = (stage_ms[2] + stage_ms[3] + stage_ms[5]) / max(n_cov, 1) if not use_graph else step_ms
+    gemm_ms = (stage_ms[2] + stage_ms[3]) / max(n_cov, 1) if not use_graph else step_ms
     t_tensor = flops / (peaks["bf16_tflops"] * 1e12)
     t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
     if t_tensor >= t_hbm:

@@ -149,15 +149,13 @@ int cmoe_layer_launch_count(const cmoe_layer* layer, int32_t* n_launches);
 
 /* Per-stage device timing with CUDA events on the forward's stream.  ring_steps > 0
  * creates a ring of events covering that many forwards (0 switches timing off);
- * while on, every forward records CMOE_N_STAGES+2 events and allocates nothing.
+ * while on, every forward records CMOE_N_STAGES+1 events and allocates nothing.
  * Stages: 0 routing (top-level router and its permutation for hierarchical layers,
- * analytical router + gates), 1 histogram/scan/permute + row gather (+ waiting for stage 5),
- * 2 gate/up GEMM with the SwiGLU epilogue (routed experts; all experts when nothing
- * overlaps), 3 down GEMM, 4 combine, 5 the shared experts' gate/up GEMM, which runs on a
- * side stream concurrently with stages 0-1 (zero when it is part of stage 2).
+ * analytical router + gates), 1 histogram/scan/permute + row gather, 2 gate/up GEMM
+ * with the SwiGLU epilogue, 3 down GEMM, 4 combine.
  * cmoe_layer_stage_times synchronises the last stream and returns, per stage, the
  * summed milliseconds over the last n_steps forwards held in the ring. */
-#define CMOE_N_STAGES 6
+#define CMOE_N_STAGES 5
 int cmoe_layer_enable_stage_timing(cmoe_layer* layer, int32_t ring_steps);
 int cmoe_layer_stage_times(cmoe_layer* layer, float* ms_sum /*[CMOE_N_STAGES]*/, int32_t* n_steps);
 

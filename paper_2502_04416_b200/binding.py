@@ -14,8 +14,8 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcmoe.so"
 
 CMOE_BF16, CMOE_FP32 = 0, 1
 GEMM_AUTO, GEMM_SIMT, GEMM_TENSOR, GEMM_TENSOR_PAIRS = 0, 1, 2, 3
-N_STAGES = 6
-STAGE_NAMES = ["route", "permute", "gemm1_swiglu", "gemm2_down", "combine", "gemm1_shared_overlapped"]
+N_STAGES = 5
+STAGE_NAMES = ["route", "permute", "gemm1_swiglu", "gemm2_down", "combine"]
 
 EXPORTS = [
     "cmoe_layer_create", "cmoe_hier_create", "cmoe_ffn_forward", "cmoe_layer_set_gate_params",

@@ -46,7 +46,6 @@ int arg_fail(int code, const char* what) {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-constexpr int kEventsPerForward = CMOE_N_STAGES + 2;   // 6 on the main stream, 2 around the side-stream GEMM
 constexpr int kPairMinRows = 1024;       // outer rows from which the expert GEMMs run on CTA pairs
 constexpr int kTmaGatherMaxRows = 512;   // routed rows up to which gather4 replaces the permuted copy of x
 
@@ -103,9 +102,6 @@ struct cmoe_layer {
   DecodePlan decode;
   Umma2Plan pair;
   float* rsk_part = nullptr;    // split-K router partial sums [slices][64 rows][64]
-  // side stream on which the shared experts' gate/up GEMM overlaps routing and permutation
-  cudaStream_t side = nullptr;
-  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   int32_t* rsk_ticket = nullptr;
 
   cudaStream_t last_stream = nullptr;
@@ -126,9 +122,6 @@ namespace {
 void free_layer(cmoe_layer* L) {
   if (!L) return;
   for (cudaEvent_t e : L->ev) cudaEventDestroy(e);
-  if (L->ev_fork) cudaEventDestroy(L->ev_fork);
-  if (L->ev_join) cudaEventDestroy(L->ev_join);
-  if (L->side) cudaStreamDestroy(L->side);
   umma_plan_destroy(&L->umma);
   cudaFree(L->w_gu); cudaFree(L->wd_p); cudaFree(L->w_rep);
   cudaFree(L->w_router); cudaFree(L->u); cudaFree(L->b); cudaFree(L->gs); cudaFree(L->ws);
@@ -272,11 +265,6 @@ int finish_layer(cmoe_layer* L, cudaStream_t st) {
     L->umma_ok = (rc == CMOE_OK);
     if (L->umma_ok && !decode_plan_create(&L->umma, &L->decode)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     if (L->umma_ok && !umma2_plan_create(&L->umma, &L->pair)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
-    if (L->umma_ok) {
-      CU_TRY(cudaStreamCreateWithFlags(&L->side, cudaStreamNonBlocking));
-      CU_TRY(cudaEventCreateWithFlags(&L->ev_fork, cudaEventDisableTiming));
-      CU_TRY(cudaEventCreateWithFlags(&L->ev_join, cudaEventDisableTiming));
-    }
   }
   CU_TRY(cudaStreamSynchronize(st));
   return CMOE_OK;
@@ -312,7 +300,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   int launches = 0;
   const T* xo = x;
   const bool use_umma = L->umma_ok && L->gemm_path != 1;     // 2: tensor, 3: tensor on CTA pairs
-  cudaEvent_t* ev = L->ev_ring ? &L->ev[(size_t)(L->ev_count % L->ev_ring) * kEventsPerForward] : nullptr;
+  cudaEvent_t* ev = L->ev_ring ? &L->ev[(size_t)(L->ev_count % L->ev_ring) * (CMOE_N_STAGES + 1)] : nullptr;
   auto mark = [&](int i) { if (ev) cudaEventRecord(ev[i], st); };
   mark(0);
 
@@ -343,32 +331,6 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   const bool decode = use_umma && R <= kDecMaxRows;      // weights-on-M streaming kernels
   if (use_umma && !umma_bind_x(&L->umma, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   if (decode && !decode_bind_x(&L->umma, &L->decode, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
-  // CTA pairs (cta_group::2, 256-row tiles) on request: measured equal to single-CTA tiles on
-  // even groups and slower on ragged ones (an odd m-tile count idles half a pair)
-  const bool pairs = use_umma && !decode && R >= kPairMinRows && L->gemm_path == 3;
-  // The shared experts do not depend on the routing: their gate/up GEMM starts on a side
-  // stream now and overlaps the router, the permutation and the row gather (which leave
-  // the tensor cores idle and fit beside the persistent GEMM CTAs on every SM).
-  const int n_shared_groups = L->n_outer, n_all_groups = L->n_groups_total();
-  const bool overlap = use_umma && !pairs && L->cfg.n_shared > 0 && n_r > 0 && n_k > 0;
-  const int32_t* ooff_plan = L->hier ? L->outer_off : nullptr;
-  if (overlap) {
-    plan_groups_kernel<<<1, 64, 0, st>>>(L->n_outer, n_r, n_tok, 0, n_shared_groups, ooff_plan, L->counts,
-                                         L->offsets, L->gr);
-    ++launches;
-    CU_TRY(cudaEventRecord(L->ev_fork, st));
-    CU_TRY(cudaStreamWaitEvent(L->side, L->ev_fork, 0));
-    if (ev) cudaEventRecord(ev[6], L->side);
-    const int n = decode ? decode_gemm1(&L->umma, &L->decode, L->gr, 0, n_shared_groups, L->err_word, L->side)
-                         : umma_gemm1(&L->umma, L->gr, false, 0, n_shared_groups, L->err_word, L->side);
-    if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
-    launches += n;
-    if (ev) cudaEventRecord(ev[7], L->side);
-    CU_TRY(cudaEventRecord(L->ev_join, L->side));
-  } else if (ev) {
-    cudaEventRecord(ev[6], st);
-    cudaEventRecord(ev[7], st);
-  }
   if (n_r > 0) {
     const int warps = (R + 1) / 2, blocks = (warps + 7) / 8;
     const int32_t* ooff = L->hier ? L->outer_off : nullptr;
@@ -377,17 +339,13 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
                                                  L->b, ooff, L->n_outer, L->scores, L->keys,      \
                                                  L->topk_idx, L->topk_gate)
     if constexpr (std::is_same<T, bf16>::value) {
-      if (use_umma && R >= 512 && !overlap) {      // needs a whole SM's shared memory: not beside the GEMM
+      if (use_umma && R >= 512) {
         if (umma_router_forward(&L->umma, R, ooff, L->err_word, st) < 0)
           return arg_fail(CMOE_ERR_CUDA, L->umma.error);
       } else if (R <= kRskMaxRows && d <= kRskMaxSlices * kRskSliceK) {
         router_splitk_kernel<<<(d + kRskSliceK - 1) / kRskSliceK, kRskThreads, 0, st>>>(
             xo, R, d, n_r, L->n_rp, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->rsk_part,
             L->rsk_ticket, L->scores, L->keys, L->topk_idx, L->topk_gate);
-      } else if (overlap) {                          // 23 KB of shared memory: fits beside a GEMM CTA
-        router_mma_kernel<4, 1><<<(R + 15) / 16, 128, 0, st>>>(
-            xo, R, d, n_r, L->n_rp, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->scores,
-            L->keys, L->topk_idx, L->topk_gate);
       } else {
         router_mma_kernel<8, 1><<<(R + 15) / 16, 256, 0, st>>>(
             xo, R, d, n_r, L->n_rp, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->scores,
@@ -406,31 +364,24 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   } else {
     mark(1);
   }
-  plan_groups_kernel<<<1, 256, 0, st>>>(L->n_outer, n_r, n_tok, overlap ? n_shared_groups : 0, n_all_groups,
-                                        ooff_plan, L->counts, L->offsets, L->gr);
+  plan_groups_kernel<<<1, 256, 0, st>>>(L->n_outer, n_r, n_tok, L->hier ? L->outer_off : nullptr,
+                                        L->counts, L->offsets, L->gr);
   ++launches;
   // Small batches: the tensor path gathers routed rows inside its TMA producer instead.
-  const bool tma_gather = use_umma && !pairs && (decode || P <= kTmaGatherMaxRows);
+  const bool tma_gather = use_umma && (decode || P <= kTmaGatherMaxRows);
   if (P > 0 && !tma_gather) {
     gather_rows_kernel<<<P, 256, 0, st>>>((const uint4*)xo, L->row_token, P, row_vec, (uint4*)L->x_perm);
     ++launches;
   }
 
-  if (overlap) CU_TRY(cudaStreamWaitEvent(st, L->ev_join, 0));
   mark(2);
-  if (use_umma && pairs) {
-    const int n = umma2_forward(&L->umma, &L->pair, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr);
-    if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
-    launches += n;
-  } else if (use_umma) {
-    const int g0 = overlap ? n_shared_groups : 0;      // the shared groups already ran on the side stream
-    int n = decode ? decode_gemm1(&L->umma, &L->decode, L->gr, g0, n_all_groups, L->err_word, st)
-                   : umma_gemm1(&L->umma, L->gr, tma_gather, g0, n_all_groups, L->err_word, st);
-    if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
-    launches += n;
-    mark(3);
-    n = decode ? decode_gemm2(&L->umma, &L->decode, L->gr, L->err_word, st)
-               : umma_gemm2(&L->umma, L->gr, L->err_word, st);
+  if (use_umma) {
+    // CTA pairs (cta_group::2, 256-row tiles) on request: measured equal to single-CTA tiles on
+    // even groups and slower on ragged ones (an odd m-tile count idles half a pair)
+    const bool pairs = !decode && !tma_gather && R >= kPairMinRows && L->gemm_path == 3;
+    const int n = decode ? decode_forward(&L->umma, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
+                : pairs  ? umma2_forward(&L->umma, &L->pair, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
+                         : umma_forward(&L->umma, L->gr, tma_gather, L->err_word, st, ev ? ev[3] : nullptr);
     if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     launches += n;
   } else {
@@ -697,7 +648,7 @@ int cmoe_layer_enable_stage_timing(cmoe_layer* L, int32_t ring_steps) {
   L->ev.clear();
   L->ev_ring = 0;
   L->ev_count = 0;
-  for (int i = 0; i < ring_steps * kEventsPerForward; ++i) {
+  for (int i = 0; i < ring_steps * (CMOE_N_STAGES + 1); ++i) {
     cudaEvent_t e;
     CU_TRY(cudaEventCreate(&e));
     L->ev.push_back(e);
@@ -714,11 +665,10 @@ int cmoe_layer_stage_times(cmoe_layer* L, float* ms_sum, int32_t* n_steps) {
   CU_TRY(cudaStreamSynchronize(L->last_stream));
   const long long n = L->ev_count < L->ev_ring ? L->ev_count : L->ev_ring;
   for (long long i = 0; i < n; ++i) {
-    cudaEvent_t* ev = &L->ev[(size_t)i * kEventsPerForward];
+    cudaEvent_t* ev = &L->ev[(size_t)i * (CMOE_N_STAGES + 1)];
     for (int s = 0; s < CMOE_N_STAGES; ++s) {
       float ms = 0.0f;
-      if (s < 5) CU_TRY(cudaEventElapsedTime(&ms, ev[s], ev[s + 1]));
-      else CU_TRY(cudaEventElapsedTime(&ms, ev[6], ev[7]));
+      CU_TRY(cudaEventElapsedTime(&ms, ev[s], ev[s + 1]));
       ms_sum[s] += ms;
     }
   }

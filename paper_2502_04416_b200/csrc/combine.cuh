@@ -20,11 +20,12 @@ gather_rows_kernel(const uint4* __restrict__ src, const int32_t* __restrict__ id
 
 // Row range of every group for this forward.  Groups: n_outer shared groups (rows of
 // the outer-row order), then n_outer*n_r routed groups (rows of the routed order).
-__global__ void plan_groups_kernel(int n_outer, int n_r, int n_tokens, int g_begin, int g_end,
+__global__ void plan_groups_kernel(int n_outer, int n_r, int n_tokens,
                                    const int32_t* __restrict__ outer_off /* null: plain layer */,
                                    const int32_t* __restrict__ counts, const int32_t* __restrict__ offsets,
                                    GroupRows* __restrict__ gr) {
-  for (int g = g_begin + threadIdx.x; g < g_end; g += blockDim.x) {
+  const int n_groups = n_outer + n_outer * n_r;
+  for (int g = threadIdx.x; g < n_groups; g += blockDim.x) {
     GroupRows r;
     if (g < n_outer) {
       r.row0 = outer_off ? outer_off[g] : 0;

@@ -100,7 +100,6 @@ struct Pair2Coord { int g, mp, nt, row0, count; };
 
 template <int MODE>
 __device__ __forceinline__ int umma2_pairs(const UmmaArgs& p, int g) {
-  if (g < p.g_begin || g >= p.g_end) return 0;
   const int m_tiles = (p.gr[g].count + kUmmaBM - 1) / kUmmaBM;
   return ((m_tiles + 1) >> 1) * umma_n_tiles<MODE>(p, g);
 }

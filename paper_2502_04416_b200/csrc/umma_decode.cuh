@@ -42,7 +42,6 @@ struct DecodeArgs {
   const GroupStatic* gs;
   const GroupRows* gr;
   int n_groups, n_outer, n_r;
-  int g_begin, g_end;    // only groups in [g_begin, g_end) are processed by this launch
   int d;
   bf16* out_s;           // mode 4: H_s ; mode 5: Y_s
   bf16* out_r;           // mode 4: H_r ; mode 5: Y_r
@@ -93,12 +92,8 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
     tmem_relinquish();
   }
   for (int g = threadIdx.x; g < p.n_groups; g += blockDim.x) {
-    int tiles = 0;
-    if (g >= p.g_begin && g < p.g_end) {
-      const int span = MODE == 4 ? p.gs[g].width : (p.gs[g].width > 0 ? p.d : 0);
-      tiles = p.gr[g].count > 0 ? (span + 127) / 128 : 0;
-    }
-    tile_start[g + 1] = tiles;
+    const int span = MODE == 4 ? p.gs[g].width : (p.gs[g].width > 0 ? p.d : 0);
+    tile_start[g + 1] = p.gr[g].count > 0 ? (span + 127) / 128 : 0;
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -309,45 +304,26 @@ inline bool decode_bind_x(UmmaPlan* P, DecodePlan* D, const void* x_rows, int n_
   return umma_encode_rows(P, &D->x_rows64, x_rows, (size_t)n_rows, (size_t)P->shape.d, kDecMaxRows, "x (decode)");
 }
 
-inline DecodeArgs decode_base_args(const UmmaPlan* P, const GroupRows* gr, int32_t* err_word) {
+// Both decode GEMMs; requires umma_bind_x and decode_bind_x for this forward and at most
+// kDecMaxRows outer rows.  Returns launches or -1.
+inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int32_t* err_word, cudaStream_t st,
+                          cudaEvent_t mid) {
   const UmmaShape& s = P->shape;
   DecodeArgs a{};
   a.gs = P->buf.gs_dev; a.gr = gr; a.n_groups = P->n_groups; a.n_outer = s.n_outer; a.n_r = s.n_r;
-  a.g_begin = 0; a.g_end = P->n_groups;
   a.d = s.d; a.row_token = P->buf.row_token; a.err = err_word;
-  return a;
-}
-
-// Decode gate/up GEMM over the groups [g_begin, g_end); requires umma_bind_x and decode_bind_x
-// for this forward and at most kDecMaxRows outer rows.  Returns launches or -1.
-inline int decode_gemm1(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int g_begin, int g_end,
-                        int32_t* err_word, cudaStream_t st) {
-  const UmmaShape& s = P->shape;
-  DecodeArgs a = decode_base_args(P, gr, err_word);
-  a.g_begin = g_begin; a.g_end = g_end;
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
   umma_decode_kernel<4><<<P->n_sms, kUmmaThreads, decode_smem_bytes<4>(), st>>>(D->w_gu, D->w_gu, D->x_rows64,
                                                                              D->x_rows64, a);
-  const cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) {
-    snprintf(P->error, sizeof(P->error), "decode gate/up GEMM launch: %s", cudaGetErrorString(e));
-    return -1;
-  }
-  return 1;
-}
-
-// Decode down GEMM over all groups.
-inline int decode_gemm2(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int32_t* err_word, cudaStream_t st) {
-  const UmmaShape& s = P->shape;
-  DecodeArgs a = decode_base_args(P, gr, err_word);
+  if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
   umma_decode_kernel<5><<<P->n_sms, kUmmaThreads, decode_smem_bytes<5>(), st>>>(D->wd_s, D->wd_r, D->h_s, D->h_r, a);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
-    snprintf(P->error, sizeof(P->error), "decode down GEMM launch: %s", cudaGetErrorString(e));
+    snprintf(P->error, sizeof(P->error), "decode GEMM launch: %s", cudaGetErrorString(e));
     return -1;
   }
-  return 1;
+  return 2;
 }
 
 }  // namespace cmoe

@@ -174,7 +174,6 @@ struct UmmaArgs {
   const GroupStatic* gs;
   const GroupRows* gr;
   int n_groups, n_outer, n_r;
-  int g_begin, g_end;    // modes 1 and 2: only groups in [g_begin, g_end) are processed by this launch
   int d;                 // model width: K of modes 1 and 3, N of mode 2
   int bn_s, bn_r;        // mode 1: neurons per tile for shared / routed groups
   bf16* out_s;           // mode 1: H_s ; mode 2: Y_s
@@ -319,12 +318,8 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
   }
   // tiles of every group, then their exclusive prefix
   for (int g = threadIdx.x; g < n_groups; g += blockDim.x) {
-    int tiles = 0;
-    if (MODE == 3 || (g >= p.g_begin && g < p.g_end)) {
-      const int m_tiles = (umma_rows<MODE>(p, g).count + kUmmaBM - 1) / kUmmaBM;
-      tiles = m_tiles * umma_n_tiles<MODE>(p, g);
-    }
-    tile_start[g + 1] = tiles;
+    const int m_tiles = (umma_rows<MODE>(p, g).count + kUmmaBM - 1) / kUmmaBM;
+    tile_start[g + 1] = m_tiles * umma_n_tiles<MODE>(p, g);
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -700,7 +695,6 @@ inline UmmaArgs umma_base_args(const UmmaPlan* P, const GroupRows* gr, int32_t* 
   const UmmaShape& s = P->shape;
   UmmaArgs a{};
   a.gs = P->buf.gs_dev; a.gr = gr; a.n_groups = P->n_groups; a.n_outer = s.n_outer; a.n_r = s.n_r;
-  a.g_begin = 0; a.g_end = P->n_groups;
   a.d = s.d; a.bn_s = P->bn_s; a.bn_r = P->bn_r; a.err = err_word;
   a.row_token = P->buf.row_token;
   a.n_rp = s.n_rp; a.n_k = s.n_k; a.u = P->buf.u; a.b = P->buf.b;
@@ -724,37 +718,25 @@ inline int umma_router_forward(UmmaPlan* P, int n_rows, const int32_t* outer_off
   return 1;
 }
 
-// Gate/up GEMM (mode 1) over the groups [g_begin, g_end).  Requires umma_bind_x for this
+// Enqueues the gate/up and the down GEMM over all groups.  Requires umma_bind_x for this
 // forward.  Returns the number of kernels launched, or -1 (P->error).
-inline int umma_gemm1(UmmaPlan* P, const GroupRows* gr, bool gather_rows, int g_begin, int g_end,
-                      int32_t* err_word, cudaStream_t st) {
+inline int umma_forward(UmmaPlan* P, const GroupRows* gr, bool gather_rows, int32_t* err_word, cudaStream_t st,
+                        cudaEvent_t mid) {
   const UmmaShape& s = P->shape;
   UmmaArgs a = umma_base_args(P, gr, err_word);
-  a.g_begin = g_begin; a.g_end = g_end;
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
   a.use_gather = gather_rows ? 1 : 0;
   umma_grouped_kernel<1><<<P->n_sms, kUmmaThreads, kUmmaSmemBytes, st>>>(
       P->x_rows, (gather_rows || !P->has_r) ? P->x_gather : P->x_perm, P->b1_s, P->b1_r, a);
-  const cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) {
-    snprintf(P->error, sizeof(P->error), "tensor-core gate/up GEMM launch: %s", cudaGetErrorString(e));
-    return -1;
-  }
-  return 1;
-}
-
-// Down GEMM (mode 2) over all groups.
-inline int umma_gemm2(UmmaPlan* P, const GroupRows* gr, int32_t* err_word, cudaStream_t st) {
-  const UmmaShape& s = P->shape;
-  UmmaArgs a = umma_base_args(P, gr, err_word);
+  if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
   umma_grouped_kernel<2><<<P->n_sms, kUmmaThreads, kUmmaSmemBytes, st>>>(P->a2_s, P->a2_r, P->b2_s, P->b2_r, a);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
-    snprintf(P->error, sizeof(P->error), "tensor-core down GEMM launch: %s", cudaGetErrorString(e));
+    snprintf(P->error, sizeof(P->error), "tensor-core GEMM launch: %s", cudaGetErrorString(e));
     return -1;
   }
-  return 1;
+  return 2;
 }
 
 }  // namespace cmoe
