@@ -306,14 +306,9 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
 
   if (L->hier) {
     if constexpr (std::is_same<T, bf16>::value) {
-      if (n_tok >= 2048)
-        outer_router_mma_kernel<4, 2><<<(n_tok + 31) / 32, 128, 0, st>>>(
-            x, n_tok, d, L->n_outer, L->outer_k, (const bf16*)L->w_router, L->outer_logits, L->outer_idx,
-            L->outer_w);
-      else
-        outer_router_mma_kernel<8, 1><<<(n_tok + 15) / 16, 256, 0, st>>>(
-            x, n_tok, d, L->n_outer, L->outer_k, (const bf16*)L->w_router, L->outer_logits, L->outer_idx,
-            L->outer_w);
+      outer_router_mma_kernel<8, 1><<<(n_tok + 15) / 16, 256, 0, st>>>(
+          x, n_tok, d, L->n_outer, L->outer_k, (const bf16*)L->w_router, L->outer_logits, L->outer_idx,
+          L->outer_w);
     } else {
       outer_router_kernel<T><<<(n_tok + 7) / 8, 256, 0, st>>>(x, n_tok, d, L->n_outer, L->outer_k,
                                                               (const T*)L->w_router, L->outer_logits,
@@ -331,6 +326,9 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   const bool decode = use_umma && R <= kDecMaxRows;      // weights-on-M streaming kernels
   if (use_umma && !umma_bind_x(&L->umma, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   if (decode && !decode_bind_x(&L->umma, &L->decode, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
+  GroupPlanOut po;                                // the permutation also writes every group's row range
+  po.gr = L->gr; po.n_outer = L->n_outer; po.n_tokens = n_tok; po.outer_off = L->hier ? L->outer_off : nullptr;
+  bool perm_fused = false;                        // decode: the router's last block also permutes
   if (n_r > 0) {
     const int warps = (R + 1) / 2, blocks = (warps + 7) / 8;
     const int32_t* ooff = L->hier ? L->outer_off : nullptr;
@@ -343,9 +341,11 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
         if (umma_router_forward(&L->umma, R, ooff, L->err_word, st) < 0)
           return arg_fail(CMOE_ERR_CUDA, L->umma.error);
       } else if (R <= kRskMaxRows && d <= kRskMaxSlices * kRskSliceK) {
+        perm_fused = G <= kRskFuseGroups;
         router_splitk_kernel<<<(d + kRskSliceK - 1) / kRskSliceK, kRskThreads, 0, st>>>(
             xo, R, d, n_r, L->n_rp, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->rsk_part,
-            L->rsk_ticket, L->scores, L->keys, L->topk_idx, L->topk_gate);
+            L->rsk_ticket, L->scores, L->keys, L->topk_idx, L->topk_gate, perm_fused ? 1 : 0, G, L->counts,
+            L->offsets, L->row_token, L->row_of, po);
       } else {
         router_mma_kernel<8, 1><<<(R + 15) / 16, 256, 0, st>>>(
             xo, R, d, n_r, L->n_rp, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->scores,
@@ -359,14 +359,15 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
 #undef CMOE_ROUTER
     ++launches;
     mark(1);
-    launches += launch_token_permute(L->topk_idx, R, n_k, G, L->counts, L->offsets, L->row_token,
-                                     L->row_of, L->perm_scratch, st);
+    if (!perm_fused)
+      launches += launch_token_permute(L->topk_idx, R, n_k, G, L->counts, L->offsets, L->row_token,
+                                       L->row_of, L->perm_scratch, st, po);
   } else {
     mark(1);
+    plan_groups_kernel<<<1, 256, 0, st>>>(L->n_outer, n_r, n_tok, L->hier ? L->outer_off : nullptr,
+                                          L->counts, L->offsets, L->gr);
+    ++launches;
   }
-  plan_groups_kernel<<<1, 256, 0, st>>>(L->n_outer, n_r, n_tok, L->hier ? L->outer_off : nullptr,
-                                        L->counts, L->offsets, L->gr);
-  ++launches;
   // Small batches: the tensor path gathers routed rows inside its TMA producer instead.
   const bool tma_gather = use_umma && (decode || P <= kTmaGatherMaxRows);
   if (P > 0 && !tma_gather) {

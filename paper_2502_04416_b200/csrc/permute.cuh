@@ -86,11 +86,36 @@ __device__ __forceinline__ void chunk_scatter(const int32_t* __restrict__ topk_i
   }
 }
 
+// Optional by-product of the permutation inside a layer's forward: the row range of every
+// expert group (n_outer shared groups over the outer rows, then the routed groups), which
+// the grouped GEMMs' tile schedulers read.  gr == nullptr: not wanted.
+struct GroupPlanOut {
+  GroupRows* gr = nullptr;
+  int n_outer = 0, n_tokens = 0;
+  const int32_t* outer_off = nullptr;    // hierarchical: row ranges of the outer experts
+};
+
+__device__ __forceinline__ void write_group_rows(const GroupPlanOut& po, int n_groups, const int32_t* counts,
+                                                 const int32_t* offsets) {
+  if (po.gr == nullptr) return;
+  for (int g = threadIdx.x; g < po.n_outer + n_groups; g += blockDim.x) {
+    GroupRows r;
+    if (g < po.n_outer) {
+      r.row0 = po.outer_off ? po.outer_off[g] : 0;
+      r.count = po.outer_off ? po.outer_off[g + 1] - po.outer_off[g] : po.n_tokens;
+    } else {
+      r.row0 = offsets[g - po.n_outer];
+      r.count = counts[g - po.n_outer];
+    }
+    po.gr[g] = r;
+  }
+}
+
 // n_rows <= kPermChunk: histogram, scan and scatter in one block.
 __global__ void __launch_bounds__(kPermChunk)
 permute_single_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k, int n_groups,
                       int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
-                      int32_t* __restrict__ row_token, int32_t* __restrict__ row_of) {
+                      int32_t* __restrict__ row_token, int32_t* __restrict__ row_of, const GroupPlanOut po) {
   extern __shared__ int32_t sm[];
   int32_t* hist = sm;                              // [n_groups]
   int32_t* offs = hist + n_groups;                 // [n_groups + 1]
@@ -101,6 +126,7 @@ permute_single_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k,
   block_scan_groups(hist, offs, n_groups, sums);
   for (int g = threadIdx.x; g < n_groups; g += blockDim.x) { counts[g] = hist[g]; offsets[g] = offs[g]; }
   if (threadIdx.x == 0) offsets[n_groups] = offs[n_groups];
+  write_group_rows(po, n_groups, hist, offs);
   chunk_scatter(topk_idx, n_rows, n_k, n_groups, row, offs, warp_cnt, row_token, row_of);
 }
 
@@ -118,7 +144,7 @@ permute_count_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k, 
 // exclusive prefixes inside the group; then the scan over groups.
 __global__ void __launch_bounds__(1024)
 permute_scan_kernel(int32_t* chunk_cnt, int n_chunks, int n_groups,
-                    int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
+                    int32_t* __restrict__ counts, int32_t* __restrict__ offsets, const GroupPlanOut po) {
   __shared__ int32_t sums[1024];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   for (int g = warp; g < n_groups; g += n_warps) {
@@ -139,6 +165,7 @@ permute_scan_kernel(int32_t* chunk_cnt, int n_chunks, int n_groups,
   }
   __syncthreads();
   block_scan_groups(counts, offsets, n_groups, sums);
+  write_group_rows(po, n_groups, counts, offsets);
 }
 
 __global__ void __launch_bounds__(kPermChunk)
@@ -164,17 +191,18 @@ inline int64_t permute_scratch_bytes(int n_rows, int n_groups) {
 // Enqueues the permutation; returns the number of kernels launched.
 inline int launch_token_permute(const int32_t* topk_idx, int n_rows, int n_k, int n_groups,
                                 int32_t* counts, int32_t* offsets, int32_t* row_token,
-                                int32_t* row_of, int32_t* scratch, cudaStream_t stream) {
+                                int32_t* row_of, int32_t* scratch, cudaStream_t stream,
+                                const GroupPlanOut po = GroupPlanOut()) {
   if (n_rows <= kPermChunk) {
     const size_t smem = (size_t)(n_groups * 2 + 1 + kPermChunk + 8 * n_groups) * sizeof(int32_t);
     permute_single_kernel<<<1, kPermChunk, smem, stream>>>(topk_idx, n_rows, n_k, n_groups, counts,
-                                                           offsets, row_token, row_of);
+                                                           offsets, row_token, row_of, po);
     return 1;
   }
   const int n_chunks = (n_rows + kPermChunk - 1) / kPermChunk;
   permute_count_kernel<<<n_chunks, kPermChunk, n_groups * sizeof(int32_t), stream>>>(
       topk_idx, n_rows, n_k, n_groups, scratch);
-  permute_scan_kernel<<<1, 1024, 0, stream>>>(scratch, n_chunks, n_groups, counts, offsets);
+  permute_scan_kernel<<<1, 1024, 0, stream>>>(scratch, n_chunks, n_groups, counts, offsets, po);
   permute_scatter_kernel<<<n_chunks, kPermChunk, 9 * n_groups * sizeof(int32_t), stream>>>(
       topk_idx, n_rows, n_k, n_groups, scratch, offsets, row_token, row_of);
   return 3;

@@ -12,6 +12,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "permute.cuh"
 #include "router.cuh"
 
 namespace cmoe {
@@ -182,11 +183,14 @@ namespace cmoe {
 // (16-row tile, 64-wide half slice) unit; the block adds its two halves in a fixed order
 // and writes the slice's partial sums to scratch [slice][row][64]; the block that takes
 // the last ticket adds the slices in ascending order (deterministic) and runs the gate
-// logic, then resets the ticket for the next call.
+// logic, then resets the ticket for the next call.  With at most kRskFuseGroups routed
+// groups the same block goes on to the histogram / scan / permutation of the selections
+// (and the groups' row ranges), which saves two launches per decode step.
 constexpr int kRskMaxRows = 64;
 constexpr int kRskSliceK = 128;
 constexpr int kRskMaxSlices = 64;           // d <= 8192
 constexpr int kRskThreads = 256;
+constexpr int kRskFuseGroups = 64;
 
 __global__ void __launch_bounds__(kRskThreads)
 router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, int n_rp, int n_k,
@@ -194,7 +198,10 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
                      const int32_t* __restrict__ outer_off, int n_outer,
                      float* __restrict__ part /*[slices][kRskMaxRows][64]*/, int32_t* __restrict__ ticket,
                      float* __restrict__ scores, float* __restrict__ keys,
-                     int32_t* __restrict__ topk_idx, float* __restrict__ topk_gate) {
+                     int32_t* topk_idx, float* __restrict__ topk_gate,
+                     int fuse_permute, int n_groups, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
+                     int32_t* __restrict__ row_token, int32_t* __restrict__ row_of, const GroupPlanOut po) {
+  static_assert(kRskThreads == kPermChunk, "the fused permutation is written for one 256-row chunk");
   __shared__ float unit[8][16][kRmStride];       // [unit = half*m_tiles + m-tile][row in tile][n]
   __shared__ int row_group[kRskMaxRows];
   __shared__ int is_last;
@@ -273,6 +280,24 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
              keys + (size_t)r * n_r, topk_idx + (size_t)r * n_k, topk_gate + (size_t)r * n_k);
   }
   if (threadIdx.x == 0) *ticket = 0;
+  if (!fuse_permute) return;
+  // ---- histogram / scan / stable permutation of the selections just written (one chunk)
+  __syncthreads();
+  int32_t* sm = reinterpret_cast<int32_t*>(&unit[0][0][0]);     // the partial sums are no longer needed
+  int32_t* hist = sm;                              // [n_groups]
+  int32_t* offs = hist + n_groups;                 // [n_groups + 1]
+  int32_t* sums = offs + n_groups + 1;             // [kPermChunk]
+  int32_t* warp_cnt = sums + kPermChunk;           // [8][n_groups]
+  int32_t* sel = warp_cnt + 8 * n_groups;          // [n_rows * n_k] copy of the selections
+  for (int i = threadIdx.x; i < n_rows * n_k; i += kRskThreads) sel[i] = __ldcg(topk_idx + i);
+  __syncthreads();
+  const int row = threadIdx.x;
+  chunk_histogram(sel, n_rows, n_k, n_groups, row, hist);
+  block_scan_groups(hist, offs, n_groups, sums);
+  for (int gq = threadIdx.x; gq < n_groups; gq += kRskThreads) { counts[gq] = hist[gq]; offsets[gq] = offs[gq]; }
+  if (threadIdx.x == 0) offsets[n_groups] = offs[n_groups];
+  write_group_rows(po, n_groups, hist, offs);
+  chunk_scatter(sel, n_rows, n_k, n_groups, row, offs, warp_cnt, row_token, row_of);
 }
 
 }  // namespace cmoe
