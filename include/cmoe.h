@@ -109,6 +109,23 @@ int cmoe_ffn_forward(cmoe_layer* layer, const void* x, int32_t T, void* out, voi
 int cmoe_layer_set_gate_params(cmoe_layer* layer, const float* gate_scale_u,
                                const float* select_bias_b, void* stream);
 
+/* Read the current gate scaling u and selection bias b back (host arrays
+ * [n_routed_groups]; either may be NULL).  Synchronises `stream`. */
+int cmoe_layer_get_gate_params(cmoe_layer* layer, float* gate_scale_u, float* select_bias_b,
+                               void* stream);
+
+/* One step of the load-balancing rule (Section 4.3) on the device, from the token counts
+ * of the LAST forward: with p_i the fraction of the routed assignments of an (outer)
+ * layer that went to its expert i, b_i -= gamma if p_i > p*_i and b_i += gamma if
+ * p_i < p*_i.  The paper's target is uniform, p* = 1/N_r, and gamma = 1e-3.
+ *   target_share: host, [n_routed_groups] or NULL (uniform); fractions per (outer) layer.
+ *   utilisation : host, [n_routed_groups] or NULL; receives p_i (the call then
+ *                 synchronises `stream`; otherwise it is asynchronous unless a target is given).
+ * Call it on the stream of the last forward (or after synchronising it).
+ * Errors: INVALID_ARG (no routed experts, no forward yet, negative gamma), CUDA. */
+int cmoe_layer_update_bias(cmoe_layer* layer, float gamma, const float* target_share,
+                           float* utilisation, void* stream);
+
 /* Choose the expert-GEMM implementation: 0 = automatic (tensor-core path when the
  * dtype is bf16 and the shape allows, else the plain SIMT path), 1 = always SIMT,
  * 2 = tensor-core (single-CTA tiles), 3 = tensor-core on CTA pairs (cta_group::2) for batches

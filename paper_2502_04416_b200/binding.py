@@ -19,7 +19,7 @@ STAGE_NAMES = ["route", "permute", "gemm1_swiglu", "gemm2_down", "combine"]
 
 EXPORTS = [
     "cmoe_layer_create", "cmoe_hier_create", "cmoe_ffn_forward", "cmoe_layer_set_gate_params",
-    "cmoe_layer_set_gemm_path", "cmoe_layer_dims", "cmoe_get_routing", "cmoe_layer_status",
+    "cmoe_layer_get_gate_params", "cmoe_layer_update_bias", "cmoe_layer_set_gemm_path", "cmoe_layer_dims", "cmoe_get_routing", "cmoe_layer_status",
     "cmoe_layer_launch_count", "cmoe_layer_enable_stage_timing", "cmoe_layer_stage_times",
     "cmoe_layer_destroy", "cmoe_token_permute_scratch_bytes",
     "cmoe_token_permute", "cmoe_token_permute_static", "cmoe_status_string", "cmoe_last_error",
@@ -57,6 +57,8 @@ def load() -> C.CDLL:
     lib.cmoe_ffn_forward.argtypes = [vp, vp, i32, vp, vp]
     lib.cmoe_layer_set_gate_params.argtypes = [vp, vp, vp, vp]
     lib.cmoe_layer_set_gemm_path.argtypes = [vp, i32]
+    lib.cmoe_layer_get_gate_params.argtypes = [vp, vp, vp, vp]
+    lib.cmoe_layer_update_bias.argtypes = [vp, C.c_float, vp, vp, vp]
     lib.cmoe_layer_dims.argtypes = [vp] + [C.POINTER(i32)] * 4
     lib.cmoe_get_routing.argtypes = [vp] * 12
     lib.cmoe_layer_status.argtypes = [vp, C.POINTER(i32)]
@@ -168,6 +170,24 @@ class Layer:
         b = None if select_bias_b is None else np.ascontiguousarray(select_bias_b, dtype=np.float32)
         _check(load().cmoe_layer_set_gate_params(self._h, _np_ptr(u), _np_ptr(b),
                                                  _stream_ptr(stream)), "cmoe_layer_set_gate_params")
+
+    def get_gate_params(self, stream=None):
+        """(gate_scale_u, select_bias_b) as float32 arrays of length n_routed_groups."""
+        n = self.dims()["n_routed_groups"]
+        u, b = np.zeros(n, np.float32), np.zeros(n, np.float32)
+        _check(load().cmoe_layer_get_gate_params(self._h, _np_ptr(u), _np_ptr(b), _stream_ptr(stream)),
+               "cmoe_layer_get_gate_params")
+        return u, b
+
+    def update_bias(self, gamma: float = 1e-3, target_share=None, want_utilisation: bool = True, stream=None):
+        """cmoe_layer_update_bias: one load-balancing step from the last forward's counts.
+        Returns the utilisation p_i (float32 [n_routed_groups]) or None."""
+        n = self.dims()["n_routed_groups"]
+        tgt = None if target_share is None else np.ascontiguousarray(target_share, dtype=np.float32)
+        util = np.zeros(n, np.float32) if want_utilisation else None
+        _check(load().cmoe_layer_update_bias(self._h, gamma, _np_ptr(tgt), _np_ptr(util),
+                                             _stream_ptr(stream)), "cmoe_layer_update_bias")
+        return util
 
     def set_gemm_path(self, path: int) -> None:
         _check(load().cmoe_layer_set_gemm_path(self._h, path), "cmoe_layer_set_gemm_path")

@@ -13,6 +13,7 @@
 #include <type_traits>
 #include <vector>
 
+#include "balance.cuh"
 #include "combine.cuh"
 #include "common.cuh"
 #include "permute.cuh"
@@ -103,6 +104,7 @@ struct cmoe_layer {
   Umma2Plan pair;
   float* rsk_part = nullptr;    // split-K router partial sums [slices][64 rows][64]
   int32_t* rsk_ticket = nullptr;
+  float *share = nullptr, *target = nullptr;   // utilisation of the last step / bias-update targets
 
   cudaStream_t last_stream = nullptr;
   int last_T = 0;
@@ -200,6 +202,8 @@ void carve_workspace(cmoe_layer* L, char* base) {
   L->gr = a.take<GroupRows>(L->n_groups_total());
   L->err_word = a.take<int32_t>(1);
   L->rsk_ticket = a.take<int32_t>(1);
+  L->share = a.take<float>(G ? G : 1);
+  L->target = a.take<float>(G ? G : 1);
   L->rsk_part = a.take<float>((size_t)kRskMaxSlices * kRskMaxRows * 64);
   L->x_perm = a.take<char>(P * d * esz);
   L->h_s = a.take<char>(R * L->shared_width() * esz);
@@ -583,6 +587,39 @@ int cmoe_ffn_forward(cmoe_layer* L, const void* x, int32_t T, void* out, void* s
 int cmoe_layer_set_gate_params(cmoe_layer* L, const float* u, const float* b, void* stream) {
   if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "null layer");
   return upload_gate_params(L, u, b, static_cast<cudaStream_t>(stream));
+}
+
+int cmoe_layer_get_gate_params(cmoe_layer* L, float* u, float* b, void* stream) {
+  if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "null layer");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t n = (size_t)L->n_outer * L->n_r;
+  if (n && u) CU_TRY(cudaMemcpyAsync(u, L->u, n * sizeof(float), cudaMemcpyDeviceToHost, st));
+  if (n && b) CU_TRY(cudaMemcpyAsync(b, L->b, n * sizeof(float), cudaMemcpyDeviceToHost, st));
+  CU_TRY(cudaStreamSynchronize(st));
+  return CMOE_OK;
+}
+
+int cmoe_layer_update_bias(cmoe_layer* L, float gamma, const float* target_share, float* utilisation,
+                           void* stream) {
+  if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "null layer");
+  if (!(gamma >= 0.0f)) return arg_fail(CMOE_ERR_INVALID_ARG, "gamma must be non-negative");
+  const size_t n = (size_t)L->n_outer * L->n_r;
+  if (n == 0 || L->cfg.top_k == 0) return arg_fail(CMOE_ERR_INVALID_ARG, "layer has no routed experts");
+  if (L->last_T == 0) return arg_fail(CMOE_ERR_INVALID_ARG, "no forward has run yet");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (target_share)
+    CU_TRY(cudaMemcpyAsync(L->target, target_share, n * sizeof(float), cudaMemcpyHostToDevice, st));
+  bias_update_kernel<<<(L->n_outer + 7) / 8, 256, 0, st>>>(L->counts, L->n_outer, L->n_r,
+                                                          target_share ? L->target : nullptr, gamma, L->b,
+                                                          L->share);
+  CU_TRY(cudaGetLastError());
+  if (utilisation) {
+    CU_TRY(cudaMemcpyAsync(utilisation, L->share, n * sizeof(float), cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
+  } else if (target_share) {
+    CU_TRY(cudaStreamSynchronize(st));      // the host array was read asynchronously
+  }
+  return CMOE_OK;
 }
 
 int cmoe_layer_set_gemm_path(cmoe_layer* L, int32_t path) {

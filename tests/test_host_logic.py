@@ -83,6 +83,8 @@ def test_null_layer_calls(lib):
     assert lib.cmoe_layer_destroy(None) == 0
     w = C.c_int32()
     assert lib.cmoe_layer_status(None, C.byref(w)) == -1
+    assert lib.cmoe_layer_update_bias(None, 1e-3, None, None, None) == -1
+    assert lib.cmoe_layer_get_gate_params(None, None, None, None) == -1
 
 
 # ------------------------------------------------------------------ workloads
