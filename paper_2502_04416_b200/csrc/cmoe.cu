@@ -372,9 +372,12 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
                                           L->counts, L->offsets, L->gr);
     ++launches;
   }
-  // Small batches: the tensor path gathers routed rows inside its TMA producer instead.
-  const bool tma_gather = use_umma && (decode || P <= kTmaGatherMaxRows);
-  if (P > 0 && !tma_gather) {
+  // The tensor path gathers routed rows inside the gate/up GEMM (decode: not at all; a few rows:
+  // TMA gather4; otherwise cp.async by dedicated warps); only CTA pairs and the SIMT path read a
+  // permuted copy of x.
+  const bool pairs = use_umma && !decode && R >= kPairMinRows && L->gemm_path == 3;
+  const int gather_mode = P <= kTmaGatherMaxRows ? 1 : 2;
+  if (P > 0 && (!use_umma || pairs)) {
     gather_rows_kernel<<<P, 256, 0, st>>>((const uint4*)xo, L->row_token, P, row_vec, (uint4*)L->x_perm);
     ++launches;
   }
@@ -383,10 +386,9 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   if (use_umma) {
     // CTA pairs (cta_group::2, 256-row tiles) on request: measured equal to single-CTA tiles on
     // even groups and slower on ragged ones (an odd m-tile count idles half a pair)
-    const bool pairs = !decode && !tma_gather && R >= kPairMinRows && L->gemm_path == 3;
     const int n = decode ? decode_forward(&L->umma, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
                 : pairs  ? umma2_forward(&L->umma, &L->pair, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
-                         : umma_forward(&L->umma, L->gr, tma_gather, L->err_word, st, ev ? ev[3] : nullptr);
+                         : umma_forward(&L->umma, L->gr, gather_mode, xo, L->err_word, st, ev ? ev[3] : nullptr);
     if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     launches += n;
   } else {

@@ -4,12 +4,14 @@
 // double-buffered so the epilogue of one tile overlaps the MMAs of the next.
 //
 //   MODE 1, gate/up GEMM: H[r, n] = Swish(x_r . Wg[n]) * (x_r . Wu[n])      (Eq. ori_ffn_method)
-//       A tile  : 128 rows of x x 64 k.  Shared groups read consecutive outer rows.  Routed
-//                 groups read a permuted copy of x, or, when the batch is small, gather
-//                 their rows straight from x with TMA tile::gather4 (4 rows per copy, one
-//                 copy per producer lane, only as many copies as the tile has rows): a
-//                 full 128-row tile needs 32 gather copies per stage, which the TMA unit
-//                 issues far slower than one tiled box, so large batches use the copy.
+//       A tile  : 128 rows of x x 64 k.  Shared groups read consecutive outer rows by TMA.
+//                 Routed groups gather their rows straight from x, so no permuted copy of
+//                 x is ever written: four extra warps (one thread per tile row) issue
+//                 16-byte cp.async copies into the 128-byte-swizzled layout the MMA expects
+//                 and arrive on the stage's barrier when their copies land.  (TMA
+//                 tile::gather4 does the same with one copy per 4 rows; it is correct but a
+//                 full tile needs 32 copies per stage, which the TMA unit issues ~3x slower
+//                 than one tiled box, so it is kept only for batches of a few rows.)
 //       B tile  : bn gate rows + bn up rows of the group's neurons x 64 k (one 3-D TMA box)
 //       D (TMEM): 128 lanes x 2*bn fp32 columns; epilogue fuses SiLU(gate)*up -> bf16 H
 //   MODE 2, down GEMM: Y[r, c] = sum_n H[r, n] Wd[c, n]
@@ -43,6 +45,7 @@ constexpr int kUmmaBBytes = 256 * kUmmaBK * 2;           // 32 KB (up to 256 B r
 constexpr int kUmmaStageBytes = kUmmaABytes + kUmmaBBytes;
 constexpr int kUmmaMaxGroups = 1088;
 constexpr int kUmmaThreads = 192;     // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr int kUmmaGatherThreads = 128;   // mode 1 only: warps 6..9, one thread per A-tile row
 constexpr int kUmmaTmemCols = 512;    // two accumulator buffers of 256 columns
 constexpr int kUmmaSmemBytes = 1024 /*alignment slack*/ + kUmmaStages * kUmmaStageBytes +
                                256 /*barriers*/ + (kUmmaMaxGroups + 1) * 4;
@@ -180,7 +183,8 @@ struct UmmaArgs {
   bf16* out_r;           // mode 1: H_r ; mode 2: Y_r
   int ld_out_s, ld_out_r;
   const int32_t* row_token;   // mode 1: outer row held by each routed row (gather source)
-  int use_gather;             // mode 1: routed A rows via gather4 from x instead of the permuted copy
+  int use_gather;             // mode 1, routed A rows: 0 permuted copy by TMA, 1 TMA gather4 from x, 2 cp.async from x
+  const bf16* x_rows_ptr;     // mode 1: the outer rows of x (source of the cp.async gather)
   int32_t* err;
   // mode 3 (router)
   const int32_t* outer_off;   // row ranges of the outer experts, or null (one range [0, n_rows))
@@ -284,7 +288,7 @@ __device__ __forceinline__ void router_row_epilogue(const float (&a)[32], const 
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(kUmmaThreads, 1)
+__global__ void __launch_bounds__(MODE == 1 ? kUmmaThreads + kUmmaGatherThreads : kUmmaThreads, 1)
 umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_constant__ CUtensorMap tm_a_r,
                     const __grid_constant__ CUtensorMap tm_b_s, const __grid_constant__ CUtensorMap tm_b_r,
                     const UmmaArgs p) {
@@ -306,7 +310,9 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
   const int n_groups = MODE == 3 ? p.n_outer : p.n_groups;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    // mode 1: besides the producer's expect_tx arrival, every gather thread arrives once per stage
+    const uint32_t full_count = MODE == 1 ? 1 + kUmmaGatherThreads : 1;
+    for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, full_count); mbar_init(empty0 + 8 * s, 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -343,7 +349,8 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
       GroupStatic g;
       if (MODE != 3) g = p.gs[c.g]; else { g.is_shared = 1; g.outer = c.g; g.width = 0; g.w_row0 = 0; }
       const int row = c.row0 + c.mt * kUmmaBM;
-      const bool gather = MODE == 1 && !g.is_shared && p.use_gather;
+      const bool gather = MODE == 1 && !g.is_shared && p.use_gather == 1;
+      const bool by_threads = MODE == 1 && !g.is_shared && p.use_gather == 2;   // the gather warps fill A
       const CUtensorMap* ta = g.is_shared ? &tm_a_s : &tm_a_r;
       const CUtensorMap* tb = g.is_shared ? &tm_b_s : &tm_b_r;
       int k_blocks, b_bytes, b_row = 0, j = 0;
@@ -378,11 +385,11 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
         if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
         const uint32_t fb = full0 + 8 * s;
         const uint32_t sa = base + s * kStageBytes, sb = sa + kUmmaABytes;
-        if (lane == 0) mbar_expect_tx(fb, a_bytes + b_bytes);
+        if (lane == 0) mbar_expect_tx(fb, (by_threads ? 0 : a_bytes) + b_bytes);
         __syncwarp();
         if (gather) {
           if (lane < n_issue) tma_gather4(sa + lane * 512, ta, fb, kb * kUmmaBK, gr0, gr1, gr2, gr3);
-        } else if (lane == 0) {
+        } else if (lane == 0 && !by_threads) {
           tma_load_2d(sa, ta, fb, kb * kUmmaBK, row);
         }
         if (lane == 0) {
@@ -418,6 +425,7 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
         for (int kb = 0; kb < k_blocks; ++kb, ++it) {
           const uint32_t s = it % kStages, n = it / kStages;
           if (!mbar_wait(full0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
+          if (MODE == 1) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // cp.async-written rows
           tc_fence_after();
           const uint32_t sa = base + s * kStageBytes, sb = sa + kUmmaABytes;
 #pragma unroll
@@ -429,6 +437,44 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
         if (ok) umma_commit(accf0 + 8 * buf);  // accumulator complete
       }
     }
+  } else if (MODE == 1 && warp >= 6) {
+    // ------------------------------------------------------------ A-row gather (mode 1, warps 6..9)
+    // Thread gt owns row gt of every A tile: for routed groups (use_gather == 2) it copies the
+    // row's 128 bytes of this k block from x with eight 16-byte cp.async into the swizzled
+    // position (16-byte chunk c of row r lives at chunk c ^ (r & 7)); otherwise it only arrives.
+    const int gt = threadIdx.x - kUmmaThreads;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      const TileCoord c = umma_decode<MODE>(p, tile_start, n_groups, t);
+      const GroupStatic g = p.gs[c.g];
+      const bool mine = !g.is_shared && p.use_gather == 2;
+      const bf16* src_row = nullptr;
+      if (mine) {
+        const int r = c.row0 + min(c.mt * kUmmaBM + gt, c.count - 1);     // rows past the group repeat its last row
+        src_row = p.x_rows_ptr + (size_t)__ldg(p.row_token + r) * p.d;
+      }
+      for (int kb = 0; kb < k_blocks_fixed; ++kb, ++it) {
+        const uint32_t s = it % kStages, n = it / kStages;
+        if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
+        const uint32_t fb = full0 + 8 * s;
+        if (mine) {
+          const uint32_t dst_row = base + s * kStageBytes + gt * 128;
+#pragma unroll
+          for (int ch = 0; ch < 8; ++ch) {
+            const int k = kb * kUmmaBK + ch * 8;
+            const uint32_t bytes = k < p.d ? 16u : 0u;                      // zero-fill past the end of the row
+            const bf16* src = src_row + (k < p.d ? k : 0);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                         ::"r"(dst_row + ((ch ^ (gt & 7)) << 4)), "l"(src), "r"(bytes) : "memory");
+          }
+          asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(fb) : "memory");
+        } else {
+          mbar_arrive(fb);
+        }
+      }
+    }
+    if (!ok) asm volatile("cp.async.wait_all;" ::: "memory");
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5)
     const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
@@ -697,6 +743,7 @@ inline UmmaArgs umma_base_args(const UmmaPlan* P, const GroupRows* gr, int32_t* 
   a.gs = P->buf.gs_dev; a.gr = gr; a.n_groups = P->n_groups; a.n_outer = s.n_outer; a.n_r = s.n_r;
   a.d = s.d; a.bn_s = P->bn_s; a.bn_r = P->bn_r; a.err = err_word;
   a.row_token = P->buf.row_token;
+  a.x_rows_ptr = nullptr;
   a.n_rp = s.n_rp; a.n_k = s.n_k; a.u = P->buf.u; a.b = P->buf.b;
   a.scores = P->buf.scores; a.keys = P->buf.keys; a.topk_idx = P->buf.topk_idx; a.topk_gate = P->buf.topk_gate;
   return a;
@@ -718,16 +765,18 @@ inline int umma_router_forward(UmmaPlan* P, int n_rows, const int32_t* outer_off
   return 1;
 }
 
-// Enqueues the gate/up and the down GEMM over all groups.  Requires umma_bind_x for this
+// Enqueues the gate/up and the down GEMM over all groups.  gather_mode: how routed groups get
+// their rows of x (0 permuted copy, 1 TMA gather4, 2 cp.async gather).  Requires umma_bind_x for this
 // forward.  Returns the number of kernels launched, or -1 (P->error).
-inline int umma_forward(UmmaPlan* P, const GroupRows* gr, bool gather_rows, int32_t* err_word, cudaStream_t st,
-                        cudaEvent_t mid) {
+inline int umma_forward(UmmaPlan* P, const GroupRows* gr, int gather_mode, const void* x_rows, int32_t* err_word,
+                        cudaStream_t st, cudaEvent_t mid) {
   const UmmaShape& s = P->shape;
   UmmaArgs a = umma_base_args(P, gr, err_word);
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
-  a.use_gather = gather_rows ? 1 : 0;
-  umma_grouped_kernel<1><<<P->n_sms, kUmmaThreads, kUmmaSmemBytes, st>>>(
-      P->x_rows, (gather_rows || !P->has_r) ? P->x_gather : P->x_perm, P->b1_s, P->b1_r, a);
+  a.use_gather = gather_mode;
+  a.x_rows_ptr = (const bf16*)x_rows;
+  umma_grouped_kernel<1><<<P->n_sms, kUmmaThreads + kUmmaGatherThreads, kUmmaSmemBytes, st>>>(
+      P->x_rows, (gather_mode != 0 || !P->has_r) ? P->x_gather : P->x_perm, P->b1_s, P->b1_r, a);
   if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
   umma_grouped_kernel<2><<<P->n_sms, kUmmaThreads, kUmmaSmemBytes, st>>>(P->a2_s, P->a2_r, P->b2_s, P->b2_r, a);
