@@ -439,34 +439,42 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
     }
   } else if (MODE == 1 && warp >= 6) {
     // ------------------------------------------------------------ A-row gather (mode 1, warps 6..9)
-    // Thread gt owns row gt of every A tile: for routed groups (use_gather == 2) it copies the
-    // row's 128 bytes of this k block from x with eight 16-byte cp.async into the swizzled
-    // position (16-byte chunk c of row r lives at chunk c ^ (r & 7)); otherwise it only arrives.
+    // For routed groups (use_gather == 2) the 128 threads copy the tile's 128 rows x 128 bytes of
+    // this k block from x: eight consecutive threads cover one row (coalesced 128-byte reads), 16
+    // rows per pass, 8 passes; 16-byte chunk c of row r goes to the swizzled chunk c ^ (r & 7).
+    // Otherwise the threads only arrive.
     const int gt = threadIdx.x - kUmmaThreads;
+    const int ch = gt & 7, r_sub = gt >> 3;
     uint32_t it = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
       const TileCoord c = umma_decode<MODE>(p, tile_start, n_groups, t);
       const GroupStatic g = p.gs[c.g];
       const bool mine = !g.is_shared && p.use_gather == 2;
-      const bf16* src_row = nullptr;
-      if (mine) {
-        const int r = c.row0 + min(c.mt * kUmmaBM + gt, c.count - 1);     // rows past the group repeat its last row
-        src_row = p.x_rows_ptr + (size_t)__ldg(p.row_token + r) * p.d;
+      const bf16* src_row[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        src_row[i] = nullptr;
+        if (mine) {                                   // rows past the group repeat its last row
+          const int r = c.row0 + min(c.mt * kUmmaBM + i * 16 + r_sub, c.count - 1);
+          src_row[i] = p.x_rows_ptr + (size_t)__ldg(p.row_token + r) * p.d;
+        }
       }
       for (int kb = 0; kb < k_blocks_fixed; ++kb, ++it) {
         const uint32_t s = it % kStages, n = it / kStages;
         if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
         const uint32_t fb = full0 + 8 * s;
         if (mine) {
-          const uint32_t dst_row = base + s * kStageBytes + gt * 128;
+          const int k = kb * kUmmaBK + ch * 8;
+          const uint32_t bytes = k < p.d ? 16u : 0u;                        // zero-fill past the end of the row
+          const int k_src = k < p.d ? k : 0;
+          const uint32_t sa = base + s * kStageBytes;
 #pragma unroll
-          for (int ch = 0; ch < 8; ++ch) {
-            const int k = kb * kUmmaBK + ch * 8;
-            const uint32_t bytes = k < p.d ? 16u : 0u;                      // zero-fill past the end of the row
-            const bf16* src = src_row + (k < p.d ? k : 0);
+          for (int i = 0; i < 8; ++i) {
+            const int r = i * 16 + r_sub;
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
-                         ::"r"(dst_row + ((ch ^ (gt & 7)) << 4)), "l"(src), "r"(bytes) : "memory");
+                         ::"r"(sa + r * 128 + ((ch ^ (r & 7)) << 4)), "l"(src_row[i] + k_src), "r"(bytes)
+                         : "memory");
           }
           asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(fb) : "memory");
         } else {
