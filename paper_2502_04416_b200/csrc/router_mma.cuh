@@ -266,15 +266,30 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
   __syncthreads();
   if (!is_last) return;
   __threadfence();
-  for (int r = warp; r < n_rows; r += kRskThreads / 32) {
-    float a = 0.0f, v = 0.0f;
-    if (lane < n_r) {
-      for (int s = 0; s < (int)gridDim.x; ++s) {           // ascending slices: deterministic
-        const float* ps = part + ((size_t)s * kRskMaxRows + r) * 64;
-        a += __ldcg(ps + lane);
-        v += __ldcg(ps + n_rp + lane);
-      }
+  // Sum the slices in ascending order (a fixed order: deterministic), all threads at once, eight
+  // loads in flight per thread; the totals go to shared memory (the unit tiles are free now).
+  float (*total)[kRmStride] = reinterpret_cast<float (*)[kRmStride]>(&unit[0][0][0]);   // [64][72]
+  const int n_slices = (int)gridDim.x;
+  for (int i = threadIdx.x; i < n_rows * 64; i += kRskThreads) {
+    const int r = i >> 6, n = i & 63;
+    if (n >= n2) continue;
+    const float* ps = part + (size_t)r * 64 + n;
+    float sum = 0.0f;
+    int s = 0;
+    for (; s + 8 <= n_slices; s += 8) {
+      float t[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) t[q] = __ldcg(ps + (size_t)(s + q) * kRskMaxRows * 64);
+#pragma unroll
+      for (int q = 0; q < 8; ++q) sum += t[q];
     }
+    for (; s < n_slices; ++s) sum += __ldcg(ps + (size_t)s * kRskMaxRows * 64);
+    total[r][n] = sum;
+  }
+  __syncthreads();
+  for (int r = warp; r < n_rows; r += kRskThreads / 32) {
+    const float a = lane < n_r ? total[r][lane] : 0.0f;
+    const float v = lane < n_r ? total[r][n_rp + lane] : 0.0f;
     const int go = row_group[r];
     gate_row(lane, n_r, n_k, a, v, u + go * n_r, b + go * n_r, go * n_r, scores + (size_t)r * n_r,
              keys + (size_t)r * n_r, topk_idx + (size_t)r * n_k, topk_gate + (size_t)r * n_k);
