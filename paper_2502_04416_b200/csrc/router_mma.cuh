@@ -202,7 +202,7 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
                      int fuse_permute, int n_groups, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
                      int32_t* __restrict__ row_token, int32_t* __restrict__ row_of, const GroupPlanOut po) {
   static_assert(kRskThreads == kPermChunk, "the fused permutation is written for one 256-row chunk");
-  __shared__ float unit[8][16][kRmStride];       // [unit = half*m_tiles + m-tile][row in tile][n]
+  __shared__ __align__(16) float unit[8][16][kRmStride];       // [unit = half*m_tiles + m-tile][row in tile][n]
   __shared__ int row_group[kRskMaxRows];
   __shared__ int is_last;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -253,12 +253,10 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
   __syncthreads();
   // slice partial = first half + second half
   float* mine = part + (size_t)blockIdx.x * kRskMaxRows * 64;
-  for (int i = threadIdx.x; i < m_tiles * 16 * 64; i += kRskThreads) {
-    const int r = i >> 6, n = i & 63;
-    if (n < n2 && r < n_rows) {
-      const int mt = r >> 4, rr = r & 15;
-      mine[r * 64 + n] = unit[mt][rr][n] + unit[m_tiles + mt][rr][n];
-    }
+  for (int i = threadIdx.x; i < n_rows * n2; i += kRskThreads) {
+    const int r = i / n2, n = i - r * n2;
+    const int mt = r >> 4, rr = r & 15;
+    mine[r * 64 + n] = unit[mt][rr][n] + unit[m_tiles + mt][rr][n];
   }
   __threadfence();
   __syncthreads();
@@ -266,25 +264,29 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
   __syncthreads();
   if (!is_last) return;
   __threadfence();
-  // Sum the slices in ascending order (a fixed order: deterministic), all threads at once, eight
-  // loads in flight per thread; the totals go to shared memory (the unit tiles are free now).
+  // Sum the slices in ascending order (a fixed order: deterministic), all threads at once, sixteen
+  // 16-byte loads in flight per thread; the totals go to shared memory (the unit tiles are free now).
   float (*total)[kRmStride] = reinterpret_cast<float (*)[kRmStride]>(&unit[0][0][0]);   // [64][72]
   const int n_slices = (int)gridDim.x;
-  for (int i = threadIdx.x; i < n_rows * 64; i += kRskThreads) {
-    const int r = i >> 6, n = i & 63;
-    if (n >= n2) continue;
-    const float* ps = part + (size_t)r * 64 + n;
-    float sum = 0.0f;
+  const int n4 = n2 >> 2;                          // n2 is a multiple of 8: whole float4 groups
+  constexpr size_t kSliceStride4 = (size_t)kRskMaxRows * 64 / 4;
+  for (int i = threadIdx.x; i < n_rows * n4; i += kRskThreads) {
+    const int r = i / n4, n = (i - r * n4) * 4;
+    const float4* ps = reinterpret_cast<const float4*>(part + (size_t)r * 64 + n);
+    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
     int s = 0;
-    for (; s + 8 <= n_slices; s += 8) {
-      float t[8];
+    for (; s + 16 <= n_slices; s += 16) {
+      float4 t[16];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) t[q] = __ldcg(ps + (size_t)(s + q) * kRskMaxRows * 64);
+      for (int q = 0; q < 16; ++q) t[q] = __ldcg(ps + (size_t)(s + q) * kSliceStride4);
 #pragma unroll
-      for (int q = 0; q < 8; ++q) sum += t[q];
+      for (int q = 0; q < 16; ++q) { sum.x += t[q].x; sum.y += t[q].y; sum.z += t[q].z; sum.w += t[q].w; }
     }
-    for (; s < n_slices; ++s) sum += __ldcg(ps + (size_t)s * kRskMaxRows * 64);
-    total[r][n] = sum;
+    for (; s < n_slices; ++s) {
+      const float4 t = __ldcg(ps + (size_t)s * kSliceStride4);
+      sum.x += t.x; sum.y += t.y; sum.z += t.z; sum.w += t.w;
+    }
+    *reinterpret_cast<float4*>(&total[r][n]) = sum;
   }
   __syncthreads();
   for (int r = warp; r < n_rows; r += kRskThreads / 32) {
