@@ -413,6 +413,23 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   mark(4);
   const int per_thread = sizeof(T) == 2 ? 16 : 8;
   const int threads = d / per_thread < 256 ? ((d / per_thread + 31) / 32 * 32) : 256;
+  bool fast_combine = false;
+  if constexpr (sizeof(T) == 2) {
+    const int th = (d / 16 + 31) / 32 * 32;
+    if (!L->hier && d % 16 == 0 && th <= 1024 && n_k <= 4 && n_tok > 64) {
+      fast_combine = true;
+      const int sms = L->umma.n_sms > 0 ? L->umma.n_sms : 148;
+      const int grid = std::min(n_tok, sms * std::max(1, 1024 / th) * 2);
+      const bf16* ys = L->cfg.n_shared > 0 ? (const bf16*)L->y_s : nullptr;
+      if (n_k <= 1)
+        combine_plain_bf16_kernel<1><<<grid, th, 0, st>>>(ys, (const bf16*)L->y_r, L->topk_gate, L->row_of, n_tok, n_k, d, (bf16*)out);
+      else if (n_k == 2)
+        combine_plain_bf16_kernel<2><<<grid, th, 0, st>>>(ys, (const bf16*)L->y_r, L->topk_gate, L->row_of, n_tok, n_k, d, (bf16*)out);
+      else
+        combine_plain_bf16_kernel<4><<<grid, th, 0, st>>>(ys, (const bf16*)L->y_r, L->topk_gate, L->row_of, n_tok, n_k, d, (bf16*)out);
+    }
+  }
+  if (!fast_combine)
   combine_kernel<T><<<n_tok, threads, 0, st>>>(
       L->cfg.n_shared > 0 ? (const T*)L->y_s : nullptr, (const T*)L->y_r, L->topk_idx, L->topk_gate,
       L->row_of, L->hier ? L->outer_row_of : nullptr, L->hier ? L->outer_w : nullptr,

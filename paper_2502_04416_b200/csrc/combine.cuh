@@ -138,4 +138,69 @@ combine_kernel(const T* __restrict__ y_s, const T* __restrict__ y_r,
   }
 }
 
+// The same sum for a plain (one-level) bf16 layer with d % 16 == 0 and n_k <= NK, written for
+// bandwidth: a block strides over tokens with one thread per 16 columns (one pass over the
+// row whatever d is), all 1 + n_k row loads of a token are issued before any arithmetic, and
+// the next token's routing words are fetched while the current rows are in flight.  The
+// arithmetic and its order are those of combine_kernel, so both give the same bits.
+__device__ __forceinline__ void ld256_stream(const bf16* p, uint32_t (&w)[8]) {
+  asm("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+      : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+      : "l"(p));
+}
+
+template <int NK>
+__global__ void __launch_bounds__(1024)
+combine_plain_bf16_kernel(const bf16* __restrict__ y_s, const bf16* __restrict__ y_r,
+                          const float* __restrict__ topk_gate, const int32_t* __restrict__ row_of,
+                          int n_tok, int n_k, int d, bf16* __restrict__ out) {
+  const int c = threadIdx.x * 16;
+  if (c >= d) return;
+  int t = blockIdx.x;
+  if (t >= n_tok) return;
+  int rows[NK], rows_next[NK];
+  float g[NK], g_next[NK];
+#pragma unroll
+  for (int j = 0; j < NK; ++j) {
+    rows[j] = j < n_k ? __ldg(row_of + (size_t)t * n_k + j) : 0;
+    g[j] = j < n_k ? __ldg(topk_gate + (size_t)t * n_k + j) : 0.0f;
+  }
+  while (true) {
+    uint32_t ws[8], wr[NK][8];
+    if (y_s) ld256_stream(y_s + (size_t)t * d + c, ws);
+#pragma unroll
+    for (int j = 0; j < NK; ++j)
+      if (j < n_k) ld256_stream(y_r + (size_t)rows[j] * d + c, wr[j]);
+    const int t_next = t + gridDim.x;
+    if (t_next < n_tok) {
+#pragma unroll
+      for (int j = 0; j < NK; ++j) {
+        rows_next[j] = j < n_k ? __ldg(row_of + (size_t)t_next * n_k + j) : 0;
+        g_next[j] = j < n_k ? __ldg(topk_gate + (size_t)t_next * n_k + j) : 0.0f;
+      }
+    }
+    float inner[16];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      inner[2 * q] = y_s ? __uint_as_float(ws[q] << 16) : 0.0f;
+      inner[2 * q + 1] = y_s ? __uint_as_float(ws[q] & 0xffff0000u) : 0.0f;
+    }
+#pragma unroll
+    for (int j = 0; j < NK; ++j) {
+      if (j < n_k) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          inner[2 * q] = fmaf(g[j], __uint_as_float(wr[j][q] << 16), inner[2 * q]);
+          inner[2 * q + 1] = fmaf(g[j], __uint_as_float(wr[j][q] & 0xffff0000u), inner[2 * q + 1]);
+        }
+      }
+    }
+    store16(out + (size_t)t * d + c, inner);      // outer weight 1: fmaf(1, inner, 0) == inner
+    if (t_next >= n_tok) break;
+    t = t_next;
+#pragma unroll
+    for (int j = 0; j < NK; ++j) { rows[j] = rows_next[j]; g[j] = g_next[j]; }
+  }
+}
+
 }  // namespace cmoe
