@@ -240,6 +240,8 @@ def run_gpu(args):
     # ---- device-resident throughput.  Large batches: direct launches with per-stage events for
     # the roofline.  Small batches are launch-bound, so the forward (same C-ABI call, same
     # kernels) is captured once into a CUDA graph and replayed; stage events are off there.
+    if args.chain == "off":
+        layer.set_launch_chaining(False)
     use_graph = args.graph == "on" or (args.graph == "auto" and T <= 512)
     sampler = ClockSampler(local)
     sampler.start()
@@ -423,6 +425,8 @@ def main():
     ap.add_argument("--cpu-sample-tokens", type=int, default=256)
     ap.add_argument("--graph", choices=["auto", "on", "off"], default="auto",
                     help="replay the forward from a CUDA graph (auto: batches of at most 512 tokens)")
+    ap.add_argument("--chain", choices=["on", "off"], default="on",
+                    help="programmatic dependent launches between the kernels of a forward (library default: on)")
     ap.add_argument("--forward-only", action="store_true",
                     help="run only the timed forward passes (for profiler captures)")
     args = ap.parse_args()

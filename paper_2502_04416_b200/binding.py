@@ -19,7 +19,8 @@ STAGE_NAMES = ["route", "permute", "gemm1_swiglu", "gemm2_down", "combine"]
 
 EXPORTS = [
     "cmoe_layer_create", "cmoe_hier_create", "cmoe_ffn_forward", "cmoe_layer_set_gate_params",
-    "cmoe_layer_get_gate_params", "cmoe_layer_update_bias", "cmoe_layer_set_gemm_path", "cmoe_layer_dims", "cmoe_get_routing", "cmoe_layer_status",
+    "cmoe_layer_get_gate_params", "cmoe_layer_update_bias", "cmoe_layer_set_gemm_path", "cmoe_layer_set_launch_chaining",
+    "cmoe_layer_dims", "cmoe_get_routing", "cmoe_layer_status",
     "cmoe_layer_launch_count", "cmoe_layer_enable_stage_timing", "cmoe_layer_stage_times",
     "cmoe_layer_destroy", "cmoe_token_permute_scratch_bytes",
     "cmoe_token_permute", "cmoe_token_permute_static", "cmoe_status_string", "cmoe_last_error",
@@ -57,6 +58,7 @@ def load() -> C.CDLL:
     lib.cmoe_ffn_forward.argtypes = [vp, vp, i32, vp, vp]
     lib.cmoe_layer_set_gate_params.argtypes = [vp, vp, vp, vp]
     lib.cmoe_layer_set_gemm_path.argtypes = [vp, i32]
+    lib.cmoe_layer_set_launch_chaining.argtypes = [vp, i32]
     lib.cmoe_layer_get_gate_params.argtypes = [vp, vp, vp, vp]
     lib.cmoe_layer_update_bias.argtypes = [vp, C.c_float, vp, vp, vp]
     lib.cmoe_layer_dims.argtypes = [vp] + [C.POINTER(i32)] * 4
@@ -191,6 +193,9 @@ class Layer:
 
     def set_gemm_path(self, path: int) -> None:
         _check(load().cmoe_layer_set_gemm_path(self._h, path), "cmoe_layer_set_gemm_path")
+
+    def set_launch_chaining(self, on: bool) -> None:
+        _check(load().cmoe_layer_set_launch_chaining(self._h, 1 if on else 0), "cmoe_layer_set_launch_chaining")
 
     def dims(self) -> Dict[str, int]:
         v = [C.c_int32() for _ in range(4)]

@@ -71,6 +71,7 @@ struct cmoe_layer {
   int device = 0;
   size_t esz = 2;
   int gemm_path = 0;
+  bool chain_launches = true;
   bool umma_ok = false;
 
   // packed weights
@@ -307,6 +308,10 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   cudaEvent_t* ev = L->ev_ring ? &L->ev[(size_t)(L->ev_count % L->ev_ring) * (CMOE_N_STAGES + 1)] : nullptr;
   auto mark = [&](int i) { if (ev) cudaEventRecord(ev[i], st); };
   mark(0);
+  // Plain bf16 layers on the tensor path chain their kernels by programmatic dependent launch
+  // (every kernel after the router may become resident early and waits on the device for its
+  // predecessor); per-stage events, the hierarchical prologue and CTA pairs use ordinary launches.
+  const bool dep = use_umma && !L->hier && !ev && L->gemm_path != 3 && L->chain_launches;
 
   if (L->hier) {
     if constexpr (std::is_same<T, bf16>::value) {
@@ -365,7 +370,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
     mark(1);
     if (!perm_fused)
       launches += launch_token_permute(L->topk_idx, R, n_k, G, L->counts, L->offsets, L->row_token,
-                                       L->row_of, L->perm_scratch, st, po);
+                                       L->row_of, L->perm_scratch, st, po, dep);
   } else {
     mark(1);
     plan_groups_kernel<<<1, 256, 0, st>>>(L->n_outer, n_r, n_tok, L->hier ? L->outer_off : nullptr,
@@ -386,9 +391,9 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   if (use_umma) {
     // CTA pairs (cta_group::2, 256-row tiles) on request: measured equal to single-CTA tiles on
     // even groups and slower on ragged ones (an odd m-tile count idles half a pair)
-    const int n = decode ? decode_forward(&L->umma, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
+    const int n = decode ? decode_forward(&L->umma, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr, dep)
                 : pairs  ? umma2_forward(&L->umma, &L->pair, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
-                         : umma_forward(&L->umma, L->gr, gather_mode, xo, L->err_word, st, ev ? ev[3] : nullptr);
+                         : umma_forward(&L->umma, L->gr, gather_mode, xo, L->err_word, st, ev ? ev[3] : nullptr, dep);
     if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     launches += n;
   } else {
@@ -422,18 +427,19 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
       const int grid = std::min(n_tok, sms * std::max(1, 1024 / th) * 2);
       const bf16* ys = L->cfg.n_shared > 0 ? (const bf16*)L->y_s : nullptr;
       if (n_k <= 1)
-        combine_plain_bf16_kernel<1><<<grid, th, 0, st>>>(ys, (const bf16*)L->y_r, L->topk_gate, L->row_of, n_tok, n_k, d, (bf16*)out);
+        launch_kernel(dep, combine_plain_bf16_kernel<1>, dim3(grid), dim3(th), 0, st, ys, (const bf16*)L->y_r, L->topk_gate, L->row_of, n_tok, n_k, d, (bf16*)out);
       else if (n_k == 2)
-        combine_plain_bf16_kernel<2><<<grid, th, 0, st>>>(ys, (const bf16*)L->y_r, L->topk_gate, L->row_of, n_tok, n_k, d, (bf16*)out);
+        launch_kernel(dep, combine_plain_bf16_kernel<2>, dim3(grid), dim3(th), 0, st, ys, (const bf16*)L->y_r, L->topk_gate, L->row_of, n_tok, n_k, d, (bf16*)out);
       else
-        combine_plain_bf16_kernel<4><<<grid, th, 0, st>>>(ys, (const bf16*)L->y_r, L->topk_gate, L->row_of, n_tok, n_k, d, (bf16*)out);
+        launch_kernel(dep, combine_plain_bf16_kernel<4>, dim3(grid), dim3(th), 0, st, ys, (const bf16*)L->y_r, L->topk_gate, L->row_of, n_tok, n_k, d, (bf16*)out);
     }
   }
   if (!fast_combine)
-  combine_kernel<T><<<n_tok, threads, 0, st>>>(
-      L->cfg.n_shared > 0 ? (const T*)L->y_s : nullptr, (const T*)L->y_r, L->topk_idx, L->topk_gate,
-      L->row_of, L->hier ? L->outer_row_of : nullptr, L->hier ? L->outer_w : nullptr,
-      L->hier ? L->outer_k : 1, n_k, d, out);
+  launch_kernel(dep, combine_kernel<T>, dim3(n_tok), dim3(threads), 0, st,
+                L->cfg.n_shared > 0 ? (const T*)L->y_s : nullptr, (const T*)L->y_r, (const int32_t*)L->topk_idx,
+                (const float*)L->topk_gate, (const int32_t*)L->row_of,
+                (const int32_t*)(L->hier ? L->outer_row_of : nullptr), (const float*)(L->hier ? L->outer_w : nullptr),
+                L->hier ? L->outer_k : 1, n_k, d, out);
   ++launches;
   mark(5);
   if (ev) ++L->ev_count;
@@ -646,6 +652,12 @@ int cmoe_layer_set_gemm_path(cmoe_layer* L, int32_t path) {
   if (path >= 2 && !L->umma_ok)
     return arg_fail(CMOE_ERR_INVALID_ARG, "tensor-core path not available for this layer");
   L->gemm_path = path;
+  return CMOE_OK;
+}
+
+int cmoe_layer_set_launch_chaining(cmoe_layer* L, int32_t on) {
+  if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "null layer");
+  L->chain_launches = on != 0;
   return CMOE_OK;
 }
 

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 namespace cmoe {
 
 constexpr int kMaxRouted = 32;   // N_r per (outer) layer: one lane per routed expert
@@ -13,6 +15,27 @@ constexpr int kMaxTopK = 8;      // N_k
 constexpr int kMaxOuter = 32;    // experts of a hierarchical layer's top level
 
 typedef __nv_bfloat16 bf16;
+
+// Programmatic dependent launch: a kernel launched as a dependent may become resident while
+// its predecessor in the stream is still running; grid_dep_wait() returns once that
+// predecessor has completed and its writes are visible, so nothing it produces may be read
+// (and nothing it reads may be written) before the call.  grid_dep_trigger() lets this grid's
+// own dependent become resident as soon as every block has executed it.  Both are no-ops in
+// a kernel that was launched the ordinary way.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KP, typename... A>
+inline cudaError_t launch_kernel(bool dependent, void (*kernel)(KP...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t st, A&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at;
+  at.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &at; cfg.numAttrs = dependent ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<A>(args)...);
+}
 
 __device__ __forceinline__ float to_float(float v) { return v; }
 __device__ __forceinline__ float to_float(bf16 v) { return __bfloat162float(v); }

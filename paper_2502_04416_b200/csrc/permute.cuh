@@ -116,6 +116,8 @@ __global__ void __launch_bounds__(kPermChunk)
 permute_single_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k, int n_groups,
                       int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
                       int32_t* __restrict__ row_token, int32_t* __restrict__ row_of, const GroupPlanOut po) {
+  grid_dep_wait();
+  grid_dep_trigger();
   extern __shared__ int32_t sm[];
   int32_t* hist = sm;                              // [n_groups]
   int32_t* offs = hist + n_groups;                 // [n_groups + 1]
@@ -133,6 +135,8 @@ permute_single_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k,
 __global__ void __launch_bounds__(kPermChunk)
 permute_count_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k, int n_groups,
                      int32_t* __restrict__ chunk_cnt /*[n_chunks][n_groups]*/) {
+  grid_dep_wait();
+  grid_dep_trigger();
   extern __shared__ int32_t sm[];
   const int row = blockIdx.x * kPermChunk + threadIdx.x;
   chunk_histogram(topk_idx, n_rows, n_k, n_groups, row, sm);
@@ -145,6 +149,8 @@ permute_count_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k, 
 __global__ void __launch_bounds__(1024)
 permute_scan_kernel(int32_t* chunk_cnt, int n_chunks, int n_groups,
                     int32_t* __restrict__ counts, int32_t* __restrict__ offsets, const GroupPlanOut po) {
+  grid_dep_wait();
+  grid_dep_trigger();
   __shared__ int32_t sums[1024];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   for (int g = warp; g < n_groups; g += n_warps) {
@@ -172,6 +178,8 @@ __global__ void __launch_bounds__(kPermChunk)
 permute_scatter_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k, int n_groups,
                        const int32_t* __restrict__ chunk_cnt, const int32_t* __restrict__ offsets,
                        int32_t* __restrict__ row_token, int32_t* __restrict__ row_of) {
+  grid_dep_wait();
+  grid_dep_trigger();
   extern __shared__ int32_t sm[];
   int32_t* base = sm;                      // [n_groups]
   int32_t* warp_cnt = base + n_groups;     // [8][n_groups]
@@ -192,19 +200,20 @@ inline int64_t permute_scratch_bytes(int n_rows, int n_groups) {
 inline int launch_token_permute(const int32_t* topk_idx, int n_rows, int n_k, int n_groups,
                                 int32_t* counts, int32_t* offsets, int32_t* row_token,
                                 int32_t* row_of, int32_t* scratch, cudaStream_t stream,
-                                const GroupPlanOut po = GroupPlanOut()) {
+                                const GroupPlanOut po = GroupPlanOut(), bool dep = false) {
   if (n_rows <= kPermChunk) {
     const size_t smem = (size_t)(n_groups * 2 + 1 + kPermChunk + 8 * n_groups) * sizeof(int32_t);
-    permute_single_kernel<<<1, kPermChunk, smem, stream>>>(topk_idx, n_rows, n_k, n_groups, counts,
-                                                           offsets, row_token, row_of, po);
+    launch_kernel(dep, permute_single_kernel, dim3(1), dim3(kPermChunk), smem, stream, topk_idx, n_rows, n_k,
+                  n_groups, counts, offsets, row_token, row_of, po);
     return 1;
   }
   const int n_chunks = (n_rows + kPermChunk - 1) / kPermChunk;
-  permute_count_kernel<<<n_chunks, kPermChunk, n_groups * sizeof(int32_t), stream>>>(
-      topk_idx, n_rows, n_k, n_groups, scratch);
-  permute_scan_kernel<<<1, 1024, 0, stream>>>(scratch, n_chunks, n_groups, counts, offsets, po);
-  permute_scatter_kernel<<<n_chunks, kPermChunk, 9 * n_groups * sizeof(int32_t), stream>>>(
-      topk_idx, n_rows, n_k, n_groups, scratch, offsets, row_token, row_of);
+  launch_kernel(dep, permute_count_kernel, dim3(n_chunks), dim3(kPermChunk), n_groups * sizeof(int32_t), stream,
+                topk_idx, n_rows, n_k, n_groups, scratch);
+  launch_kernel(dep, permute_scan_kernel, dim3(1), dim3(1024), 0, stream, scratch, n_chunks, n_groups, counts,
+                offsets, po);
+  launch_kernel(dep, permute_scatter_kernel, dim3(n_chunks), dim3(kPermChunk), 9 * n_groups * sizeof(int32_t), stream,
+                topk_idx, n_rows, n_k, n_groups, scratch, offsets, row_token, row_of);
   return 3;
 }
 

@@ -30,7 +30,7 @@ stream_kernel(const __grid_constant__ CUtensorMap tm, int box_rows, int n_kb, in
     for (int t = blockIdx.x; t < n_tiles; t += gridDim.x)
       for (int kb = 0; kb < n_kb; ++kb, ++it) {
         const uint32_t s = it % stages, n = it / stages;
-        while (!mbar_try_wait(empty0 + 8 * s, (n & 1) ^ 1)) {}
+        for (long long spin = 0; !mbar_try_wait(empty0 + 8 * s, (n & 1) ^ 1); ++spin) if (spin > (1ll << 28)) return;
         mbar_expect_tx(full0 + 8 * s, box_rows * 128);
         tma_load_2d(base + s * stage_bytes, &tm, full0 + 8 * s, kb * 64, t * box_rows);
       }
@@ -40,7 +40,7 @@ stream_kernel(const __grid_constant__ CUtensorMap tm, int box_rows, int n_kb, in
     for (int t = blockIdx.x; t < n_tiles; t += gridDim.x)
       for (int kb = 0; kb < n_kb; ++kb, ++it) {
         const uint32_t s = it % stages, n = it / stages;
-        while (!mbar_try_wait(full0 + 8 * s, n & 1)) {}
+        for (long long spin = 0; !mbar_try_wait(full0 + 8 * s, n & 1); ++spin) if (spin > (1ll << 28)) return;
         acc += *reinterpret_cast<volatile unsigned*>(smem_raw + (base - raw) + s * stage_bytes);
         mbar_arrive(empty0 + 8 * s);
       }
@@ -60,7 +60,7 @@ int main() {
   unsigned long long* sink; cudaMalloc(&sink, 8);
   cudaFuncSetAttribute(stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
   cudaEvent_t e0, e1; cudaEventCreate(&e0); cudaEventCreate(&e1);
-  const int cols_list[] = {4096, 1376};
+  const int cols_list[] = {4096, 1376, 64};   // 64: every box is one contiguous 128 B x box_rows chunk
   for (int cols : cols_list)
   for (int promo = 0; promo < 2; ++promo)
   for (int box_rows : {64, 128, 256})

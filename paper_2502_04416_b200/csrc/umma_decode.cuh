@@ -62,6 +62,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_constant__ CUtensorMap tm_w_r,
                    const __grid_constant__ CUtensorMap tm_x_s, const __grid_constant__ CUtensorMap tm_x_r,
                    const DecodeArgs p) {
+  grid_dep_wait();
+  grid_dep_trigger();
   constexpr int kStages = DecodeCfg<MODE>::kStages;
   constexpr int kWBytes = DecodeCfg<MODE>::kWBytes;
   constexpr int kStageBytes = kWBytes + kDecXBytes;
@@ -307,17 +309,18 @@ inline bool decode_bind_x(UmmaPlan* P, DecodePlan* D, const void* x_rows, int n_
 // Both decode GEMMs; requires umma_bind_x and decode_bind_x for this forward and at most
 // kDecMaxRows outer rows.  Returns launches or -1.
 inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int32_t* err_word, cudaStream_t st,
-                          cudaEvent_t mid) {
+                          cudaEvent_t mid, bool dep = false) {
   const UmmaShape& s = P->shape;
   DecodeArgs a{};
   a.gs = P->buf.gs_dev; a.gr = gr; a.n_groups = P->n_groups; a.n_outer = s.n_outer; a.n_r = s.n_r;
   a.d = s.d; a.row_token = P->buf.row_token; a.err = err_word;
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
-  umma_decode_kernel<4><<<P->n_sms, kUmmaThreads, decode_smem_bytes<4>(), st>>>(D->w_gu, D->w_gu, D->x_rows64,
-                                                                             D->x_rows64, a);
+  launch_kernel(dep, umma_decode_kernel<4>, dim3(P->n_sms), dim3(kUmmaThreads), decode_smem_bytes<4>(), st, D->w_gu,
+                D->w_gu, D->x_rows64, D->x_rows64, a);
   if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
-  umma_decode_kernel<5><<<P->n_sms, kUmmaThreads, decode_smem_bytes<5>(), st>>>(D->wd_s, D->wd_r, D->h_s, D->h_r, a);
+  launch_kernel(dep, umma_decode_kernel<5>, dim3(P->n_sms), dim3(kUmmaThreads), decode_smem_bytes<5>(), st, D->wd_s,
+                D->wd_r, D->h_s, D->h_r, a);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
     snprintf(P->error, sizeof(P->error), "decode GEMM launch: %s", cudaGetErrorString(e));

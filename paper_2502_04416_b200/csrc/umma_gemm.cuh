@@ -292,6 +292,8 @@ __global__ void __launch_bounds__(MODE == 1 ? kUmmaThreads + kUmmaGatherThreads 
 umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_constant__ CUtensorMap tm_a_r,
                     const __grid_constant__ CUtensorMap tm_b_s, const __grid_constant__ CUtensorMap tm_b_r,
                     const UmmaArgs p) {
+  grid_dep_wait();
+  grid_dep_trigger();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -777,17 +779,18 @@ inline int umma_router_forward(UmmaPlan* P, int n_rows, const int32_t* outer_off
 // their rows of x (0 permuted copy, 1 TMA gather4, 2 cp.async gather).  Requires umma_bind_x for this
 // forward.  Returns the number of kernels launched, or -1 (P->error).
 inline int umma_forward(UmmaPlan* P, const GroupRows* gr, int gather_mode, const void* x_rows, int32_t* err_word,
-                        cudaStream_t st, cudaEvent_t mid) {
+                        cudaStream_t st, cudaEvent_t mid, bool dep = false) {
   const UmmaShape& s = P->shape;
   UmmaArgs a = umma_base_args(P, gr, err_word);
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
   a.use_gather = gather_mode;
   a.x_rows_ptr = (const bf16*)x_rows;
-  umma_grouped_kernel<1><<<P->n_sms, kUmmaThreads + kUmmaGatherThreads, kUmmaSmemBytes, st>>>(
-      P->x_rows, (gather_mode != 0 || !P->has_r) ? P->x_gather : P->x_perm, P->b1_s, P->b1_r, a);
+  launch_kernel(dep, umma_grouped_kernel<1>, dim3(P->n_sms), dim3(kUmmaThreads + kUmmaGatherThreads), kUmmaSmemBytes,
+                st, P->x_rows, (gather_mode != 0 || !P->has_r) ? P->x_gather : P->x_perm, P->b1_s, P->b1_r, a);
   if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
-  umma_grouped_kernel<2><<<P->n_sms, kUmmaThreads, kUmmaSmemBytes, st>>>(P->a2_s, P->a2_r, P->b2_s, P->b2_r, a);
+  launch_kernel(dep, umma_grouped_kernel<2>, dim3(P->n_sms), dim3(kUmmaThreads), kUmmaSmemBytes, st, P->a2_s,
+                P->a2_r, P->b2_s, P->b2_r, a);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
     snprintf(P->error, sizeof(P->error), "tensor-core GEMM launch: %s", cudaGetErrorString(e));

@@ -132,6 +132,47 @@ def test_call_contract():
     layer.destroy()
 
 
+def test_launch_chaining_is_bit_identical():
+    """Programmatic dependent launches change when kernels become resident, never what they compute:
+    outputs and routing with chaining on and off agree bit for bit, directly and under graph replay."""
+    import torch
+    inp = _inputs("c2_llama2_7b", d_model=256, tokens=(1400,), m=160)
+    lay = inp.layers[0]
+    layer = parity.gpu_layer(lay, 1400)
+    x = parity.to_device(inp.x, "bf16")
+    for t in (1, 16, 64, 65, 300, 700, 1400):          # decode, mid-size and tcgen05 routers
+        layer.set_launch_chaining(False)
+        ref = layer.forward(x[:t]).clone()
+        ref_routing = layer.routing(t, lay.shape.n_routed)
+        layer.set_launch_chaining(True)
+        for _ in range(3):
+            got = layer.forward(x[:t]).clone()
+            torch.cuda.synchronize()
+            assert layer.status() == 0
+            assert torch.equal(got.view(torch.int16), ref.view(torch.int16)), t
+        now = layer.routing(t, lay.shape.n_routed)
+        for k in ("topk_idx", "counts", "offsets", "row_token", "row_of"):
+            np.testing.assert_array_equal(now[k], ref_routing[k])
+        parity.check_plain_layer(layer, lay, inp.x[:t])
+    out = torch.empty_like(x[:64])
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        layer.forward(x[:64], out)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    ref = out.clone()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        layer.forward(x[:64], out)
+    for _ in range(5):
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), ref.view(torch.int16))
+    layer.destroy()
+
+
 @pytest.mark.parametrize("n_rows,n_k,n_groups", [(1, 2, 6), (255, 2, 6), (256, 4, 28), (257, 4, 28),
                                                  (5000, 2, 56), (16384, 4, 14), (3000, 8, 1000),
                                                  (700, 1, 3), (40, 0, 5)])
