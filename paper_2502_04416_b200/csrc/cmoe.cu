@@ -105,6 +105,8 @@ struct cmoe_layer {
   Umma2Plan pair;
   float* rsk_part = nullptr;    // split-K router partial sums [slices][64 rows][64]
   int32_t* rsk_ticket = nullptr;
+  float* dec_part = nullptr;    // decode GEMMs: K-slice partial sums, tickets per (tile, epilogue warp)
+  int32_t* dec_ticket = nullptr;
   float *share = nullptr, *target = nullptr;   // utilisation of the last step / bias-update targets
 
   cudaStream_t last_stream = nullptr;
@@ -206,6 +208,12 @@ void carve_workspace(cmoe_layer* L, char* base) {
   L->share = a.take<float>(G ? G : 1);
   L->target = a.take<float>(G ? G : 1);
   L->rsk_part = a.take<float>((size_t)kRskMaxSlices * kRskMaxRows * 64);
+  if (esz == 2) {
+    const size_t t1 = (size_t)L->n_outer * ((L->shared_width() + 127) / 128 + nr * ((L->m + 127) / 128));
+    const size_t t2 = (size_t)L->n_groups_total() * ((d + 127) / 128);
+    L->dec_ticket = a.take<int32_t>(4 * (t1 > t2 ? t1 : t2));
+    L->dec_part = a.take<float>((size_t)kDecMaxSlots * kDecSlotFloats);
+  }
   L->x_perm = a.take<char>(P * d * esz);
   L->h_s = a.take<char>(R * L->shared_width() * esz);
   L->h_r = a.take<char>(P * L->m * esz);
@@ -269,6 +277,7 @@ int finish_layer(cmoe_layer* L, cudaStream_t st) {
     if (rc == CMOE_ERR_CUDA) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     L->umma_ok = (rc == CMOE_OK);
     if (L->umma_ok && !decode_plan_create(&L->umma, &L->decode)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
+    L->decode.part = L->dec_part; L->decode.ticket = L->dec_ticket;
     if (L->umma_ok && !umma2_plan_create(&L->umma, &L->pair)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   }
   CU_TRY(cudaStreamSynchronize(st));

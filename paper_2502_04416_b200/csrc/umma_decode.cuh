@@ -14,8 +14,14 @@
 //       group's epilogue simply stores the columns of the tokens that selected it.
 //   MODE 5, down:     D[c, t] = Wd[c] . H_t ,  epilogue Y[t, c] = D
 //       tile = 128 output channels of one group.
-// Tiles are dealt to the persistent CTAs in snake order (left to right, then right to
-// left), which balances the long shared-expert tiles against the short routed ones.
+// With few active experts there are fewer tiles than SMs and one SM cannot pull more than
+// ~100 GB/s through TMA, so a tile's K range is split into Z slices when that brings the
+// unit count closer to the SM count (Z = k blocks of the tile / (all k blocks / CTAs),
+// rounded down, per group).  A slice leaves its fp32 partial accumulators in a scratch slot;
+// each epilogue warp takes a ticket for its 32 weight rows of the tile, and the warp that
+// takes the last one adds the Z partials in slice order (a fixed order: deterministic) and
+// finishes the tile.  Units are dealt to the persistent CTAs in snake order (left to right,
+// then right to left), which balances long shared-expert units against short routed ones.
 // Same warp roles, bounded waits and teardown as the token-major kernels.
 #pragma once
 
@@ -27,7 +33,14 @@ constexpr int kDecMaxRows = 64;            // rows per group this path takes
 constexpr int kDecXBytes = kDecMaxRows * kUmmaBK * 2;      // 8 KB token tile
 constexpr int kDecTmemCols = 256;          // two buffers of (64 gate + 64 up) columns
 
-constexpr int kDecInvOff = 256 + ((kUmmaMaxGroups + 1) * 4 + 15) / 16 * 16;   // per-warp token tables
+constexpr int kDecMaxSplit = 8;            // K slices per tile at most
+constexpr int kDecMinSliceKb = 6;          // k blocks per slice at least
+constexpr int kDecMaxSlots = 256;          // scratch slots for slice partials (>= CTAs)
+constexpr int kDecSlotFloats = 128 * 2 * kDecMaxRows;      // 128 weight rows x (gate, up) x 64 tokens
+
+// per group: first unit / tile / slot, split, k blocks per tile
+struct DecGroup { int32_t unit0, tile0, slot0; int16_t z, kb; };
+constexpr int kDecInvOff = 256 + ((kUmmaMaxGroups + 1) * (int)sizeof(DecGroup) + 15) / 16 * 16;   // per-warp token tables
 
 template <int MODE> struct DecodeCfg;
 template <> struct DecodeCfg<4> { static constexpr int kWBytes = 2 * 128 * kUmmaBK * 2, kStages = 5; };
@@ -48,6 +61,8 @@ struct DecodeArgs {
   int ld_out_s, ld_out_r;
   const int32_t* row_token;
   int32_t* err;
+  float* part;           // [kDecMaxSlots][kDecSlotFloats] slice partials
+  int32_t* ticket;       // [tiles][4 epilogue warps], zero between launches
 };
 
 // Tile handled by CTA `cta` in its `round`-th turn: even rounds run left to right, odd
@@ -77,7 +92,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   const uint32_t full0 = bars, empty0 = bars + 64, accf0 = bars + 128, acce0 = bars + 144;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_gen + 160);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
-  int32_t* tile_start = reinterpret_cast<int32_t*>(bars_gen + 256);
+  DecGroup* grp = reinterpret_cast<DecGroup*>(bars_gen + 256);       // [n_groups + 1]
   int32_t* inv_tables = reinterpret_cast<int32_t*>(bars_gen + kDecInvOff);     // [4 warps][64]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -93,30 +108,56 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
     tmem_alloc(smem_u32(tmem_slot), kDecTmemCols);
     tmem_relinquish();
   }
+  // per group: tile count (in .tile0 for now) and k blocks per tile
   for (int g = threadIdx.x; g < p.n_groups; g += blockDim.x) {
     const int span = MODE == 4 ? p.gs[g].width : (p.gs[g].width > 0 ? p.d : 0);
-    tile_start[g + 1] = p.gr[g].count > 0 ? (span + 127) / 128 : 0;
+    grp[g].tile0 = p.gr[g].count > 0 ? (span + 127) / 128 : 0;
+    grp[g].kb = (int16_t)(((MODE == 4 ? p.d : p.gs[g].width) + kUmmaBK - 1) / kUmmaBK);
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    int run = 0;
-    tile_start[0] = 0;
-    for (int g = 0; g < p.n_groups; ++g) { run += tile_start[g + 1]; tile_start[g + 1] = run; }
+    long long all_kb = 0;
+    for (int g = 0; g < p.n_groups; ++g) all_kb += (long long)grp[g].tile0 * grp[g].kb;
+    int per_cta = (int)((all_kb + gridDim.x - 1) / gridDim.x);       // k blocks a CTA streams if all share evenly
+    if (per_cta < kDecMinSliceKb) per_cta = kDecMinSliceKb;
+    int units = 0, tiles = 0, slots = 0;
+    for (int g = 0; g < p.n_groups; ++g) {
+      const int n_t = grp[g].tile0, kb = grp[g].kb;
+      int z = kb / per_cta;
+      z = z < 1 ? 1 : (z > kDecMaxSplit ? kDecMaxSplit : z);
+      if (z > 1 && slots + n_t * z > kDecMaxSlots) z = 1;
+      grp[g].unit0 = units; grp[g].tile0 = tiles; grp[g].z = (int16_t)z; grp[g].slot0 = slots;
+      units += n_t * z; tiles += n_t; slots += z > 1 ? n_t * z : 0;
+    }
+    grp[p.n_groups].unit0 = units; grp[p.n_groups].tile0 = tiles; grp[p.n_groups].z = 1; grp[p.n_groups].kb = 0;
+    grp[p.n_groups].slot0 = slots;
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int total_tiles = tile_start[p.n_groups];
+  const int total_units = grp[p.n_groups].unit0;
   const int cta = blockIdx.x, n_ctas = gridDim.x;
 
-  auto find_group = [&](int t) {
+  // unit -> group, tile within the group, K slice
+  struct Unit { int gi, nt, z, n_z, kb0, kb1; };
+  auto find_unit = [&](int uid) {
     int lo = 0, hi = p.n_groups;
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
-      if (tile_start[mid] <= t) lo = mid; else hi = mid;
+      if (grp[mid].unit0 <= uid) lo = mid; else hi = mid;
     }
-    return lo;
+    Unit u;
+    u.gi = lo; u.n_z = grp[lo].z;
+    const int local = uid - grp[lo].unit0, k_blocks = grp[lo].kb;
+    if (u.n_z == 1) {
+      u.nt = local; u.z = 0; u.kb0 = 0; u.kb1 = k_blocks;
+    } else {
+      u.nt = local / u.n_z; u.z = local - u.nt * u.n_z;
+      u.kb0 = u.z * k_blocks / u.n_z;
+      u.kb1 = (u.z + 1) * k_blocks / u.n_z;
+    }
+    return u;
   };
 
   if (warp == 0) {
@@ -124,17 +165,17 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
     uint32_t it = 0;
     bool ok = true;
     for (int round = 0; ok; ++round) {
-      const int t = snake_tile(round, cta, n_ctas, total_tiles);
+      const int t = snake_tile(round, cta, n_ctas, total_units);
       if (t < 0) break;
-      const int gi = find_group(t), nt = t - tile_start[gi];
+      const Unit un = find_unit(t);
+      const int gi = un.gi, nt = un.nt;
       const GroupStatic g = p.gs[gi];
       // mode 4: token rows of the group's outer expert; mode 5: the group's own H rows
       const GroupRows r = MODE == 4 ? p.gr[g.outer] : p.gr[gi];
       const CUtensorMap* tw = g.is_shared ? &tm_w_s : &tm_w_r;
       const CUtensorMap* tx = g.is_shared ? &tm_x_s : &tm_x_r;
-      const int k_blocks = ((MODE == 4 ? p.d : g.width) + kUmmaBK - 1) / kUmmaBK;
       const int j = g.is_shared ? 0 : (gi - p.n_outer) - g.outer * p.n_r;
-      for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+      for (int kb = un.kb0; kb < un.kb1; ++kb, ++it) {
         const uint32_t s = it % kStages, n = it / kStages;
         if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
         const uint32_t fb = full0 + 8 * s;
@@ -156,25 +197,25 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
       uint32_t it = 0;
       bool ok = true;
       for (int round = 0; ok; ++round) {
-        const int t = snake_tile(round, cta, n_ctas, total_tiles);
+        const int t = snake_tile(round, cta, n_ctas, total_units);
         if (t < 0) break;
-        const int gi = find_group(t);
+        const Unit un = find_unit(t);
+        const int gi = un.gi;
         const GroupStatic g = p.gs[gi];
-        const int k_blocks = ((MODE == 4 ? p.d : g.width) + kUmmaBK - 1) / kUmmaBK;
         const int n_mma = ((MODE == 4 ? p.gr[g.outer].count : p.gr[gi].count) + 15) & ~15;   // columns, rounded to 16
         const uint32_t idesc = umma_idesc(n_mma);
         const uint32_t buf = round & 1, use = round >> 1;
         if (!mbar_wait(acce0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.err, kErrWaitAccEmpty)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * 128;
-        for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+        for (int kb = un.kb0; kb < un.kb1; ++kb, ++it) {
           const uint32_t s = it % kStages, n = it / kStages;
           if (!mbar_wait(full0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sw = base + s * kStageBytes, sx = sw + kWBytes;
 #pragma unroll
           for (int k = 0; k < kUmmaBK / 16; ++k) {
-            const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
+            const uint32_t acc = (kb != un.kb0 || k != 0) ? 1u : 0u;
             umma_bf16(d_tmem, umma_smem_desc(sw + k * 32), umma_smem_desc(sx + k * 32), idesc, acc);
             if (MODE == 4)
               umma_bf16(d_tmem + 64, umma_smem_desc(sw + 128 * kUmmaBK * 2 + k * 32),
@@ -190,9 +231,10 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
     const int quad = warp & 3;
     bool ok = true;
     for (int round = 0; ok; ++round) {
-      const int t = snake_tile(round, cta, n_ctas, total_tiles);
+      const int t = snake_tile(round, cta, n_ctas, total_units);
       if (t < 0) break;
-      const int gi = find_group(t), nt = t - tile_start[gi];
+      const Unit un = find_unit(t);
+      const int gi = un.gi, nt = un.nt;
       const GroupStatic g = p.gs[gi];
       const GroupRows r = p.gr[gi];
       const uint32_t buf = round & 1, use = round >> 1;
@@ -217,27 +259,68 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         for (int c = lane; c < r.count; c += 32) inv[__ldg(p.row_token + r.row0 + c) - rs.row0] = c;
         __syncwarp();
       }
-      for (int c0 = 0; c0 < n_cols; c0 += 16) {
-        float a[16], b[16];
-        tmem_ld16(taddr + c0, a);
-        if (MODE == 4) tmem_ld16(taddr + 64 + c0, b);
-        tmem_ld_wait();
-        if (wr < span) {
+      const bool row_live = wr < span;
+      auto finish = [&](int c, float a, float b) {       // accumulator column c of this thread's weight row
+        if (row_live && c < n_cols) {
+          const int pos = lookup ? inv[c] : c;
+          if (pos >= 0) {
+            const float v = MODE == 4 ? a / (1.0f + __expf(-a)) * b : a;
+            dst[(size_t)pos * ld] = __float2bfloat16_rn(v);
+          }
+        }
+      };
+      if (un.n_z == 1) {
+        for (int c0 = 0; c0 < n_cols; c0 += 16) {
+          float a[16], b[16];
+          tmem_ld16(taddr + c0, a);
+          if (MODE == 4) tmem_ld16(taddr + 64 + c0, b);
+          tmem_ld_wait();
+#pragma unroll
+          for (int q = 0; q < 16; ++q) finish(c0 + q, a[q], MODE == 4 ? b[q] : 0.0f);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acce0 + 8 * buf);
+      } else {
+        // K slice of a split tile: park the partial sums, take this warp's ticket for the tile
+        constexpr int kPlanes = MODE == 4 ? 2 : 1;
+        const int slot0 = grp[gi].slot0 + nt * un.n_z;
+        float* mine = p.part + (size_t)(slot0 + un.z) * kDecSlotFloats + quad * 32 + lane;
+        for (int c0 = 0; c0 < n_cols; c0 += 16) {
+          float a[16], b[16];
+          tmem_ld16(taddr + c0, a);
+          if (MODE == 4) tmem_ld16(taddr + 64 + c0, b);
+          tmem_ld_wait();
 #pragma unroll
           for (int q = 0; q < 16; ++q) {
             if (c0 + q < n_cols) {
-              const int pos = lookup ? inv[c0 + q] : c0 + q;
-              if (pos >= 0) {
-                const float v = MODE == 4 ? a[q] / (1.0f + __expf(-a[q])) * b[q] : a[q];
-                dst[(size_t)pos * ld] = __float2bfloat16_rn(v);
-              }
+              __stcg(mine + (size_t)((c0 + q) * kPlanes) * 128, a[q]);
+              if (MODE == 4) __stcg(mine + (size_t)((c0 + q) * kPlanes + 1) * 128, b[q]);
             }
           }
         }
+        tc_fence_before();
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acce0 + 8 * buf);
+        int32_t* tk = p.ticket + (size_t)(grp[gi].tile0 + nt) * 4 + quad;
+        int last = 0;
+        if (lane == 0) last = atomicAdd(tk, 1) == un.n_z - 1;
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+          __threadfence();
+          const float* all = p.part + (size_t)slot0 * kDecSlotFloats + quad * 32 + lane;
+          for (int c = 0; c < n_cols; ++c) {
+            float a = 0.0f, b = 0.0f;
+            for (int z = 0; z < un.n_z; ++z) {             // ascending slice order
+              a += __ldcg(all + (size_t)z * kDecSlotFloats + (size_t)(c * kPlanes) * 128);
+              if (MODE == 4) b += __ldcg(all + (size_t)z * kDecSlotFloats + (size_t)(c * kPlanes + 1) * 128);
+            }
+            finish(c, a, b);
+          }
+          if (lane == 0) *tk = 0;                          // ready for the next launch
+        }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(acce0 + 8 * buf);
     }
   }
   tc_fence_before();
@@ -251,6 +334,8 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
 // ----------------------------------------------------------------------------- host
 struct DecodePlan {
   bool built = false;
+  float* part = nullptr;            // kDecMaxSlots slots of slice partials (caller-owned workspace)
+  int32_t* ticket = nullptr;        // zeroed once; the kernels leave it zero
   CUtensorMap w_gu;                 // stacked gate/up rows, box 64 k x 128 rows x 2 planes
   CUtensorMap wd_s, wd_r;           // W_down blocks, 128-channel boxes
   CUtensorMap x_rows64;             // x, 64-row boxes (bound per forward for a plain layer)
@@ -314,6 +399,7 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int32
   DecodeArgs a{};
   a.gs = P->buf.gs_dev; a.gr = gr; a.n_groups = P->n_groups; a.n_outer = s.n_outer; a.n_r = s.n_r;
   a.d = s.d; a.row_token = P->buf.row_token; a.err = err_word;
+  a.part = D->part; a.ticket = D->ticket;
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
   launch_kernel(dep, umma_decode_kernel<4>, dim3(P->n_sms), dim3(kUmmaThreads), decode_smem_bytes<4>(), st, D->w_gu,
                 D->w_gu, D->x_rows64, D->x_rows64, a);

@@ -42,6 +42,7 @@ SMALL = [
     ("c3_llama3_8b", 256, None, (33, 517)),
     ("c5_skew_13b", 320, None, (129, 700)),
     ("c2_llama2_7b", 512, 200, (1000,)),       # m = 200: neither a multiple of 16 nor of 64
+    ("c2_llama2_7b", 1024, 768, (1, 7, 64)),   # decode GEMMs with K split 2-4 ways per tile
 ]
 
 
