@@ -208,12 +208,6 @@ void carve_workspace(cmoe_layer* L, char* base) {
   L->share = a.take<float>(G ? G : 1);
   L->target = a.take<float>(G ? G : 1);
   L->rsk_part = a.take<float>((size_t)kRskMaxSlices * kRskMaxRows * 64);
-  if (esz == 2) {
-    const size_t t1 = (size_t)L->n_outer * ((L->shared_width() + 127) / 128 + nr * ((L->m + 127) / 128));
-    const size_t t2 = (size_t)L->n_groups_total() * ((d + 127) / 128);
-    L->dec_ticket = a.take<int32_t>(4 * (t1 > t2 ? t1 : t2));
-    L->dec_part = a.take<float>((size_t)kDecMaxSlots * kDecSlotFloats);
-  }
   L->x_perm = a.take<char>(P * d * esz);
   L->h_s = a.take<char>(R * L->shared_width() * esz);
   L->h_r = a.take<char>(P * L->m * esz);
@@ -229,6 +223,12 @@ void carve_workspace(cmoe_layer* L, char* base) {
     L->outer_row_of = a.take<int32_t>(R);
     L->outer_scratch = a.take<int32_t>(permute_scratch_bytes((int)T, L->n_outer) / 4);
     L->xo = a.take<char>(R * d * esz);
+  }
+  if (esz == 2) {
+    const size_t t1 = (size_t)L->n_outer * ((L->shared_width() + 127) / 128 + nr * ((L->m + 127) / 128));
+    const size_t t2 = (size_t)L->n_groups_total() * ((d + 127) / 128);
+    L->dec_ticket = a.take<int32_t>(4 * (t1 > t2 ? t1 : t2));
+    L->dec_part = a.take<float>((size_t)kDecMaxSlots * kDecSlotFloats);
   }
   L->ws_bytes = align_up(a.used + 256, 256);
 }
@@ -400,7 +400,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   if (use_umma) {
     // CTA pairs (cta_group::2, 256-row tiles) on request: measured equal to single-CTA tiles on
     // even groups and slower on ragged ones (an odd m-tile count idles half a pair)
-    const int n = decode ? decode_forward(&L->umma, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr, dep)
+    const int n = decode ? decode_forward(&L->umma, &L->decode, L->gr, R, L->err_word, st, ev ? ev[3] : nullptr, dep)
                 : pairs  ? umma2_forward(&L->umma, &L->pair, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
                          : umma_forward(&L->umma, L->gr, gather_mode, xo, L->err_word, st, ev ? ev[3] : nullptr, dep);
     if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);

@@ -72,7 +72,9 @@ __device__ __forceinline__ int snake_tile(int round, int cta, int n_ctas, int to
   return t < total ? t : -1;
 }
 
-template <int MODE>
+// SPLIT = false is the plain form (one unit per tile, no scratch); the host picks SPLIT = true
+// only when even the largest possible set of active experts leaves tiles to split.
+template <int MODE, bool SPLIT>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_constant__ CUtensorMap tm_w_r,
                    const __grid_constant__ CUtensorMap tm_x_s, const __grid_constant__ CUtensorMap tm_x_r,
@@ -92,7 +94,8 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   const uint32_t full0 = bars, empty0 = bars + 64, accf0 = bars + 128, acce0 = bars + 144;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_gen + 160);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
-  DecGroup* grp = reinterpret_cast<DecGroup*>(bars_gen + 256);       // [n_groups + 1]
+  DecGroup* grp = reinterpret_cast<DecGroup*>(bars_gen + 256);       // SPLIT: [n_groups + 1]
+  int32_t* tile_start = reinterpret_cast<int32_t*>(bars_gen + 256);  // !SPLIT: [n_groups + 1], same bytes
   int32_t* inv_tables = reinterpret_cast<int32_t*>(bars_gen + kDecInvOff);     // [4 warps][64]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -108,41 +111,80 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
     tmem_alloc(smem_u32(tmem_slot), kDecTmemCols);
     tmem_relinquish();
   }
-  // per group: tile count (in .tile0 for now) and k blocks per tile
-  for (int g = threadIdx.x; g < p.n_groups; g += blockDim.x) {
-    const int span = MODE == 4 ? p.gs[g].width : (p.gs[g].width > 0 ? p.d : 0);
-    grp[g].tile0 = p.gr[g].count > 0 ? (span + 127) / 128 : 0;
-    grp[g].kb = (int16_t)(((MODE == 4 ? p.d : p.gs[g].width) + kUmmaBK - 1) / kUmmaBK);
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    long long all_kb = 0;
-    for (int g = 0; g < p.n_groups; ++g) all_kb += (long long)grp[g].tile0 * grp[g].kb;
-    int per_cta = (int)((all_kb + gridDim.x - 1) / gridDim.x);       // k blocks a CTA streams if all share evenly
-    if (per_cta < kDecMinSliceKb) per_cta = kDecMinSliceKb;
-    int units = 0, tiles = 0, slots = 0;
-    for (int g = 0; g < p.n_groups; ++g) {
-      const int n_t = grp[g].tile0, kb = grp[g].kb;
-      int z = kb / per_cta;
-      z = z < 1 ? 1 : (z > kDecMaxSplit ? kDecMaxSplit : z);
-      if (z > 1 && slots + n_t * z > kDecMaxSlots) z = 1;
-      grp[g].unit0 = units; grp[g].tile0 = tiles; grp[g].z = (int16_t)z; grp[g].slot0 = slots;
-      units += n_t * z; tiles += n_t; slots += z > 1 ? n_t * z : 0;
+  if constexpr (!SPLIT) {
+    for (int g = threadIdx.x; g < p.n_groups; g += blockDim.x) {
+      const int span = MODE == 4 ? p.gs[g].width : (p.gs[g].width > 0 ? p.d : 0);
+      tile_start[g + 1] = p.gr[g].count > 0 ? (span + 127) / 128 : 0;
     }
-    grp[p.n_groups].unit0 = units; grp[p.n_groups].tile0 = tiles; grp[p.n_groups].z = 1; grp[p.n_groups].kb = 0;
-    grp[p.n_groups].slot0 = slots;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int run = 0;
+      tile_start[0] = 0;
+      for (int g = 0; g < p.n_groups; ++g) { run += tile_start[g + 1]; tile_start[g + 1] = run; }
+    }
+  } else {
+    // per group: tile count (in .tile0 for now) and k blocks per tile
+    for (int g = threadIdx.x; g < p.n_groups; g += blockDim.x) {
+      const int span = MODE == 4 ? p.gs[g].width : (p.gs[g].width > 0 ? p.d : 0);
+      grp[g].tile0 = p.gr[g].count > 0 ? (span + 127) / 128 : 0;
+      grp[g].kb = (int16_t)(((MODE == 4 ? p.d : p.gs[g].width) + kUmmaBK - 1) / kUmmaBK);
+    }
+    __syncthreads();
+    if (warp == 0) {                 // unit / tile / slot prefix sums over the groups, 32 groups per step
+      int all_kb = 0;
+      for (int g = lane; g < p.n_groups; g += 32) all_kb += grp[g].tile0 * grp[g].kb;
+  #pragma unroll
+      for (int o = 16; o > 0; o >>= 1) all_kb += __shfl_xor_sync(0xffffffffu, all_kb, o);
+      int per_cta = (all_kb + (int)gridDim.x - 1) / (int)gridDim.x;    // k blocks a CTA streams if all share evenly
+      if (per_cta < kDecMinSliceKb) per_cta = kDecMinSliceKb;
+      // sum over split groups of tiles * z <= all_kb / per_cta <= CTAs, so the slots suffice for grids up to kDecMaxSlots
+      const bool may_split = (int)gridDim.x <= kDecMaxSlots;
+      int units = 0, tiles = 0, slots = 0;
+      for (int g0 = 0; g0 < p.n_groups; g0 += 32) {
+        const int g = g0 + lane;
+        const bool in = g < p.n_groups;
+        const int n_t = in ? grp[g].tile0 : 0;
+        int z = in ? grp[g].kb / per_cta : 1;
+        z = (z < 1 || !may_split) ? 1 : (z > kDecMaxSplit ? kDecMaxSplit : z);
+        const int u = n_t * z, sl = z > 1 ? u : 0;
+        int iu = u, it = n_t, is = sl;                       // inclusive scans
+  #pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int au = __shfl_up_sync(0xffffffffu, iu, o), at = __shfl_up_sync(0xffffffffu, it, o),
+                    as = __shfl_up_sync(0xffffffffu, is, o);
+          if (lane >= o) { iu += au; it += at; is += as; }
+        }
+        if (in) { grp[g].unit0 = units + iu - u; grp[g].tile0 = tiles + it - n_t; grp[g].slot0 = slots + is - sl; grp[g].z = (int16_t)z; }
+        units += __shfl_sync(0xffffffffu, iu, 31);
+        tiles += __shfl_sync(0xffffffffu, it, 31);
+        slots += __shfl_sync(0xffffffffu, is, 31);
+      }
+      if (lane == 0) {
+        grp[p.n_groups].unit0 = units; grp[p.n_groups].tile0 = tiles; grp[p.n_groups].slot0 = slots;
+        grp[p.n_groups].z = 1; grp[p.n_groups].kb = 0;
+      }
+    }
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int total_units = grp[p.n_groups].unit0;
+  const int total_units = SPLIT ? grp[p.n_groups].unit0 : tile_start[p.n_groups];
   const int cta = blockIdx.x, n_ctas = gridDim.x;
 
   // unit -> group, tile within the group, K slice
   struct Unit { int gi, nt, z, n_z, kb0, kb1; };
   auto find_unit = [&](int uid) {
     int lo = 0, hi = p.n_groups;
+    if constexpr (!SPLIT) {
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (tile_start[mid] <= uid) lo = mid; else hi = mid;
+      }
+      Unit u;
+      u.gi = lo; u.nt = uid - tile_start[lo]; u.z = 0; u.n_z = 1; u.kb0 = 0; u.kb1 = 0;   // kb1: see k_end
+      return u;
+    }
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
       if (grp[mid].unit0 <= uid) lo = mid; else hi = mid;
@@ -175,7 +217,8 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
       const CUtensorMap* tw = g.is_shared ? &tm_w_s : &tm_w_r;
       const CUtensorMap* tx = g.is_shared ? &tm_x_s : &tm_x_r;
       const int j = g.is_shared ? 0 : (gi - p.n_outer) - g.outer * p.n_r;
-      for (int kb = un.kb0; kb < un.kb1; ++kb, ++it) {
+      const int k_end = SPLIT ? un.kb1 : ((MODE == 4 ? p.d : g.width) + kUmmaBK - 1) / kUmmaBK;
+      for (int kb = un.kb0; kb < k_end; ++kb, ++it) {
         const uint32_t s = it % kStages, n = it / kStages;
         if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
         const uint32_t fb = full0 + 8 * s;
@@ -208,7 +251,8 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         if (!mbar_wait(acce0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.err, kErrWaitAccEmpty)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * 128;
-        for (int kb = un.kb0; kb < un.kb1; ++kb, ++it) {
+        const int k_end = SPLIT ? un.kb1 : ((MODE == 4 ? p.d : g.width) + kUmmaBK - 1) / kUmmaBK;
+        for (int kb = un.kb0; kb < k_end; ++kb, ++it) {
           const uint32_t s = it % kStages, n = it / kStages;
           if (!mbar_wait(full0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
           tc_fence_after();
@@ -269,7 +313,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
           }
         }
       };
-      if (un.n_z == 1) {
+      if (!SPLIT || un.n_z == 1) {
         for (int c0 = 0; c0 < n_cols; c0 += 16) {
           float a[16], b[16];
           tmem_ld16(taddr + c0, a);
@@ -281,7 +325,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(acce0 + 8 * buf);
-      } else {
+      } else if constexpr (SPLIT) {
         // K slice of a split tile: park the partial sums, take this warp's ticket for the tile
         constexpr int kPlanes = MODE == 4 ? 2 : 1;
         const int slot0 = grp[gi].slot0 + nt * un.n_z;
@@ -373,10 +417,16 @@ inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
   if (!ok) return false;
   if (!P->has_r) { D->wd_r = D->wd_s; D->h_r = D->h_s; }
   if (!P->has_s) { D->wd_s = D->wd_r; D->h_s = D->h_r; }
-  cudaError_t e = cudaFuncSetAttribute(umma_decode_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(umma_decode_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        decode_smem_bytes<4>());
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(umma_decode_kernel<5>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(umma_decode_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             decode_smem_bytes<4>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(umma_decode_kernel<5, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             decode_smem_bytes<5>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(umma_decode_kernel<5, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              decode_smem_bytes<5>());
   if (e != cudaSuccess) {
     snprintf(P->error, sizeof(P->error), "cudaFuncSetAttribute (decode): %s", cudaGetErrorString(e));
@@ -391,22 +441,37 @@ inline bool decode_bind_x(UmmaPlan* P, DecodePlan* D, const void* x_rows, int n_
   return umma_encode_rows(P, &D->x_rows64, x_rows, (size_t)n_rows, (size_t)P->shape.d, kDecMaxRows, "x (decode)");
 }
 
-// Both decode GEMMs; requires umma_bind_x and decode_bind_x for this forward and at most
-// kDecMaxRows outer rows.  Returns launches or -1.
-inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int32_t* err_word, cudaStream_t st,
-                          cudaEvent_t mid, bool dep = false) {
+// Both decode GEMMs; requires umma_bind_x and decode_bind_x for this forward and n_rows <=
+// kDecMaxRows outer rows.  The K-splitting form of a kernel is launched only when the device-side
+// rule would split some group even if the largest possible set of experts were active for
+// n_rows rows (fewer active experts only split more).  Returns launches or -1.
+inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n_rows, int32_t* err_word,
+                          cudaStream_t st, cudaEvent_t mid, bool dep = false) {
   const UmmaShape& s = P->shape;
+  const long long act_s = P->has_s ? (s.n_outer < n_rows ? s.n_outer : n_rows) : 0;
+  const long long all_r = (long long)s.n_outer * s.n_r, picks = (long long)n_rows * s.n_k;
+  const long long act_r = P->has_r ? (all_r < picks ? all_r : picks) : 0;
+  auto splits = [&](long long all_kb, int kb_max) {
+    long long per_cta = (all_kb + P->n_sms - 1) / P->n_sms;
+    if (per_cta < kDecMinSliceKb) per_cta = kDecMinSliceKb;
+    return D->part != nullptr && P->n_sms <= kDecMaxSlots && kb_max / per_cta >= 2;
+  };
+  const int kb_d = (s.d + kUmmaBK - 1) / kUmmaBK, kb_s = (s.shared_width + kUmmaBK - 1) / kUmmaBK,
+            kb_m = (s.m + kUmmaBK - 1) / kUmmaBK;
+  const bool split1 = splits((act_s * ((s.shared_width + 127) / 128) + act_r * ((s.m + 127) / 128)) * kb_d, kb_d);
+  const bool split2 = splits((long long)((s.d + 127) / 128) * (act_s * kb_s + act_r * kb_m),
+                             (act_s && kb_s > kb_m) || !act_r ? kb_s : kb_m);
   DecodeArgs a{};
   a.gs = P->buf.gs_dev; a.gr = gr; a.n_groups = P->n_groups; a.n_outer = s.n_outer; a.n_r = s.n_r;
   a.d = s.d; a.row_token = P->buf.row_token; a.err = err_word;
   a.part = D->part; a.ticket = D->ticket;
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
-  launch_kernel(dep, umma_decode_kernel<4>, dim3(P->n_sms), dim3(kUmmaThreads), decode_smem_bytes<4>(), st, D->w_gu,
-                D->w_gu, D->x_rows64, D->x_rows64, a);
+  launch_kernel(dep, split1 ? umma_decode_kernel<4, true> : umma_decode_kernel<4, false>, dim3(P->n_sms),
+                dim3(kUmmaThreads), decode_smem_bytes<4>(), st, D->w_gu, D->w_gu, D->x_rows64, D->x_rows64, a);
   if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
-  launch_kernel(dep, umma_decode_kernel<5>, dim3(P->n_sms), dim3(kUmmaThreads), decode_smem_bytes<5>(), st, D->wd_s,
-                D->wd_r, D->h_s, D->h_r, a);
+  launch_kernel(dep, split2 ? umma_decode_kernel<5, true> : umma_decode_kernel<5, false>, dim3(P->n_sms),
+                dim3(kUmmaThreads), decode_smem_bytes<5>(), st, D->wd_s, D->wd_r, D->h_s, D->h_r, a);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
     snprintf(P->error, sizeof(P->error), "decode GEMM launch: %s", cudaGetErrorString(e));
