@@ -105,7 +105,6 @@ struct cmoe_layer {
   Umma2Plan pair;
   float* rsk_part = nullptr;    // split-K router partial sums [slices][64 rows][64]
   int32_t* rsk_ticket = nullptr;
-  int32_t* g1_counter = nullptr;   // tile counter of the gate/up GEMM
   float* dec_part = nullptr;    // decode GEMMs: K-slice partial sums, tickets per (tile, epilogue warp)
   int32_t* dec_ticket = nullptr;
   float *share = nullptr, *target = nullptr;   // utilisation of the last step / bias-update targets
@@ -206,7 +205,6 @@ void carve_workspace(cmoe_layer* L, char* base) {
   L->gr = a.take<GroupRows>(L->n_groups_total());
   L->err_word = a.take<int32_t>(1);
   L->rsk_ticket = a.take<int32_t>(1);
-  L->g1_counter = a.take<int32_t>(1);
   L->share = a.take<float>(G ? G : 1);
   L->target = a.take<float>(G ? G : 1);
   L->rsk_part = a.take<float>((size_t)kRskMaxSlices * kRskMaxRows * 64);
@@ -280,7 +278,6 @@ int finish_layer(cmoe_layer* L, cudaStream_t st) {
     L->umma_ok = (rc == CMOE_OK);
     if (L->umma_ok && !decode_plan_create(&L->umma, &L->decode)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     L->decode.part = L->dec_part; L->decode.ticket = L->dec_ticket;
-    L->umma.tile_counter = L->g1_counter;
     if (L->umma_ok && !umma2_plan_create(&L->umma, &L->pair)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   }
   CU_TRY(cudaStreamSynchronize(st));
@@ -405,7 +402,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
     // even groups and slower on ragged ones (an odd m-tile count idles half a pair)
     const int n = decode ? decode_forward(&L->umma, &L->decode, L->gr, R, L->err_word, st, ev ? ev[3] : nullptr, dep)
                 : pairs  ? umma2_forward(&L->umma, &L->pair, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
-                         : umma_forward(&L->umma, L->gr, R, gather_mode, xo, L->err_word, st, ev ? ev[3] : nullptr, dep);
+                         : umma_forward(&L->umma, L->gr, gather_mode, xo, L->err_word, st, ev ? ev[3] : nullptr, dep);
     if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     launches += n;
   } else {

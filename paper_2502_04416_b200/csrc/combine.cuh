@@ -50,8 +50,8 @@ combine_kernel(const T* __restrict__ y_s, const T* __restrict__ y_r,
                const int32_t* __restrict__ topk_idx, const float* __restrict__ topk_gate,
                const int32_t* __restrict__ row_of, const int32_t* __restrict__ outer_row_of,
                const float* __restrict__ outer_w, int outer_k, int n_k, int d, T* __restrict__ out) {
-  grid_dep_trigger();
   grid_dep_wait();
+  grid_dep_trigger();
   (void)topk_idx;
   const int t = blockIdx.x;
   constexpr bool kWide = sizeof(T) == 2;
@@ -156,8 +156,8 @@ __global__ void __launch_bounds__(1024)
 combine_plain_bf16_kernel(const bf16* __restrict__ y_s, const bf16* __restrict__ y_r,
                           const float* __restrict__ topk_gate, const int32_t* __restrict__ row_of,
                           int n_tok, int n_k, int d, bf16* __restrict__ out) {
-  grid_dep_trigger();
   grid_dep_wait();
+  grid_dep_trigger();
   const int c = threadIdx.x * 16;
   if (c >= d) return;
   int t = blockIdx.x;

@@ -116,8 +116,8 @@ __global__ void __launch_bounds__(kPermChunk)
 permute_single_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k, int n_groups,
                       int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
                       int32_t* __restrict__ row_token, int32_t* __restrict__ row_of, const GroupPlanOut po) {
-  grid_dep_trigger();
   grid_dep_wait();
+  grid_dep_trigger();
   extern __shared__ int32_t sm[];
   int32_t* hist = sm;                              // [n_groups]
   int32_t* offs = hist + n_groups;                 // [n_groups + 1]
@@ -135,8 +135,8 @@ permute_single_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k,
 __global__ void __launch_bounds__(kPermChunk)
 permute_count_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k, int n_groups,
                      int32_t* __restrict__ chunk_cnt /*[n_chunks][n_groups]*/) {
-  grid_dep_trigger();
   grid_dep_wait();
+  grid_dep_trigger();
   extern __shared__ int32_t sm[];
   const int row = blockIdx.x * kPermChunk + threadIdx.x;
   chunk_histogram(topk_idx, n_rows, n_k, n_groups, row, sm);
@@ -149,8 +149,8 @@ permute_count_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k, 
 __global__ void __launch_bounds__(1024)
 permute_scan_kernel(int32_t* chunk_cnt, int n_chunks, int n_groups,
                     int32_t* __restrict__ counts, int32_t* __restrict__ offsets, const GroupPlanOut po) {
-  grid_dep_trigger();
   grid_dep_wait();
+  grid_dep_trigger();
   __shared__ int32_t sums[1024];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   for (int g = warp; g < n_groups; g += n_warps) {
@@ -178,8 +178,8 @@ __global__ void __launch_bounds__(kPermChunk)
 permute_scatter_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k, int n_groups,
                        const int32_t* __restrict__ chunk_cnt, const int32_t* __restrict__ offsets,
                        int32_t* __restrict__ row_token, int32_t* __restrict__ row_of) {
-  grid_dep_trigger();
   grid_dep_wait();
+  grid_dep_trigger();
   extern __shared__ int32_t sm[];
   int32_t* base = sm;                      // [n_groups]
   int32_t* warp_cnt = base + n_groups;     // [8][n_groups]

@@ -107,8 +107,8 @@ router_mma_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, int n
                   const int32_t* __restrict__ outer_off, int n_outer,
                   float* __restrict__ scores, float* __restrict__ keys,
                   int32_t* __restrict__ topk_idx, float* __restrict__ topk_gate) {
-  grid_dep_trigger();
   grid_dep_wait();
+  grid_dep_trigger();
   constexpr int ROWS = 16 * MT;
   __shared__ float part[WARPS][ROWS][kRmStride];
   __shared__ float fin[ROWS][kRmStride];
@@ -203,8 +203,8 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
                      int32_t* topk_idx, float* __restrict__ topk_gate,
                      int fuse_permute, int n_groups, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
                      int32_t* __restrict__ row_token, int32_t* __restrict__ row_of, const GroupPlanOut po) {
-  grid_dep_trigger();
   grid_dep_wait();
+  grid_dep_trigger();
   static_assert(kRskThreads == kPermChunk, "the fused permutation is written for one 256-row chunk");
   __shared__ __align__(16) float unit[8][16][kRmStride];       // [unit = half*m_tiles + m-tile][row in tile][n]
   __shared__ int row_group[kRskMaxRows];

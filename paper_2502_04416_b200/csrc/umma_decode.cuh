@@ -79,8 +79,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_constant__ CUtensorMap tm_w_r,
                    const __grid_constant__ CUtensorMap tm_x_s, const __grid_constant__ CUtensorMap tm_x_r,
                    const DecodeArgs p) {
-  grid_dep_trigger();
   grid_dep_wait();
+  grid_dep_trigger();
   constexpr int kStages = DecodeCfg<MODE>::kStages;
   constexpr int kWBytes = DecodeCfg<MODE>::kWBytes;
   constexpr int kStageBytes = kWBytes + kDecXBytes;

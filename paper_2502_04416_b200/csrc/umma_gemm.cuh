@@ -47,14 +47,11 @@ constexpr int kUmmaMaxGroups = 1088;
 constexpr int kUmmaThreads = 192;     // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
 constexpr int kUmmaGatherThreads = 128;   // mode 1 only: warps 6..9, one thread per A-tile row
 constexpr int kUmmaTmemCols = 512;    // two accumulator buffers of 256 columns
-constexpr int kUmmaRing = 4;          // mode 1: tiles announced ahead by the scheduling warp
-constexpr int kUmmaRingOff = 256 + ((kUmmaMaxGroups + 1) * 4 + 15) / 16 * 16;   // after barriers and tile_start
-constexpr int kUmmaSmemBytes = 1024 /*alignment slack*/ + kUmmaStages * kUmmaStageBytes + kUmmaRingOff +
-                               kUmmaRing * 32;
+constexpr int kUmmaSmemBytes = 1024 /*alignment slack*/ + kUmmaStages * kUmmaStageBytes +
+                               256 /*barriers*/ + (kUmmaMaxGroups + 1) * 4;
 constexpr long long kUmmaWaitCycles = 2000000000LL;   // ~1 s at SM clock
 
-enum { kErrWaitFull = 1, kErrWaitEmpty = 2, kErrWaitAccFull = 3, kErrWaitAccEmpty = 4, kErrWaitRingFull = 5,
-       kErrWaitRingEmpty = 6 };
+enum { kErrWaitFull = 1, kErrWaitEmpty = 2, kErrWaitAccFull = 3, kErrWaitAccEmpty = 4 };
 
 // ----------------------------------------------------------------------------- PTX
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -189,11 +186,6 @@ struct UmmaArgs {
   int use_gather;             // mode 1, routed A rows: 0 permuted copy by TMA, 1 TMA gather4 from x, 2 cp.async from x
   const bf16* x_rows_ptr;     // mode 1: the outer rows of x (source of the cp.async gather)
   int32_t* err;
-  // mode 1: tiles are handed out through a counter in global memory (zero at launch; mode 2
-  // clears it again).  The first n_static tiles, those of a plain layer's shared expert over
-  // rows [0, n_rows), need nothing that this forward's router or permutation produce.
-  int32_t* tile_counter;
-  int n_static;
   // mode 3 (router)
   const int32_t* outer_off;   // row ranges of the outer experts, or null (one range [0, n_rows))
   int n_rows, n_rp, n_k;      // n_rp: N_r rounded up to 8 (rows per block of the padded W^R)
@@ -300,10 +292,8 @@ __global__ void __launch_bounds__(MODE == 1 ? kUmmaThreads + kUmmaGatherThreads 
 umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_constant__ CUtensorMap tm_a_r,
                     const __grid_constant__ CUtensorMap tm_b_s, const __grid_constant__ CUtensorMap tm_b_r,
                     const UmmaArgs p) {
-  // Mode 1 starts on the tiles that do not depend on the kernels before it and waits for those
-  // kernels only when the scheduling warp reaches the first tile that does.
+  grid_dep_wait();
   grid_dep_trigger();
-  if (MODE != 1) grid_dep_wait();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -317,9 +307,6 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_gen + 160);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
   int32_t* tile_start = reinterpret_cast<int32_t*>(bars_gen + 256);
-  // mode 1 tile ring: ring_full[4] ring_empty[4] in the barrier block, TileCoord slots after tile_start
-  const uint32_t ringf0 = bars + 168, ringe0 = bars + 200;
-  volatile int32_t* ring = reinterpret_cast<volatile int32_t*>(bars_gen + kUmmaRingOff);   // [kUmmaRing][8]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_groups = MODE == 3 ? p.n_outer : p.n_groups;
@@ -329,8 +316,6 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
     const uint32_t full_count = MODE == 1 ? 1 + kUmmaGatherThreads : 1;
     for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, full_count); mbar_init(empty0 + 8 * s, 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 4); }
-    if (MODE == 1)           // a slot is free again once the MMA thread, 4 epilogue and 4 gather warps have read it
-      for (int r = 0; r < kUmmaRing; ++r) { mbar_init(ringf0 + 8 * r, 1); mbar_init(ringe0 + 8 * r, 9); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -339,101 +324,30 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
     tmem_alloc(smem_u32(tmem_slot), kUmmaTmemCols);
     tmem_relinquish();
   }
-  if (MODE != 1) {
-    // tiles of every group, then their exclusive prefix (mode 1: the scheduling warp does this
-    // itself once the kernels before it are complete)
-    for (int g = threadIdx.x; g < n_groups; g += blockDim.x) {
-      const int m_tiles = (umma_rows<MODE>(p, g).count + kUmmaBM - 1) / kUmmaBM;
-      tile_start[g + 1] = m_tiles * umma_n_tiles<MODE>(p, g);
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      int run = 0;
-      tile_start[0] = 0;
-      for (int g = 0; g < n_groups; ++g) { run += tile_start[g + 1]; tile_start[g + 1] = run; }
-      if (MODE == 2 && blockIdx.x == 0 && p.tile_counter) *p.tile_counter = 0;   // mode 1 of this forward is complete
-    }
+  // tiles of every group, then their exclusive prefix
+  for (int g = threadIdx.x; g < n_groups; g += blockDim.x) {
+    const int m_tiles = (umma_rows<MODE>(p, g).count + kUmmaBM - 1) / kUmmaBM;
+    tile_start[g + 1] = m_tiles * umma_n_tiles<MODE>(p, g);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int run = 0;
+    tile_start[0] = 0;
+    for (int g = 0; g < n_groups; ++g) { run += tile_start[g + 1]; tile_start[g + 1] = run; }
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int total_tiles = MODE == 1 ? 0 : tile_start[n_groups];
+  const int total_tiles = tile_start[n_groups];
   const int k_blocks_fixed = (p.d + kUmmaBK - 1) / kUmmaBK;      // modes 1 and 3: K = d
-
-  // Tile sequence of a role.  Modes 2 and 3: every role strides over the tile list on its own.
-  // Mode 1: warp 0 draws tile numbers from the global counter and announces each tile (or the
-  // end, g = -1) in a ring slot; the other roles read the slots in order.
-  uint32_t seq = 0;                     // tiles this role has taken
-  bool dep_done = MODE != 1;            // this thread has waited for the preceding kernels
-  auto schedule_next = [&](TileCoord& c) -> int {      // warp 0 only; 1 tile, 0 end, -1 wait timed out
-    if (MODE != 1) {
-      const int t = blockIdx.x + seq * gridDim.x;
-      ++seq;
-      if (t >= total_tiles) return 0;
-      c = umma_decode<MODE>(p, tile_start, n_groups, t);
-      return 1;
-    }
-    int t = 0;
-    if (lane == 0) t = atomicAdd(p.tile_counter, 1);
-    t = __shfl_sync(0xffffffffu, t, 0);
-    if (t < p.n_static) {
-      const int m_tiles = (p.n_rows + kUmmaBM - 1) / kUmmaBM;
-      c.g = 0; c.mt = t % m_tiles; c.nt = t / m_tiles; c.row0 = 0; c.count = p.n_rows;
-    } else {
-      if (!dep_done) {
-        grid_dep_wait();
-        dep_done = true;
-        for (int g = lane; g < n_groups; g += 32) {
-          const int m_tiles = (p.gr[g].count + kUmmaBM - 1) / kUmmaBM;
-          tile_start[g + 1] = m_tiles * umma_n_tiles<MODE>(p, g);
-        }
-        __syncwarp();
-        if (lane == 0) {
-          int run = 0;
-          tile_start[0] = 0;
-          for (int g = 0; g < n_groups; ++g) { run += tile_start[g + 1]; tile_start[g + 1] = run; }
-        }
-        __syncwarp();
-      }
-      if (t < tile_start[n_groups]) c = umma_decode<MODE>(p, tile_start, n_groups, t);
-      else c.g = -1;
-    }
-    const uint32_t slot = seq % kUmmaRing, n = seq / kUmmaRing;
-    ++seq;
-    if (!mbar_wait(ringe0 + 8 * slot, (n & 1) ^ 1, abort_flag, p.err, kErrWaitRingEmpty)) return -1;
-    if (lane == 0) {
-      volatile int32_t* r = ring + slot * 8;
-      r[0] = c.g; r[1] = c.mt; r[2] = c.nt; r[3] = c.row0; r[4] = c.count;
-      mbar_arrive(ringf0 + 8 * slot);
-    }
-    __syncwarp();
-    return c.g >= 0 ? 1 : 0;
-  };
-  auto follow_next = [&](TileCoord& c) -> int {        // the other roles; whole warps or the single MMA thread
-    if (MODE != 1) {
-      const int t = blockIdx.x + seq * gridDim.x;
-      ++seq;
-      if (t >= total_tiles) return 0;
-      c = umma_decode<MODE>(p, tile_start, n_groups, t);
-      return 1;
-    }
-    const uint32_t slot = seq % kUmmaRing, n = seq / kUmmaRing;
-    ++seq;
-    if (!mbar_wait(ringf0 + 8 * slot, n & 1, abort_flag, p.err, kErrWaitRingFull)) return -1;
-    volatile int32_t* r = ring + slot * 8;
-    c.g = r[0]; c.mt = r[1]; c.nt = r[2]; c.row0 = r[3]; c.count = r[4];
-    return c.g >= 0 ? 1 : 0;
-  };
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (whole warp)
     uint32_t it = 0;
     bool ok = true;
-    while (ok) {
-      TileCoord c;
-      const int got = schedule_next(c);
-      if (got <= 0) { ok = got == 0; break; }
+    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      const TileCoord c = umma_decode<MODE>(p, tile_start, n_groups, t);
       GroupStatic g;
       if (MODE != 3) g = p.gs[c.g]; else { g.is_shared = 1; g.outer = c.g; g.width = 0; g.w_row0 = 0; }
       const int row = c.row0 + c.mt * kUmmaBM;
@@ -454,10 +368,10 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
           a_bytes = n_issue * 512;
           const int last = c.row0 + c.count - 1;
           const int r = row + 4 * lane;
-          gr0 = __ldcg(p.row_token + min(r, last));
-          gr1 = __ldcg(p.row_token + min(r + 1, last));
-          gr2 = __ldcg(p.row_token + min(r + 2, last));
-          gr3 = __ldcg(p.row_token + min(r + 3, last));
+          gr0 = __ldg(p.row_token + min(r, last));
+          gr1 = __ldg(p.row_token + min(r + 1, last));
+          gr2 = __ldg(p.row_token + min(r + 2, last));
+          gr3 = __ldg(p.row_token + min(r + 3, last));
         }
       } else if (MODE == 2) {
         k_blocks = (g.width + kUmmaBK - 1) / kUmmaBK;
@@ -494,11 +408,8 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
     if (lane == 0) {
       uint32_t it = 0, tile_n = 0;
       bool ok = true;
-      for (; ok; ++tile_n) {
-        TileCoord c;
-        const int got = follow_next(c);
-        if (MODE == 1 && got >= 0) mbar_arrive(ringe0 + 8 * ((seq - 1) % kUmmaRing));
-        if (got <= 0) break;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_n) {
+        const TileCoord c = umma_decode<MODE>(p, tile_start, n_groups, t);
         int k_blocks, n_mma;
         if (MODE == 1) {
           const GroupStatic g = p.gs[c.g];
@@ -538,22 +449,17 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
     const int ch = gt & 7, r_sub = gt >> 3;
     uint32_t it = 0;
     bool ok = true;
-    while (ok) {
-      TileCoord c;
-      const int got = follow_next(c);
-      __syncwarp();
-      if (got >= 0 && lane == 0) mbar_arrive(ringe0 + 8 * ((seq - 1) % kUmmaRing));
-      if (got <= 0) break;
+    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      const TileCoord c = umma_decode<MODE>(p, tile_start, n_groups, t);
       const GroupStatic g = p.gs[c.g];
       const bool mine = !g.is_shared && p.use_gather == 2;
-      if (mine && !dep_done) { grid_dep_wait(); dep_done = true; }      // row_token comes from the permutation
       const bf16* src_row[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         src_row[i] = nullptr;
         if (mine) {                                   // rows past the group repeat its last row
           const int r = c.row0 + min(c.mt * kUmmaBM + i * 16 + r_sub, c.count - 1);
-          src_row[i] = p.x_rows_ptr + (size_t)__ldcg(p.row_token + r) * p.d;
+          src_row[i] = p.x_rows_ptr + (size_t)__ldg(p.row_token + r) * p.d;
         }
       }
       for (int kb = 0; kb < k_blocks_fixed; ++kb, ++it) {
@@ -584,14 +490,8 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
     const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
     uint32_t tile_n = 0;
     bool ok = true;
-    for (; ok; ++tile_n) {
-      TileCoord c;
-      const int got = follow_next(c);
-      if (MODE == 1) {
-        __syncwarp();
-        if (got >= 0 && lane == 0) mbar_arrive(ringe0 + 8 * ((seq - 1) % kUmmaRing));
-      }
-      if (got <= 0) break;
+    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_n) {
+      const TileCoord c = umma_decode<MODE>(p, tile_start, n_groups, t);
       const uint32_t buf = tile_n & 1, use = tile_n >> 1;
       if (!mbar_wait(accf0 + 8 * buf, use & 1, abort_flag, p.err, kErrWaitAccFull)) { ok = false; break; }
       tc_fence_after();
@@ -675,8 +575,6 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
       if (lane == 0) mbar_arrive(acce0 + 8 * buf);
     }
   }
-  // no CTA leaves before the kernels ahead of it are complete: the kernels behind it rely on that
-  if (MODE == 1) grid_dep_wait();
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -716,7 +614,6 @@ struct UmmaPlan {
   UmmaShape shape;
   UmmaBuffers buf;
   int bn_s = 128, bn_r = 128, n_sms = 0, n_groups = 0;
-  int32_t* tile_counter = nullptr;         // gate/up GEMM tile counter (caller's workspace, zeroed once)
   bool has_s = false, has_r = false;
   PFN_encodeTiled encode = nullptr;
   CUtensorMap x_rows, x_gather;            // x: 64 x 128 boxes for consecutive rows, 64 x 1 for gather4
@@ -881,14 +778,10 @@ inline int umma_router_forward(UmmaPlan* P, int n_rows, const int32_t* outer_off
 // Enqueues the gate/up and the down GEMM over all groups.  gather_mode: how routed groups get
 // their rows of x (0 permuted copy, 1 TMA gather4, 2 cp.async gather).  Requires umma_bind_x for this
 // forward.  Returns the number of kernels launched, or -1 (P->error).
-inline int umma_forward(UmmaPlan* P, const GroupRows* gr, int n_rows, int gather_mode, const void* x_rows,
-                        int32_t* err_word, cudaStream_t st, cudaEvent_t mid, bool dep = false) {
+inline int umma_forward(UmmaPlan* P, const GroupRows* gr, int gather_mode, const void* x_rows, int32_t* err_word,
+                        cudaStream_t st, cudaEvent_t mid, bool dep = false) {
   const UmmaShape& s = P->shape;
   UmmaArgs a = umma_base_args(P, gr, err_word);
-  // plain layer: the shared expert's tiles over rows [0, n_rows) are known before any routing
-  const bool plain = s.n_outer == 1 && P->buf.x_fixed == nullptr;
-  a.tile_counter = P->tile_counter; a.n_rows = n_rows;
-  a.n_static = (plain && P->has_s) ? ((n_rows + kUmmaBM - 1) / kUmmaBM) * ((s.shared_width + P->bn_s - 1) / P->bn_s) : 0;
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
   a.use_gather = gather_mode;
   a.x_rows_ptr = (const bf16*)x_rows;
