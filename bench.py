@@ -167,7 +167,7 @@ def prepare_inputs(name: str):
 # DRAM bytes (read + write) per forward of the dominant kernels from the ncu captures summarised
 # under profiles/ (taken on this kernel version); None where no capture exists.
 NCU_TRAFFIC = {
-    ("c2_llama2_7b", 4096): {"bytes": 287.3e6 + 38.6e6 + 135.4e6 + 68.4e6,
+    ("c2_llama2_7b", 4096): {"bytes": 251.1e6 + 38.5e6 + 135.4e6 + 70.6e6,
                              "source": "profiles/umma_grouped_gemm_c2_llama2_7b_T4096.md"},
 }
 
