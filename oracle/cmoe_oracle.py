@@ -18,7 +18,9 @@ the reconstruction-error identity (Eq. recon_error), router score = dense
 hidden activation of the representative neuron (Eq. rep_neuron/router),
 closed forms of the gate (Section 4.3), brute-force top-k, scalar per-neuron
 brute force, a library fp64 SwiGLU, permutation invariants, and hierarchical
-all-on = the original MoE layer (Section 4.4).
+all-on = the original MoE layer (Section 4.4); for the activation profiling
+stage (Appendix "Complete Activation Analysis Pipeline"): scalar brute force,
+row/column invariants, sign and scale invariance of ATopK, a hand-worked case.
 Parity unpinned (conventions the paper does not fix): the outer router's
 weights for an existing MoE layer (softmax over the selected logits), the
 tie-break between equal keys (lower index wins) and the NaN policy.
@@ -281,3 +283,67 @@ def fit_select_bias(s, top_k: int, target_share, iters: int = 4000,
         gamma = gamma_hi * (gamma_lo / gamma_hi) ** (it / max(iters - 1, 1))
         b = bias_update(b, counts, target, gamma)
     return b, counts
+
+
+# ------------------------------------------- Section 4.1 / Appendix: profiling
+def atopk(h, k_a: int) -> np.ndarray:
+    """Binary activation matrix A (Eq. atopk_appendix): A[t, i] = 1 when |h[t, i]|
+    is among the K_a largest magnitudes of row t.  Equal magnitudes at the cut
+    go to the lower neuron index (a convention; the paper does not fix it).
+    h: [q, d_h] -> uint8 [q, d_h]."""
+    mag = np.abs(_f64(h))
+    order = np.argsort(-mag, axis=1, kind="stable")[:, :k_a]
+    a = np.zeros(mag.shape, dtype=np.uint8)
+    np.put_along_axis(a, order, 1, axis=1)
+    return a
+
+
+def atopk_margin(h, k_a: int) -> np.ndarray:
+    """Relative gap between the K_a-th and (K_a+1)-th largest |h| of each row,
+    (m_K - m_{K+1}) / m_K: how far a row is from a different ATopK set."""
+    mag = -np.sort(-np.abs(_f64(h)), axis=1)
+    if k_a >= mag.shape[1]:
+        return np.full(mag.shape[0], np.inf)
+    top, nxt = mag[:, k_a - 1], mag[:, k_a]
+    return (top - nxt) / np.maximum(top, np.finfo(F64).tiny)
+
+
+def activation_counts(a) -> np.ndarray:
+    """Number of tokens for which each neuron is active; mu_i = counts_i / q
+    (Eq. mu_appendix).  a: [q, d_h] -> int64 [d_h]."""
+    return np.asarray(a, dtype=np.int64).sum(axis=0)
+
+
+def activation_rates(a) -> np.ndarray:
+    a = np.asarray(a)
+    return activation_counts(a) / F64(a.shape[0])
+
+
+def select_shared(counts, n_select: int) -> np.ndarray:
+    """The n_select = N_s*m neurons with the highest activation rate
+    (Eq. S_Ns_appendix), listed from the highest rate down; equal rates go to
+    the lower neuron index."""
+    counts = np.asarray(counts, dtype=np.int64)
+    return np.argsort(-counts, kind="stable")[:n_select].astype(np.int64)
+
+
+def pack_columns(a) -> np.ndarray:
+    """Bit-packed columns of A: word [i, t // 32] holds A[t, i] in bit t % 32
+    (the storage both sides use for the activation feature vectors c_i)."""
+    a = np.asarray(a, dtype=np.uint8)
+    q, d_h = a.shape
+    words = (q + 31) // 32
+    padded = np.zeros((words * 32, d_h), dtype=np.uint8)
+    padded[:q] = a
+    bits = padded.reshape(words, 32, d_h).astype(np.uint64)
+    weights = (np.uint64(1) << np.arange(32, dtype=np.uint64))[None, :, None]
+    return (bits * weights).sum(axis=1).astype(np.uint32).T.copy()
+
+
+def profile_activations(x, w_gate, w_up, k_a: int, n_select: int):
+    """Steps 1-4 of the profiling pipeline on calibration rows x [q, d]:
+    H (Eq. h_matrix_appendix), A (ATopK), counts (q * mu), shared-neuron list."""
+    h = hidden_activations(x, w_gate, w_up)
+    a = atopk(h, k_a)
+    counts = activation_counts(a)
+    return h, a, counts, select_shared(counts, n_select)

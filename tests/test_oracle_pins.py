@@ -307,11 +307,95 @@ def pin_hierarchical_is_weighted_sum_of_layers(o):
     np.testing.assert_allclose(sub, out[ids], rtol=1e-12, atol=1e-14)
 
 
+
+def pin_atopk_brute_force(o):
+    """ATopK against a scalar selection loop, with exact ties across the cut."""
+    rng = np.random.default_rng(21)
+    h = rng.normal(size=(23, 40))
+    h[3, [5, 9, 30]] = [2.5, -2.5, 2.5]          # equal magnitudes, mixed signs
+    h[3, 12] = 7.0
+    h[7] = np.round(h[7], 1)                      # many ties
+    for k_a in (1, 2, 3, 10):
+        a = o.atopk(h, k_a)
+        for t in range(h.shape[0]):
+            taken = []
+            for _ in range(k_a):
+                best = None
+                for i in range(h.shape[1]):
+                    if i in taken:
+                        continue
+                    if best is None or abs(h[t, i]) > abs(h[t, best]):   # strict: the lower index keeps a tie
+                        best = i
+                taken.append(best)
+            want = np.zeros(h.shape[1], dtype=np.uint8)
+            want[taken] = 1
+            np.testing.assert_array_equal(a[t], want)
+
+
+def pin_atopk_invariants(o):
+    rng = np.random.default_rng(22)
+    h = rng.normal(size=(50, 64))
+    a = o.atopk(h, 10)
+    assert a.dtype == np.uint8 and set(np.unique(a)) <= {0, 1}
+    np.testing.assert_array_equal(a.sum(axis=1), 10)                      # K_a ones per token
+    np.testing.assert_array_equal(o.atopk(-h, 10), a)                     # magnitude, not sign
+    np.testing.assert_array_equal(o.atopk(3.0 * h, 10), a)                # scale-free
+    np.testing.assert_array_equal(o.atopk(h, 64), np.ones_like(a))        # K_a = d_h: everything
+    big = np.abs(h) >= np.sort(np.abs(h), axis=1)[:, -10][:, None]
+    np.testing.assert_array_equal(a, big.astype(np.uint8))                # no ties here: a threshold test
+    perm = rng.permutation(64)
+    np.testing.assert_array_equal(o.atopk(h[:, perm], 10), a[:, perm])    # neuron order does not matter
+    m = o.atopk_margin(h, 10)
+    srt = -np.sort(-np.abs(h), axis=1)
+    np.testing.assert_allclose(m, (srt[:, 9] - srt[:, 10]) / srt[:, 9], rtol=1e-12)
+
+
+def pin_activation_rates_and_shared(o):
+    """Hand-worked: 4 tokens, 5 neurons, K_a = 2."""
+    h = np.array([[0.1, -3.0, 2.0, 0.0, 0.5],
+                  [4.0, -0.2, 0.3, 0.1, -5.0],
+                  [0.0, 1.0, -1.0, 0.2, 0.1],        # |1.0| ties |-1.0|: both are in the top two
+                  [0.3, 0.2, 0.1, -0.9, 0.8]])
+    a = o.atopk(h, 2)
+    np.testing.assert_array_equal(a, [[0, 1, 1, 0, 0], [1, 0, 0, 0, 1], [0, 1, 1, 0, 0], [0, 0, 0, 1, 1]])
+    counts = o.activation_counts(a)
+    np.testing.assert_array_equal(counts, [1, 2, 2, 1, 2])
+    np.testing.assert_allclose(o.activation_rates(a), [0.25, 0.5, 0.5, 0.25, 0.5])
+    assert counts.sum() == 2 * 4                                          # sum_i mu_i = K_a
+    np.testing.assert_array_equal(o.select_shared(counts, 3), [1, 2, 4])  # ties: lower index first
+    np.testing.assert_array_equal(o.select_shared(counts, 4), [1, 2, 4, 0])
+    bits = o.pack_columns(a)
+    assert bits.shape == (5, 1) and bits.dtype == np.uint32
+    np.testing.assert_array_equal(bits[:, 0], [0b0010, 0b0101, 0b0101, 0b1000, 0b1010])
+    rng = np.random.default_rng(23)
+    big = (rng.random((70, 9)) < 0.3).astype(np.uint8)
+    pb = o.pack_columns(big)
+    for t in range(70):
+        np.testing.assert_array_equal((pb[:, t // 32] >> np.uint32(t % 32)) & 1, big[t])
+    np.testing.assert_array_equal([sum(bin(int(w)).count("1") for w in row) for row in pb], big.sum(axis=0))
+
+
+def pin_profile_pipeline(o):
+    """Steps 1-4 chained: H is the dense hidden activation, a neuron whose gate and up vectors are
+    scaled up is active for almost every token and is selected first."""
+    shape, x, lay = small_layer(seed=24, d=16, n_experts=4, m=8, n_tok=29)
+    wg, wu = lay.w_gate.copy(), lay.w_up.copy()
+    wu[5] *= 1024.0                                # h is linear in the up vector: neuron 5 dominates
+    h, a, counts, shared = o.profile_activations(x, wg, wu, 3, 8)
+    np.testing.assert_allclose(h, o.hidden_activations(x, wg, wu), rtol=0, atol=0)
+    np.testing.assert_allclose(h[:, 5], 1024.0 * o.hidden_activations(x, lay.w_gate, lay.w_up)[:, 5], rtol=1e-12)
+    in_top3 = (np.abs(h) > np.abs(h[:, 5:6])).sum(axis=1) < 3
+    assert counts[5] == in_top3.sum() and counts[5] > 0.8 * x.shape[0] and shared[0] == 5
+    assert len(shared) == 8 and len(set(shared.tolist())) == 8
+    assert counts[shared].min() >= np.delete(counts, shared).max()
+
+
 PINS = [pin_dense_closed_form, pin_dense_library, pin_dense_per_neuron_brute_force,
         pin_all_experts_on_is_dense, pin_reconstruction_error_identity, pin_shared_always_on,
         pin_router_is_representative_activation, pin_gate_closed_forms, pin_topk_brute_force,
         pin_moe_linear_in_gates, pin_permutation, pin_logit_margin, pin_bias_update_rule,
-        pin_hierarchical_all_on_is_original_moe, pin_hierarchical_is_weighted_sum_of_layers]
+        pin_hierarchical_all_on_is_original_moe, pin_hierarchical_is_weighted_sum_of_layers,
+        pin_atopk_brute_force, pin_atopk_invariants, pin_activation_rates_and_shared, pin_profile_pipeline]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda p: p.__name__)
@@ -349,6 +433,15 @@ MUTATIONS = {
     "offsets_inclusive": ("off[e + 1] = off[e] + cnt[e]", "off[e + 1] = off[e] + cnt[e] + (e == 0)"),
     "outer_weights_unnormalised": ("outer_w = softmax(sel_logits)", "outer_w = np.exp(sel_logits)"),
     "bias_rule_sign": ("b[p > target] -= gamma", "b[p > target] += gamma"),
+    "atopk_signed": ("mag = np.abs(_f64(h))\n    order", "mag = _f64(h)\n    order"),
+    "atopk_smallest": ("order = np.argsort(-mag, axis=1, kind=\"stable\")[:, :k_a]",
+                       "order = np.argsort(mag, axis=1, kind=\"stable\")[:, :k_a]"),
+    "atopk_wrong_axis": ("np.put_along_axis(a, order, 1, axis=1)", "np.put_along_axis(a, order[:a.shape[1]].T[:a.shape[0]], 1, axis=0)"),
+    "counts_over_neurons": ("return np.asarray(a, dtype=np.int64).sum(axis=0)",
+                            "return np.asarray(a, dtype=np.int64).sum(axis=1)"),
+    "shared_lowest_rate": ("return np.argsort(-counts, kind=\"stable\")[:n_select]",
+                           "return np.argsort(counts, kind=\"stable\")[:n_select]"),
+    "pack_bit_order": ("np.uint64(1) << np.arange(32, dtype=np.uint64)", "np.uint64(1) << np.arange(31, -1, -1, dtype=np.uint64)"),
 }
 
 
