@@ -126,6 +126,36 @@ int cmoe_layer_get_gate_params(cmoe_layer* layer, float* gate_scale_u, float* se
 int cmoe_layer_update_bias(cmoe_layer* layer, float gamma, const float* target_share,
                            float* utilisation, void* stream);
 
+/* Activation profiling, steps 1-3 of the paper's pipeline (Section 4.1 "Activation Profiling";
+ * Appendix "Complete Activation Analysis Pipeline", Eq. h_matrix_appendix, Eq. atopk_appendix,
+ * Eq. mu_appendix): for n_tokens calibration rows x, H = Swish(x W_gate) * (x W_up), then per
+ * token the k_a hidden activations of largest magnitude (equal magnitudes at the cut go to the
+ * lower neuron index; NaN ranks last).  Neuron i of a selected pair (token, i) gets bit
+ * (token0 + t) % 32 of word act_bits[i * words_per_neuron + (token0 + t) / 32] set (its
+ * activation feature vector c_i, bit-packed) and act_count[i] incremented (q * mu_i).
+ *   layer    : a plain layer created with n_shared == n_experts and top_k == 0, i.e. the dense
+ *              FFN itself; neuron index i means position i of the neuron_perm it was created
+ *              with (the identity gives original neuron numbers).  H is held in the layer's
+ *              storage type (bf16 or fp32) and the selection is taken on those stored values.
+ *   x        : device, [n_tokens, d_model] in the layer's dtype, 16-byte aligned; 0 <= n_tokens <= max_tokens.
+ *   token0   : position of x's first row in the calibration set, so that a set larger than
+ *              max_tokens is profiled in chunks.
+ *   act_bits : device, uint32 [d_ff, words_per_neuron], words_per_neuron * 32 >= token0 + n_tokens.
+ *   act_count: device, int32 [d_ff].
+ * Both outputs accumulate: the caller zeroes them before the first chunk.  Asynchronous on
+ * `stream`; the buffers belong to the caller.  Errors: INVALID_ARG (layer has routed experts or
+ * is hierarchical, k_a outside [1, d_ff], null or misaligned pointers), CAPACITY, CUDA. */
+int cmoe_profile_activations(cmoe_layer* layer, const void* x, int32_t n_tokens, int32_t k_a, int32_t token0,
+                             uint32_t* act_bits, int32_t words_per_neuron, int32_t* act_count, void* stream);
+
+/* Step 4 (Eq. S_Ns_appendix): the n_select = N_s * m neurons with the highest activation
+ * count, written to shared_idx[0 .. n_select) from the highest count down; equal counts go
+ * to the lower neuron index.  act_count: device int32 [d_ff]; shared_idx: device int32
+ * [n_select].  No layer and no scratch memory are involved.  Asynchronous on `stream`.
+ * Errors: INVALID_ARG (n_select outside [0, d_ff], null pointers), CUDA. */
+int cmoe_select_shared(const int32_t* act_count, int32_t d_ff, int32_t n_select, int32_t* shared_idx,
+                       void* stream);
+
 /* Choose the expert-GEMM implementation: 0 = automatic (tensor-core path when the
  * dtype is bf16 and the shape allows, else the plain SIMT path), 1 = always SIMT,
  * 2 = tensor-core (single-CTA tiles), 3 = tensor-core on CTA pairs (cta_group::2) for batches

@@ -19,7 +19,7 @@ STAGE_NAMES = ["route", "permute", "gemm1_swiglu", "gemm2_down", "combine"]
 
 EXPORTS = [
     "cmoe_layer_create", "cmoe_hier_create", "cmoe_ffn_forward", "cmoe_layer_set_gate_params",
-    "cmoe_layer_get_gate_params", "cmoe_layer_update_bias", "cmoe_layer_set_gemm_path", "cmoe_layer_set_launch_chaining",
+    "cmoe_layer_get_gate_params", "cmoe_layer_update_bias", "cmoe_profile_activations", "cmoe_select_shared", "cmoe_layer_set_gemm_path", "cmoe_layer_set_launch_chaining",
     "cmoe_layer_dims", "cmoe_get_routing", "cmoe_layer_status",
     "cmoe_layer_launch_count", "cmoe_layer_enable_stage_timing", "cmoe_layer_stage_times",
     "cmoe_layer_destroy", "cmoe_token_permute_scratch_bytes",
@@ -59,6 +59,8 @@ def load() -> C.CDLL:
     lib.cmoe_layer_set_gate_params.argtypes = [vp, vp, vp, vp]
     lib.cmoe_layer_set_gemm_path.argtypes = [vp, i32]
     lib.cmoe_layer_set_launch_chaining.argtypes = [vp, i32]
+    lib.cmoe_profile_activations.argtypes = [vp, vp, i32, i32, i32, vp, i32, vp, vp]
+    lib.cmoe_select_shared.argtypes = [vp, i32, i32, vp, vp]
     lib.cmoe_layer_get_gate_params.argtypes = [vp, vp, vp, vp]
     lib.cmoe_layer_update_bias.argtypes = [vp, C.c_float, vp, vp, vp]
     lib.cmoe_layer_dims.argtypes = [vp] + [C.POINTER(i32)] * 4
@@ -191,6 +193,13 @@ class Layer:
                                              _stream_ptr(stream)), "cmoe_layer_update_bias")
         return util
 
+    def profile_activations(self, x, k_a: int, act_bits, act_count, token0: int = 0, stream=None) -> None:
+        """cmoe_profile_activations on CUDA tensors: x [n, d_model] in the layer's dtype, act_bits
+        int32/uint32-sized [d_ff, words], act_count int32 [d_ff]; both accumulate."""
+        _check(load().cmoe_profile_activations(self._h, x.data_ptr(), x.shape[0], k_a, token0, act_bits.data_ptr(),
+                                               act_bits.shape[1], act_count.data_ptr(), _stream_ptr(stream)),
+               "cmoe_profile_activations")
+
     def set_gemm_path(self, path: int) -> None:
         _check(load().cmoe_layer_set_gemm_path(self._h, path), "cmoe_layer_set_gemm_path")
 
@@ -279,6 +288,15 @@ def token_permute(topk_idx, n_groups: int, stream=None):
                                    scratch.data_ptr(), nbytes, _stream_ptr(stream))
     _check(st, "cmoe_token_permute")
     return counts, offsets, row_token[:n_rows * n_k], row_of
+
+
+def select_shared(act_count, n_select: int, stream=None):
+    """cmoe_select_shared on a CUDA int32 tensor [d_ff]; returns a CUDA int32 tensor [n_select]."""
+    import torch
+    out = torch.empty(max(n_select, 1), dtype=torch.int32, device=act_count.device)
+    _check(load().cmoe_select_shared(act_count.data_ptr(), act_count.shape[0], n_select, out.data_ptr(),
+                                     _stream_ptr(stream)), "cmoe_select_shared")
+    return out[:n_select]
 
 
 STATIC_PERMUTE_MAX_CELLS = 262144

@@ -17,6 +17,7 @@
 #include "combine.cuh"
 #include "common.cuh"
 #include "permute.cuh"
+#include "profile.cuh"
 #include "router.cuh"
 #include "router_mma.cuh"
 #include "simt_gemm.cuh"
@@ -305,7 +306,7 @@ int pack_weights(cmoe_layer* L, const void* w_gate, const void* w_up, const void
 }
 
 template <typename T>
-int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) {
+int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, bool gate_up_only = false) {
   const int d = L->cfg.d_model, n_r = L->n_r, n_k = L->cfg.top_k;
   const int R = n_tok * (L->hier ? L->outer_k : 1);
   const int P = R * n_k;
@@ -314,7 +315,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   int launches = 0;
   const T* xo = x;
   const bool use_umma = L->umma_ok && L->gemm_path != 1;     // 2: tensor, 3: tensor on CTA pairs
-  cudaEvent_t* ev = L->ev_ring ? &L->ev[(size_t)(L->ev_count % L->ev_ring) * (CMOE_N_STAGES + 1)] : nullptr;
+  cudaEvent_t* ev = (L->ev_ring && !gate_up_only) ? &L->ev[(size_t)(L->ev_count % L->ev_ring) * (CMOE_N_STAGES + 1)] : nullptr;
   auto mark = [&](int i) { if (ev) cudaEventRecord(ev[i], st); };
   mark(0);
   // Plain bf16 layers on the tensor path chain their kernels by programmatic dependent launch
@@ -400,9 +401,9 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
   if (use_umma) {
     // CTA pairs (cta_group::2, 256-row tiles) on request: measured equal to single-CTA tiles on
     // even groups and slower on ragged ones (an odd m-tile count idles half a pair)
-    const int n = decode ? decode_forward(&L->umma, &L->decode, L->gr, R, L->err_word, st, ev ? ev[3] : nullptr, dep)
+    const int n = decode ? decode_forward(&L->umma, &L->decode, L->gr, R, L->err_word, st, ev ? ev[3] : nullptr, dep, gate_up_only)
                 : pairs  ? umma2_forward(&L->umma, &L->pair, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
-                         : umma_forward(&L->umma, L->gr, gather_mode, xo, L->err_word, st, ev ? ev[3] : nullptr, dep);
+                         : umma_forward(&L->umma, L->gr, gather_mode, xo, L->err_word, st, ev ? ev[3] : nullptr, dep, gate_up_only);
     if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     launches += n;
   } else {
@@ -416,6 +417,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
     dim3 g1((R + kSimtTile - 1) / kSimtTile, (max_w + kSimtTile - 1) / kSimtTile, L->n_groups_total());
     simt_gemm1_kernel<T><<<g1, 256, 0, st>>>(a);
     mark(3);
+    if (gate_up_only) { L->launches = launches + 1; CU_TRY(cudaGetLastError()); return CMOE_OK; }
     a.a_shared = (const T*)L->h_s; a.a_routed = (const T*)L->h_r;
     a.w_gate = (const T*)L->wd_p; a.w_up = nullptr;
     a.c_shared = (T*)L->y_s; a.c_routed = (T*)L->y_r;
@@ -424,6 +426,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st) 
     launches += 2;
   }
 
+  if (gate_up_only) { L->launches = launches; CU_TRY(cudaGetLastError()); return CMOE_OK; }   // H_s is complete
   mark(4);
   const int per_thread = sizeof(T) == 2 ? 16 : 8;
   const int threads = d / per_thread < 256 ? ((d / per_thread + 31) / 32 * 32) : 256;
@@ -616,6 +619,51 @@ int cmoe_ffn_forward(cmoe_layer* L, const void* x, int32_t T, void* out, void* s
   L->last_T = T;
   return L->cfg.dtype == CMOE_BF16 ? forward_impl<bf16>(L, (const bf16*)x, T, (bf16*)out, st)
                                    : forward_impl<float>(L, (const float*)x, T, (float*)out, st);
+}
+
+int cmoe_profile_activations(cmoe_layer* L, const void* x, int32_t T, int32_t k_a, int32_t token0,
+                             uint32_t* act_bits, int32_t words_per_neuron, int32_t* act_count, void* stream) {
+  if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "null layer");
+  if (L->hier || L->n_r != 0 || L->cfg.n_shared != L->cfg.n_experts)
+    return arg_fail(CMOE_ERR_INVALID_ARG, "profiling needs a plain layer whose experts are all shared");
+  if (T < 0 || token0 < 0) return arg_fail(CMOE_ERR_INVALID_ARG, "negative token count / offset");
+  if (T == 0) return CMOE_OK;
+  if (!x || !act_bits || !act_count) return arg_fail(CMOE_ERR_INVALID_ARG, "null x / act_bits / act_count");
+  if (T > L->cfg.max_tokens) return arg_fail(CMOE_ERR_CAPACITY, "T exceeds max_tokens");
+  if (k_a < 1 || k_a > L->cfg.d_ff) return arg_fail(CMOE_ERR_INVALID_ARG, "k_a outside [1, d_ff]");
+  if ((long long)words_per_neuron * 32 < (long long)token0 + T)
+    return arg_fail(CMOE_ERR_CAPACITY, "words_per_neuron too small for token0 + n_tokens");
+  if (reinterpret_cast<uintptr_t>(x) & 15) return arg_fail(CMOE_ERR_INVALID_ARG, "x must be 16-byte aligned");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  L->last_stream = st;
+  L->last_T = T;
+  const int d_ff = L->cfg.d_ff;
+  int rc;
+  if (L->cfg.dtype == CMOE_BF16) {
+    rc = forward_impl<bf16>(L, (const bf16*)x, T, nullptr, st, true);
+    if (rc == CMOE_OK)
+      atopk_kernel<bf16><<<T, kAtopkThreads, 0, st>>>((const bf16*)L->h_s, d_ff, d_ff, k_a, token0, act_bits,
+                                                      words_per_neuron, act_count);
+  } else {
+    rc = forward_impl<float>(L, (const float*)x, T, nullptr, st, true);
+    if (rc == CMOE_OK)
+      atopk_kernel<float><<<T, kAtopkThreads, 0, st>>>((const float*)L->h_s, d_ff, d_ff, k_a, token0, act_bits,
+                                                       words_per_neuron, act_count);
+  }
+  if (rc != CMOE_OK) return rc;
+  L->launches += 1;
+  CU_TRY(cudaGetLastError());
+  return CMOE_OK;
+}
+
+int cmoe_select_shared(const int32_t* act_count, int32_t d_ff, int32_t n_select, int32_t* shared_idx, void* stream) {
+  if (d_ff < 0 || n_select < 0 || n_select > d_ff) return arg_fail(CMOE_ERR_INVALID_ARG, "n_select outside [0, d_ff]");
+  if (d_ff == 0 || n_select == 0) return CMOE_OK;
+  if (!act_count || !shared_idx) return arg_fail(CMOE_ERR_INVALID_ARG, "null act_count / shared_idx");
+  select_shared_kernel<<<(d_ff + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(act_count, d_ff, n_select,
+                                                                                         shared_idx);
+  CU_TRY(cudaGetLastError());
+  return CMOE_OK;
 }
 
 int cmoe_layer_set_gate_params(cmoe_layer* L, const float* u, const float* b, void* stream) {

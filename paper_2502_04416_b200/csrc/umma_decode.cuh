@@ -446,7 +446,7 @@ inline bool decode_bind_x(UmmaPlan* P, DecodePlan* D, const void* x_rows, int n_
 // rule would split some group even if the largest possible set of experts were active for
 // n_rows rows (fewer active experts only split more).  Returns launches or -1.
 inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n_rows, int32_t* err_word,
-                          cudaStream_t st, cudaEvent_t mid, bool dep = false) {
+                          cudaStream_t st, cudaEvent_t mid, bool dep = false, bool gate_up_only = false) {
   const UmmaShape& s = P->shape;
   const long long act_s = P->has_s ? (s.n_outer < n_rows ? s.n_outer : n_rows) : 0;
   const long long all_r = (long long)s.n_outer * s.n_r, picks = (long long)n_rows * s.n_k;
@@ -470,14 +470,15 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n
                 dim3(kUmmaThreads), decode_smem_bytes<4>(), st, D->w_gu, D->w_gu, D->x_rows64, D->x_rows64, a);
   if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
-  launch_kernel(dep, split2 ? umma_decode_kernel<5, true> : umma_decode_kernel<5, false>, dim3(P->n_sms),
-                dim3(kUmmaThreads), decode_smem_bytes<5>(), st, D->wd_s, D->wd_r, D->h_s, D->h_r, a);
+  if (!gate_up_only)
+    launch_kernel(dep, split2 ? umma_decode_kernel<5, true> : umma_decode_kernel<5, false>, dim3(P->n_sms),
+                  dim3(kUmmaThreads), decode_smem_bytes<5>(), st, D->wd_s, D->wd_r, D->h_s, D->h_r, a);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
     snprintf(P->error, sizeof(P->error), "decode GEMM launch: %s", cudaGetErrorString(e));
     return -1;
   }
-  return 2;
+  return gate_up_only ? 1 : 2;
 }
 
 }  // namespace cmoe

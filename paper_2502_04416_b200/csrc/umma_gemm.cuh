@@ -779,7 +779,7 @@ inline int umma_router_forward(UmmaPlan* P, int n_rows, const int32_t* outer_off
 // their rows of x (0 permuted copy, 1 TMA gather4, 2 cp.async gather).  Requires umma_bind_x for this
 // forward.  Returns the number of kernels launched, or -1 (P->error).
 inline int umma_forward(UmmaPlan* P, const GroupRows* gr, int gather_mode, const void* x_rows, int32_t* err_word,
-                        cudaStream_t st, cudaEvent_t mid, bool dep = false) {
+                        cudaStream_t st, cudaEvent_t mid, bool dep = false, bool gate_up_only = false) {
   const UmmaShape& s = P->shape;
   UmmaArgs a = umma_base_args(P, gr, err_word);
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
@@ -789,14 +789,15 @@ inline int umma_forward(UmmaPlan* P, const GroupRows* gr, int gather_mode, const
                 st, P->x_rows, (gather_mode != 0 || !P->has_r) ? P->x_gather : P->x_perm, P->b1_s, P->b1_r, a);
   if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
-  launch_kernel(dep, umma_grouped_kernel<2>, dim3(P->n_sms), dim3(kUmmaThreads), kUmmaSmemBytes, st, P->a2_s,
-                P->a2_r, P->b2_s, P->b2_r, a);
+  if (!gate_up_only)
+    launch_kernel(dep, umma_grouped_kernel<2>, dim3(P->n_sms), dim3(kUmmaThreads), kUmmaSmemBytes, st, P->a2_s,
+                  P->a2_r, P->b2_s, P->b2_r, a);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
     snprintf(P->error, sizeof(P->error), "tensor-core GEMM launch: %s", cudaGetErrorString(e));
     return -1;
   }
-  return 2;
+  return gate_up_only ? 1 : 2;
 }
 
 }  // namespace cmoe
