@@ -382,6 +382,97 @@ def run_gpu(args):
 
 
 # ------------------------------------------------------------ reference arm
+# ------------------------------------------------- activation profiling stage
+def run_profile(args):
+    """Steps 1-4 of the paper's activation-profiling pipeline on a synthetic calibration set of the
+    paper's size (8 x 2048 tokens, K_a = 10) for the workload's FFN: a step is one pass over the set
+    in chunks of 4096 rows plus the shared-neuron selection."""
+    import dataclasses
+    import numpy as np
+    import torch
+    from paper_2502_04416_b200 import binding, torch_io
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    binding.load()
+    w = wl.WORKLOADS[args.workload]
+    shape = dataclasses.replace(w.shape, n_shared=w.shape.n_experts, top_k=0)
+    inputs = wl.make_inputs(dataclasses.replace(w, shape=shape, tokens=(8,), n_outer=0))
+    lay = inputs.layers[0]
+    lay.neuron_perm = np.arange(shape.d_ff, dtype=np.int32)
+    lay.rep_idx = np.zeros(0, dtype=np.int32)
+    q, chunk, k_a = args.tokens or 16384, 4096, 10
+    n_select = 2 * (shape.d_ff // shape.n_experts)
+    rng = np.random.Generator(np.random.PCG64(1234))
+    x_host = wl.round_to_storage(rng.standard_normal((q, shape.d_model), dtype=np.float32), shape.dtype)
+    layer = torch_io.layer_from_inputs(lay, min(chunk, q))
+    x = torch_io.to_device(x_host, shape.dtype)
+    bits = torch.zeros((shape.d_ff, (q + 31) // 32), dtype=torch.int32, device="cuda")
+    count = torch.zeros(shape.d_ff, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        bits.zero_()
+        count.zero_()
+        for t0 in range(0, q, chunk):
+            layer.profile_activations(x[t0:t0 + chunk], k_a, bits, count, token0=t0)
+        return binding.select_shared(count, n_select)
+
+    steps = min(args.steps, 200)
+    sampler = ClockSampler(local)
+    sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler.wait_first()
+    sampler.mark_begin()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    sampler.mark_end()
+    time.sleep(0.12)
+    clocks = sampler.stop()
+    ms_total = max_over_ranks(e0.elapsed_time(e1), "cuda")
+    assert layer.status() == 0
+    value = world * q * steps / (ms_total * 1e-3)
+    peaks = load_peaks()
+    flops = 4.0 * shape.d_model * shape.d_ff * q
+    ach = flops / (ms_total / steps * 1e-3) / 1e12
+    line = {
+        "metric": "activation_profile_tokens_per_s", "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_total / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": shape.dtype, "data": "synthetic",
+        "config": {"workload": f"{w.name} profiling q={q} K_a={k_a}", "d_model": shape.d_model, "d_ff": shape.d_ff,
+                   "chunk": chunk, "l2": "weights and H exceed the 126 MB L2"},
+        "gpu_launches": (3 * ((q + chunk - 1) // chunk) + 1) * steps, "clocks": clocks,
+        "roofline": {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": ach / peaks["bf16_tflops"], "traffic": None,
+                     "kernel": "whole profiling pass (gate/up GEMM + ATopK + selection)",
+                     "peak_source": peaks["source"]},
+    }
+    if rank == 0:
+        from oracle import cmoe_oracle as oracle
+        sample = min(args.cpu_sample_tokens, q)
+        t0 = time.perf_counter()
+        oracle.profile_activations(x_host[:sample], lay.w_gate, lay.w_up, k_a, n_select)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": sample / dt, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+                                "sample": f"first {sample} calibration rows, one pass, {dt:.2f} s"}
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    return line if rank == 0 else None
+
+
 def run_reference(args):
     """The CPU oracle, unmodified, timed on the host cores on a bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
@@ -427,6 +518,8 @@ def main():
                     help="replay the forward from a CUDA graph (auto: batches of at most 512 tokens)")
     ap.add_argument("--chain", choices=["on", "off"], default="on",
                     help="programmatic dependent launches between the kernels of a forward (library default: on)")
+    ap.add_argument("--stage", choices=["forward", "profile"], default="forward",
+                    help="forward: the MoE forward pass (the headline metric); profile: the activation-profiling pass")
     ap.add_argument("--forward-only", action="store_true",
                     help="run only the timed forward passes (for profiler captures)")
     args = ap.parse_args()
@@ -434,7 +527,7 @@ def main():
         line = run_reference(args)
     else:
         args.warmup = max(args.warmup, 3)
-        line = run_gpu(args)
+        line = run_profile(args) if args.stage == "profile" else run_gpu(args)
     if line is not None:
         print(json.dumps(line))
 
