@@ -41,7 +41,7 @@ typedef enum {
   CMOE_ERR_CAPACITY = -4,        /* T > max_tokens, or a size beyond a stated maximum */
   CMOE_ERR_CUDA = -5,            /* a CUDA runtime/driver call failed (see cmoe_last_error) */
   CMOE_ERR_DEVICE_TIMEOUT = -6,  /* a bounded device-side wait gave up (see cmoe_layer_status) */
-  CMOE_ERR_UNSUPPORTED = -7      /* the device is not compute capability 10.x */
+  CMOE_ERR_UNSUPPORTED = -7      /* the device is not compute capability 10.x, or a size beyond a stated limit */
 } cmoe_status;
 
 typedef enum { CMOE_BF16 = 0, CMOE_FP32 = 1 } cmoe_dtype;
@@ -144,7 +144,8 @@ int cmoe_layer_update_bias(cmoe_layer* layer, float gamma, const float* target_s
  *   act_count: device, int32 [d_ff].
  * Both outputs accumulate: the caller zeroes them before the first chunk.  Asynchronous on
  * `stream`; the buffers belong to the caller.  Errors: INVALID_ARG (layer has routed experts or
- * is hierarchical, k_a outside [1, d_ff], null or misaligned pointers), CAPACITY, CUDA. */
+ * is hierarchical, k_a outside [1, d_ff], null or misaligned pointers), CAPACITY, UNSUPPORTED
+ * (d_ff above 24576 for bf16 or 12288 for fp32: a row's keys are staged in 48 KB of shared memory), CUDA. */
 int cmoe_profile_activations(cmoe_layer* layer, const void* x, int32_t n_tokens, int32_t k_a, int32_t token0,
                              uint32_t* act_bits, int32_t words_per_neuron, int32_t* act_count, void* stream);
 

@@ -638,16 +638,18 @@ int cmoe_profile_activations(cmoe_layer* L, const void* x, int32_t T, int32_t k_
   L->last_stream = st;
   L->last_T = T;
   const int d_ff = L->cfg.d_ff;
+  if ((size_t)d_ff * L->esz > 48 * 1024)      // the row's keys are staged in (default-sized) shared memory
+    return arg_fail(CMOE_ERR_UNSUPPORTED, "profiling supports d_ff up to 24576 (bf16) / 12288 (fp32)");
   int rc;
   if (L->cfg.dtype == CMOE_BF16) {
     rc = forward_impl<bf16>(L, (const bf16*)x, T, nullptr, st, true);
     if (rc == CMOE_OK)
-      atopk_kernel<bf16><<<T, kAtopkThreads, 0, st>>>((const bf16*)L->h_s, d_ff, d_ff, k_a, token0, act_bits,
+      atopk_kernel<bf16><<<T, kAtopkThreads, (size_t)d_ff * sizeof(uint16_t), st>>>((const bf16*)L->h_s, d_ff, d_ff, k_a, token0, act_bits,
                                                       words_per_neuron, act_count);
   } else {
     rc = forward_impl<float>(L, (const float*)x, T, nullptr, st, true);
     if (rc == CMOE_OK)
-      atopk_kernel<float><<<T, kAtopkThreads, 0, st>>>((const float*)L->h_s, d_ff, d_ff, k_a, token0, act_bits,
+      atopk_kernel<float><<<T, kAtopkThreads, (size_t)d_ff * sizeof(uint32_t), st>>>((const float*)L->h_s, d_ff, d_ff, k_a, token0, act_bits,
                                                        words_per_neuron, act_count);
   }
   if (rc != CMOE_OK) return rc;
@@ -660,7 +662,7 @@ int cmoe_select_shared(const int32_t* act_count, int32_t d_ff, int32_t n_select,
   if (d_ff < 0 || n_select < 0 || n_select > d_ff) return arg_fail(CMOE_ERR_INVALID_ARG, "n_select outside [0, d_ff]");
   if (d_ff == 0 || n_select == 0) return CMOE_OK;
   if (!act_count || !shared_idx) return arg_fail(CMOE_ERR_INVALID_ARG, "null act_count / shared_idx");
-  select_shared_kernel<<<(d_ff + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(act_count, d_ff, n_select,
+  select_shared_kernel<<<(d_ff + 31) / 32, 256, 0, static_cast<cudaStream_t>(stream)>>>(act_count, d_ff, n_select,
                                                                                          shared_idx);
   CU_TRY(cudaGetLastError());
   return CMOE_OK;
