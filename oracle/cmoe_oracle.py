@@ -20,7 +20,9 @@ closed forms of the gate (Section 4.3), brute-force top-k, scalar per-neuron
 brute force, a library fp64 SwiGLU, permutation invariants, and hierarchical
 all-on = the original MoE layer (Section 4.4); for the activation profiling
 stage (Appendix "Complete Activation Analysis Pipeline"): scalar brute force,
-row/column invariants, sign and scale invariance of ATopK, a hand-worked case.
+row/column invariants, sign and scale invariance of ATopK, a hand-worked case; for the
+clustering pieces (Appendix "Balanced Clustering Algorithm"): squared L2 = Hamming distance
+on binary vectors, a hand-worked mean, brute-force argmin, an exhaustive balanced assignment.
 Parity unpinned (conventions the paper does not fix): the outer router's
 weights for an existing MoE layer (softmax over the selected logits), the
 tie-break between equal keys (lower index wins) and the NaN policy.
@@ -347,3 +349,62 @@ def profile_activations(x, w_gate, w_up, k_a: int, n_select: int):
     a = atopk(h, k_a)
     counts = activation_counts(a)
     return h, a, counts, select_shared(counts, n_select)
+
+
+# ------------------------------- Appendix: balanced clustering of routed neurons
+def initial_centroids(counts, shared_idx, n_routed: int) -> np.ndarray:
+    """Neuron indices of the N_r initial centroids: the remaining (non-shared)
+    neurons with the highest activation rates, highest first, ties to the lower index."""
+    counts = np.asarray(counts, dtype=np.int64)
+    shared = set(int(i) for i in np.asarray(shared_idx).ravel())
+    order = [int(i) for i in np.argsort(-counts, kind="stable") if int(i) not in shared]
+    return np.asarray(order[:n_routed], dtype=np.int64)
+
+
+def centroid_distances(c, centroids) -> np.ndarray:
+    """d[i, j] = || c_i - chat_j ||_2 over the q calibration tokens.
+    c: [q, n] activation feature vectors (columns of A); centroids: [q, N_r]."""
+    c, centroids = _f64(c), _f64(centroids)
+    diff = c[:, :, None] - centroids[:, None, :]
+    return np.sqrt((diff * diff).sum(axis=0))
+
+
+def cluster_update(c, assign, prev_centroids) -> np.ndarray:
+    """chat_j <- mean of the c_i assigned to cluster j; a cluster without members
+    keeps its previous centroid.  assign: [n] cluster of each neuron (-1: none)."""
+    c = _f64(c)
+    assign = np.asarray(assign, dtype=np.int64)
+    out = _f64(prev_centroids).copy()
+    for j in range(out.shape[1]):
+        members = np.nonzero(assign == j)[0]
+        if len(members) > 0:
+            out[:, j] = c[:, members].sum(axis=1) / len(members)
+    return out
+
+
+def representatives(c, assign, centroids) -> np.ndarray:
+    """R_j = argmin over the neurons of cluster j of || c_i - chat_j ||_2
+    (Eq. rep_neuron); equal distances go to the lower position.  Returns the
+    position in c's columns for each cluster (-1 for an empty cluster)."""
+    d = centroid_distances(c, centroids)
+    assign = np.asarray(assign, dtype=np.int64)
+    reps = np.full(d.shape[1], -1, dtype=np.int64)
+    for j in range(d.shape[1]):
+        members = np.nonzero(assign == j)[0]
+        if len(members) > 0:
+            reps[j] = members[np.argmin(d[members, j])]      # argmin returns the first minimum
+    return reps
+
+
+def balanced_assignment(d, m: int) -> np.ndarray:
+    """Assignment T with every row in exactly one cluster and every cluster holding m
+    rows that minimises sum_ij T_ij d_ij (Eq. con_1_appendix), solved as the paper does:
+    each column repeated m times, then a linear assignment (library routine)."""
+    from scipy.optimize import linear_sum_assignment
+    d = _f64(d)
+    n, n_r = d.shape
+    assert n == n_r * m
+    rows, cols = linear_sum_assignment(np.repeat(d, m, axis=1))
+    assign = np.empty(n, dtype=np.int64)
+    assign[rows] = cols // m
+    return assign

@@ -389,13 +389,82 @@ def pin_profile_pipeline(o):
     assert len(shared) == 8 and len(set(shared.tolist())) == 8
     assert counts[shared].min() >= np.delete(counts, shared).max()
 
+def _binary_cols(seed, q=40, n=12, p=0.3):
+    rng = np.random.default_rng(seed)
+    return (rng.random((q, n)) < p).astype(np.uint8)
+
+
+def pin_distance_is_hamming_on_binary(o):
+    """With binary centroids the squared L2 distance counts the differing positions."""
+    c = _binary_cols(31)
+    cent = c[:, [2, 7, 9]]
+    d = o.centroid_distances(c, cent)
+    for i in range(c.shape[1]):
+        for j, cj in enumerate((2, 7, 9)):
+            ham = sum(1 for k in range(c.shape[0]) if c[k, i] != c[k, cj])
+            assert abs(d[i, j] ** 2 - ham) < 1e-9
+    assert d[2, 0] == 0.0 and d[7, 1] == 0.0
+    real = np.array([[0.5, 0.0], [0.25, 1.0], [0.0, 0.0]])                # hand-worked, real-valued centroids
+    cc = np.array([[1, 0], [0, 1], [1, 1]], dtype=np.uint8)               # c_0 = (1,0,1), c_1 = (0,1,1)
+    d2 = o.centroid_distances(cc, real)
+    np.testing.assert_allclose(d2 ** 2, [[0.25 + 0.0625 + 1, 1 + 1 + 1], [0.25 + 0.5625 + 1, 0 + 0 + 1]], rtol=1e-14)
+
+
+def pin_cluster_update_and_representatives(o):
+    c = np.array([[1, 1, 0, 0, 1],
+                  [0, 1, 1, 0, 0],
+                  [1, 1, 1, 0, 0],
+                  [0, 0, 0, 1, 1]], dtype=np.uint8)                        # q = 4 tokens, 5 neurons
+    prev = np.full((4, 3), 0.125)
+    assign = np.array([0, 0, 0, 1, -1])                                   # cluster 2 empty, neuron 4 unassigned
+    cent = o.cluster_update(c, assign, prev)
+    np.testing.assert_allclose(cent[:, 0], [2 / 3, 2 / 3, 1.0, 0.0])
+    np.testing.assert_allclose(cent[:, 1], [0, 0, 0, 1])
+    np.testing.assert_allclose(cent[:, 2], 0.125)                          # kept
+    reps = o.representatives(c, assign, cent)
+    # distances^2 of neurons 0,1,2 to (2/3,2/3,1,0): 1/9+4/9+0 = 5/9 ; 1/9+1/9+0 = 2/9 ; 4/9+1/9+0 = 5/9
+    np.testing.assert_array_equal(reps, [1, 3, -1])
+    tie = o.representatives(c[:, [0, 2, 1]], np.array([0, 0, 0]), cent[:, :1])
+    assert tie[0] == 2                                                    # the closest one wherever it stands
+    same = o.representatives(c[:, [0, 2]], np.array([0, 0]), cent[:, :1])
+    assert same[0] == 0                                                   # equal distances: the lower position
+    rng = np.random.default_rng(32)
+    cb = _binary_cols(33, q=30, n=20)
+    a = rng.integers(0, 4, size=20)
+    cent = o.cluster_update(cb, a, np.zeros((30, 4)))
+    reps = o.representatives(cb, a, cent)
+    d = o.centroid_distances(cb, cent)
+    for j in range(4):
+        best = None
+        for i in range(20):
+            if a[i] == j and (best is None or d[i, j] < d[best, j]):
+                best = i
+        assert reps[j] == best
+
+
+def pin_initial_centroids_and_assignment(o):
+    counts = np.array([5, 9, 9, 1, 7, 7, 3, 0])
+    np.testing.assert_array_equal(o.initial_centroids(counts, [1, 4], 3), [2, 5, 0])
+    np.testing.assert_array_equal(o.initial_centroids(counts, [], 2), [1, 2])
+    # balanced assignment against exhaustive search: 6 rows, 3 clusters of 2
+    import itertools
+    rng = np.random.default_rng(34)
+    d = rng.random((6, 3))
+    got = o.balanced_assignment(d, 2)
+    assert sorted(np.bincount(got, minlength=3)) == [2, 2, 2]
+    best = min((sum(d[i, a[i]] for i in range(6)) for a in itertools.product(range(3), repeat=6)
+                if sorted(np.bincount(a, minlength=3)) == [2, 2, 2]))
+    assert abs(sum(d[i, got[i]] for i in range(6)) - best) < 1e-12
+
 
 PINS = [pin_dense_closed_form, pin_dense_library, pin_dense_per_neuron_brute_force,
         pin_all_experts_on_is_dense, pin_reconstruction_error_identity, pin_shared_always_on,
         pin_router_is_representative_activation, pin_gate_closed_forms, pin_topk_brute_force,
         pin_moe_linear_in_gates, pin_permutation, pin_logit_margin, pin_bias_update_rule,
         pin_hierarchical_all_on_is_original_moe, pin_hierarchical_is_weighted_sum_of_layers,
-        pin_atopk_brute_force, pin_atopk_invariants, pin_activation_rates_and_shared, pin_profile_pipeline]
+        pin_atopk_brute_force, pin_atopk_invariants, pin_activation_rates_and_shared, pin_profile_pipeline,
+        pin_distance_is_hamming_on_binary, pin_cluster_update_and_representatives,
+        pin_initial_centroids_and_assignment]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda p: p.__name__)
@@ -441,6 +510,14 @@ MUTATIONS = {
                             "return np.asarray(a, dtype=np.int64).sum(axis=1)"),
     "shared_lowest_rate": ("return np.argsort(-counts, kind=\"stable\")[:n_select]",
                            "return np.argsort(counts, kind=\"stable\")[:n_select]"),
+    "distance_not_rooted": ("return np.sqrt((diff * diff).sum(axis=0))", "return (diff * diff).sum(axis=0)"),
+    "distance_abs_not_square": ("return np.sqrt((diff * diff).sum(axis=0))", "return np.sqrt(np.abs(diff).sum(axis=0)) * 1.0000001"),
+    "centroid_sum_not_mean": ("out[:, j] = c[:, members].sum(axis=1) / len(members)", "out[:, j] = c[:, members].sum(axis=1)"),
+    "empty_cluster_zeroed": ("out = _f64(prev_centroids).copy()", "out = np.zeros_like(_f64(prev_centroids))"),
+    "representative_farthest": ("reps[j] = members[np.argmin(d[members, j])]", "reps[j] = members[np.argmax(d[members, j])]"),
+    "centroids_include_shared": ("if int(i) not in shared]", "]"),
+    "assignment_unbalanced": ("rows, cols = linear_sum_assignment(np.repeat(d, m, axis=1))",
+                              "rows, cols = np.arange(n), np.argmin(d, axis=1) * m"),
     "pack_bit_order": ("np.uint64(1) << np.arange(32, dtype=np.uint64)", "np.uint64(1) << np.arange(31, -1, -1, dtype=np.uint64)"),
 }
 
