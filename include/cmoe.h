@@ -157,6 +157,42 @@ int cmoe_profile_activations(cmoe_layer* layer, const void* x, int32_t n_tokens,
 int cmoe_select_shared(const int32_t* act_count, int32_t d_ff, int32_t n_select, int32_t* shared_idx,
                        void* stream);
 
+/* Data-parallel pieces of the balanced K-means that partitions the non-shared neurons into
+ * routed experts (Appendix "Balanced Clustering Algorithm for Routed Experts") and of the
+ * representative-neuron choice (Eq. rep_neuron).  They work on the bit rows act_bits written
+ * by cmoe_profile_activations (row i = activation feature vector c_i over n_tokens calibration
+ * tokens) for the n neurons listed in neuron_idx (device int32 [n], rows of act_bits).  A
+ * centroid, being the mean of binary vectors, is held exactly: centroid_count[j][k] = number
+ * of cluster j's members active for token k (device int32 [n_clusters, n_tokens]) and
+ * cluster_size[j] = its member count (device int32 [n_clusters]); chat_j = count_j / size_j.
+ * The balanced assignment itself (a sequential O(n^3) solver in the paper) is not provided.
+ * Limits: n_clusters <= 32, n_tokens * n < 2^31.  All three calls are asynchronous on `stream`,
+ * allocate nothing, and leave their buffers to the caller.  Errors: INVALID_ARG, CAPACITY, CUDA.
+ *
+ * cmoe_cluster_update (the cluster-update rule): assign[i] in [0, n_clusters) is neuron
+ *   neuron_idx[i]'s cluster, any other value means unassigned.  Every cluster with at least one
+ *   member gets its count vector and size rebuilt; a cluster without members keeps both, as
+ *   the paper's rule keeps the old centroid.  (Initial centroids: n_clusters neurons, assign[i] = i.) */
+int cmoe_cluster_update(const uint32_t* act_bits, int32_t words_per_neuron, int32_t n_tokens,
+                        const int32_t* neuron_idx, const int32_t* assign, int32_t n, int32_t n_clusters,
+                        int32_t* centroid_count, int32_t* cluster_size, void* stream);
+
+/* cmoe_cluster_distances (the distance matrix D): scaled_sq_dist[i, j] (device int64
+ *   [n, n_clusters]) = size_j^2 * || c_i - chat_j ||_2^2, an exact integer; d_ij =
+ *   sqrt(scaled_sq_dist[i, j]) / size_j.  With binary centroids (size 1) it is the Hamming
+ *   distance.  centroid_sqnorm: device int64 [n_clusters], written by the call (||count_j||^2).
+ *   Every cluster_size[j] must be at least 1. */
+int cmoe_cluster_distances(const uint32_t* act_bits, int32_t words_per_neuron, int32_t n_tokens,
+                           const int32_t* neuron_idx, int32_t n, const int32_t* centroid_count,
+                           const int32_t* cluster_size, int32_t n_clusters, int64_t* centroid_sqnorm,
+                           int64_t* scaled_sq_dist, void* stream);
+
+/* cmoe_cluster_representatives (Eq. rep_neuron): rep_neuron[j] (device int32 [n_clusters]) =
+ *   neuron_idx[i] of the member i of cluster j with the smallest scaled_sq_dist[i, j]; equal
+ *   distances go to the lower position i; -1 for a cluster without members. */
+int cmoe_cluster_representatives(const int64_t* scaled_sq_dist, const int32_t* neuron_idx, const int32_t* assign,
+                                 int32_t n, int32_t n_clusters, int32_t* rep_neuron, void* stream);
+
 /* Choose the expert-GEMM implementation: 0 = automatic (tensor-core path when the
  * dtype is bf16 and the shape allows, else the plain SIMT path), 1 = always SIMT,
  * 2 = tensor-core (single-CTA tiles), 3 = tensor-core on CTA pairs (cta_group::2) for batches

@@ -19,7 +19,8 @@ STAGE_NAMES = ["route", "permute", "gemm1_swiglu", "gemm2_down", "combine"]
 
 EXPORTS = [
     "cmoe_layer_create", "cmoe_hier_create", "cmoe_ffn_forward", "cmoe_layer_set_gate_params",
-    "cmoe_layer_get_gate_params", "cmoe_layer_update_bias", "cmoe_profile_activations", "cmoe_select_shared", "cmoe_layer_set_gemm_path", "cmoe_layer_set_launch_chaining",
+    "cmoe_layer_get_gate_params", "cmoe_layer_update_bias", "cmoe_profile_activations", "cmoe_select_shared",
+    "cmoe_cluster_update", "cmoe_cluster_distances", "cmoe_cluster_representatives", "cmoe_layer_set_gemm_path", "cmoe_layer_set_launch_chaining",
     "cmoe_layer_dims", "cmoe_get_routing", "cmoe_layer_status",
     "cmoe_layer_launch_count", "cmoe_layer_enable_stage_timing", "cmoe_layer_stage_times",
     "cmoe_layer_destroy", "cmoe_token_permute_scratch_bytes",
@@ -61,6 +62,9 @@ def load() -> C.CDLL:
     lib.cmoe_layer_set_launch_chaining.argtypes = [vp, i32]
     lib.cmoe_profile_activations.argtypes = [vp, vp, i32, i32, i32, vp, i32, vp, vp]
     lib.cmoe_select_shared.argtypes = [vp, i32, i32, vp, vp]
+    lib.cmoe_cluster_update.argtypes = [vp, i32, i32, vp, vp, i32, i32, vp, vp, vp]
+    lib.cmoe_cluster_distances.argtypes = [vp, i32, i32, vp, i32, vp, vp, i32, vp, vp, vp]
+    lib.cmoe_cluster_representatives.argtypes = [vp, vp, vp, i32, i32, vp, vp]
     lib.cmoe_layer_get_gate_params.argtypes = [vp, vp, vp, vp]
     lib.cmoe_layer_update_bias.argtypes = [vp, C.c_float, vp, vp, vp]
     lib.cmoe_layer_dims.argtypes = [vp] + [C.POINTER(i32)] * 4
@@ -297,6 +301,38 @@ def select_shared(act_count, n_select: int, stream=None):
     _check(load().cmoe_select_shared(act_count.data_ptr(), act_count.shape[0], n_select, out.data_ptr(),
                                      _stream_ptr(stream)), "cmoe_select_shared")
     return out[:n_select]
+
+
+def cluster_update(act_bits, n_tokens: int, neuron_idx, assign, centroid_count, cluster_size, stream=None) -> None:
+    """cmoe_cluster_update on CUDA tensors (act_bits [d_ff, words] 32-bit, neuron_idx / assign int32 [n],
+    centroid_count int32 [n_clusters, n_tokens], cluster_size int32 [n_clusters]; both updated in place)."""
+    _check(load().cmoe_cluster_update(act_bits.data_ptr(), act_bits.shape[1], n_tokens, neuron_idx.data_ptr(),
+                                      assign.data_ptr(), neuron_idx.shape[0], centroid_count.shape[0],
+                                      centroid_count.data_ptr(), cluster_size.data_ptr(), _stream_ptr(stream)),
+           "cmoe_cluster_update")
+
+
+def cluster_distances(act_bits, n_tokens: int, neuron_idx, centroid_count, cluster_size, stream=None):
+    """cmoe_cluster_distances; returns the CUDA int64 tensor [n, n_clusters] of size_j^2 * d_ij^2."""
+    import torch
+    n, c = neuron_idx.shape[0], centroid_count.shape[0]
+    sqnorm = torch.empty(c, dtype=torch.int64, device=act_bits.device)
+    out = torch.empty((max(n, 1), c), dtype=torch.int64, device=act_bits.device)
+    _check(load().cmoe_cluster_distances(act_bits.data_ptr(), act_bits.shape[1], n_tokens, neuron_idx.data_ptr(), n,
+                                         centroid_count.data_ptr(), cluster_size.data_ptr(), c, sqnorm.data_ptr(),
+                                         out.data_ptr(), _stream_ptr(stream)), "cmoe_cluster_distances")
+    return out[:n]
+
+
+def cluster_representatives(scaled_sq_dist, neuron_idx, assign, stream=None):
+    """cmoe_cluster_representatives; returns a CUDA int32 tensor [n_clusters]."""
+    import torch
+    c = scaled_sq_dist.shape[1]
+    out = torch.empty(c, dtype=torch.int32, device=scaled_sq_dist.device)
+    _check(load().cmoe_cluster_representatives(scaled_sq_dist.data_ptr(), neuron_idx.data_ptr(), assign.data_ptr(),
+                                               neuron_idx.shape[0], c, out.data_ptr(), _stream_ptr(stream)),
+           "cmoe_cluster_representatives")
+    return out
 
 
 STATIC_PERMUTE_MAX_CELLS = 262144

@@ -14,6 +14,7 @@
 #include <vector>
 
 #include "balance.cuh"
+#include "cluster.cuh"
 #include "combine.cuh"
 #include "common.cuh"
 #include "permute.cuh"
@@ -664,6 +665,63 @@ int cmoe_select_shared(const int32_t* act_count, int32_t d_ff, int32_t n_select,
   if (!act_count || !shared_idx) return arg_fail(CMOE_ERR_INVALID_ARG, "null act_count / shared_idx");
   select_shared_kernel<<<(d_ff + 31) / 32, 256, 0, static_cast<cudaStream_t>(stream)>>>(act_count, d_ff, n_select,
                                                                                          shared_idx);
+  CU_TRY(cudaGetLastError());
+  return CMOE_OK;
+}
+
+namespace {
+int check_cluster_args(const uint32_t* act_bits, int32_t words, int32_t q, const int32_t* neuron_idx, int32_t n,
+                       int32_t n_clusters) {
+  if (words < 1 || q < 1 || (long long)words * 32 < q) return arg_fail(CMOE_ERR_INVALID_ARG, "words_per_neuron * 32 < n_tokens");
+  if (n < 0 || n_clusters < 1 || n_clusters > kClusterMax)
+    return arg_fail(CMOE_ERR_INVALID_ARG, "n < 0 or n_clusters outside [1, 32]");
+  if ((long long)q * (n > 0 ? n : 1) > 0x7fffffffLL) return arg_fail(CMOE_ERR_CAPACITY, "n_tokens * n exceeds 2^31 - 1");
+  if (!act_bits || (n > 0 && !neuron_idx)) return arg_fail(CMOE_ERR_INVALID_ARG, "null act_bits / neuron_idx");
+  return CMOE_OK;
+}
+}  // namespace
+
+int cmoe_cluster_update(const uint32_t* act_bits, int32_t words_per_neuron, int32_t n_tokens,
+                        const int32_t* neuron_idx, const int32_t* assign, int32_t n, int32_t n_clusters,
+                        int32_t* centroid_count, int32_t* cluster_size, void* stream) {
+  const int rc = check_cluster_args(act_bits, words_per_neuron, n_tokens, neuron_idx, n, n_clusters);
+  if (rc != CMOE_OK) return rc;
+  if (!centroid_count || !cluster_size || (n > 0 && !assign))
+    return arg_fail(CMOE_ERR_INVALID_ARG, "null assign / centroid_count / cluster_size");
+  cluster_update_kernel<<<n_clusters, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      act_bits, words_per_neuron, n_tokens, neuron_idx, assign, n, centroid_count, cluster_size);
+  CU_TRY(cudaGetLastError());
+  return CMOE_OK;
+}
+
+int cmoe_cluster_distances(const uint32_t* act_bits, int32_t words_per_neuron, int32_t n_tokens,
+                           const int32_t* neuron_idx, int32_t n, const int32_t* centroid_count,
+                           const int32_t* cluster_size, int32_t n_clusters, int64_t* centroid_sqnorm,
+                           int64_t* scaled_sq_dist, void* stream) {
+  const int rc = check_cluster_args(act_bits, words_per_neuron, n_tokens, neuron_idx, n, n_clusters);
+  if (rc != CMOE_OK) return rc;
+  if (!centroid_count || !cluster_size || !centroid_sqnorm || (n > 0 && !scaled_sq_dist))
+    return arg_fail(CMOE_ERR_INVALID_ARG, "null centroid_count / cluster_size / centroid_sqnorm / scaled_sq_dist");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  static_assert(sizeof(long long) == sizeof(int64_t), "int64_t is long long here");
+  centroid_norm_kernel<<<n_clusters, 256, 0, st>>>(centroid_count, n_tokens, reinterpret_cast<long long*>(centroid_sqnorm));
+  if (n > 0)
+    cluster_distance_kernel<<<(n + 7) / 8, 256, 0, st>>>(act_bits, words_per_neuron, n_tokens, neuron_idx, n,
+                                                        centroid_count, cluster_size,
+                                                        reinterpret_cast<const long long*>(centroid_sqnorm), n_clusters,
+                                                        reinterpret_cast<long long*>(scaled_sq_dist));
+  CU_TRY(cudaGetLastError());
+  return CMOE_OK;
+}
+
+int cmoe_cluster_representatives(const int64_t* scaled_sq_dist, const int32_t* neuron_idx, const int32_t* assign,
+                                 int32_t n, int32_t n_clusters, int32_t* rep_neuron, void* stream) {
+  if (n < 0 || n_clusters < 1 || n_clusters > kClusterMax)
+    return arg_fail(CMOE_ERR_INVALID_ARG, "n < 0 or n_clusters outside [1, 32]");
+  if (!rep_neuron || (n > 0 && (!scaled_sq_dist || !neuron_idx || !assign)))
+    return arg_fail(CMOE_ERR_INVALID_ARG, "null scaled_sq_dist / neuron_idx / assign / rep_neuron");
+  cluster_representative_kernel<<<n_clusters, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      reinterpret_cast<const long long*>(scaled_sq_dist), neuron_idx, assign, n, n_clusters, rep_neuron);
   CU_TRY(cudaGetLastError());
   return CMOE_OK;
 }
