@@ -473,6 +473,92 @@ def run_profile(args):
     return line if rank == 0 else None
 
 
+# ----------------------------------------------------- clustering-round stage
+def run_cluster(args):
+    """One round of the data-parallel clustering pieces (centroid update, distance matrix,
+    representatives) at the paper's scale: 16384 calibration tokens, K_a = 10, the workload's d_h,
+    N_r clusters of m neurons.  The activation matrix and the balanced assignment are synthetic
+    inputs (the assignment solver is a sequential CPU algorithm and not part of the step)."""
+    import numpy as np
+    import torch
+    from paper_2502_04416_b200 import binding
+
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if int(os.environ.get("RANK", "0")) != 0:
+        return None
+    torch.cuda.set_device(local)
+    binding.load()
+    w = wl.WORKLOADS[args.workload]
+    s = w.shape
+    q, k_a, m, n_r = args.tokens or 16384, 10, s.d_ff // s.n_experts, s.n_routed
+    rng = np.random.Generator(np.random.PCG64(4321))
+    # K_a active neurons per token, popularity skewed as in the paper's rate histogram
+    pop = np.exp(rng.normal(scale=1.0, size=s.d_ff))
+    picks = np.stack([rng.choice(s.d_ff, size=k_a, replace=False, p=pop / pop.sum()) for _ in range(q)])
+    words = (q + 31) // 32
+    bits_host = np.zeros((s.d_ff, words), dtype=np.uint32)
+    t = np.repeat(np.arange(q), k_a)
+    np.bitwise_or.at(bits_host, (picks.ravel(), t // 32), (np.uint32(1) << (t % 32).astype(np.uint32)))
+    counts = np.bincount(picks.ravel(), minlength=s.d_ff)
+    order = np.argsort(-counts, kind="stable")
+    rest = np.sort(order[s.n_shared * m:]).astype(np.int32)          # the N_r * m neurons to cluster
+    assign_host = rng.permutation(np.repeat(np.arange(n_r), m)).astype(np.int32)
+    bits = torch.from_numpy(bits_host.view(np.int32)).cuda()
+    rest_d, assign_d = torch.from_numpy(rest).cuda(), torch.from_numpy(assign_host).cuda()
+    count = torch.zeros((n_r, q), dtype=torch.int32, device="cuda")
+    size = torch.ones(n_r, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        binding.cluster_update(bits, q, rest_d, assign_d, count, size)
+        sd = binding.cluster_distances(bits, q, rest_d, count, size)
+        return binding.cluster_representatives(sd, rest_d, assign_d)
+
+    steps = min(args.steps, 200)
+    sampler = ClockSampler(local)
+    sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler.wait_first()
+    sampler.mark_begin()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    sampler.mark_end()
+    time.sleep(0.12)
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / steps
+    n = len(rest)
+    peaks = load_peaks()
+    alg_bytes = 2.0 * n * words * 4 + 3.0 * n_r * q * 4 + n * n_r * 8     # bit rows twice, counts written/read, D written
+    line = {
+        "metric": "cluster_round_neurons_per_s", "value": n / (ms * 1e-3), "unit": "neurons/s", "n_gpus": 1,
+        "steps": steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "config": {"workload": f"{w.name} clustering round q={q} K_a={k_a}", "neurons": n, "clusters": n_r,
+                   "l2": "inputs (19 MB) fit the 126 MB L2: a latency-bound step"},
+        "gpu_launches": 5 * steps, "clocks": clocks,
+        "roofline": {"bound": "hbm", "achieved": alg_bytes / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": alg_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                     "kernel": "centroid update + distance matrix + representatives", "peak_source": peaks["source"]},
+    }
+    from oracle import cmoe_oracle as oracle
+    sample_q, sample_n = min(q, 512), min(n, 1024)
+    a = ((bits_host[rest[:sample_n]][:, np.arange(sample_q) // 32] >> (np.arange(sample_q) % 32).astype(np.uint32)) & 1).T
+    sub = np.minimum(assign_host[:sample_n], n_r - 1)
+    t0 = time.perf_counter()
+    cent = oracle.cluster_update(a, sub, np.zeros((sample_q, n_r)))
+    oracle.representatives(a, sub, cent)
+    dt = time.perf_counter() - t0
+    line["cpu_baseline"] = {"value": sample_n / dt, "unit": "neurons/s", "cores": host_threads(), "kind": "oracle",
+                            "sample": f"{sample_n} neurons x {sample_q} tokens, one round, {dt:.2f} s"}
+    return line
+
+
 def run_reference(args):
     """The CPU oracle, unmodified, timed on the host cores on a bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
@@ -518,8 +604,9 @@ def main():
                     help="replay the forward from a CUDA graph (auto: batches of at most 512 tokens)")
     ap.add_argument("--chain", choices=["on", "off"], default="on",
                     help="programmatic dependent launches between the kernels of a forward (library default: on)")
-    ap.add_argument("--stage", choices=["forward", "profile"], default="forward",
-                    help="forward: the MoE forward pass (the headline metric); profile: the activation-profiling pass")
+    ap.add_argument("--stage", choices=["forward", "profile", "cluster"], default="forward",
+                    help="forward: the MoE forward pass (the headline metric); profile: the activation-profiling "
+                         "pass; cluster: one round of the GPU clustering pieces")
     ap.add_argument("--forward-only", action="store_true",
                     help="run only the timed forward passes (for profiler captures)")
     args = ap.parse_args()
@@ -527,7 +614,8 @@ def main():
         line = run_reference(args)
     else:
         args.warmup = max(args.warmup, 3)
-        line = run_profile(args) if args.stage == "profile" else run_gpu(args)
+        line = (run_profile(args) if args.stage == "profile" else
+                run_cluster(args) if args.stage == "cluster" else run_gpu(args))
     if line is not None:
         print(json.dumps(line))
 

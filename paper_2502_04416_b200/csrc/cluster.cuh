@@ -16,12 +16,12 @@ namespace cmoe {
 
 constexpr int kClusterMax = 32;      // clusters per call (N_r of one layer)
 
-// One block per cluster j: count the members (rows i with assign[i] == j); a cluster without
-// members keeps its centroid; otherwise the count vector is rebuilt from the members' bits.
+// Centroid update, first half.  One block per cluster j: count the members (rows i with
+// assign[i] == j); a cluster without members keeps its centroid, otherwise its size is set and
+// its count vector cleared for the second half.
 __global__ void __launch_bounds__(256)
-cluster_update_kernel(const uint32_t* __restrict__ act_bits, int words, int q, const int32_t* __restrict__ neuron_idx,
-                      const int32_t* __restrict__ assign, int n, int32_t* __restrict__ centroid_count,
-                      int32_t* __restrict__ cluster_size) {
+cluster_reset_kernel(const int32_t* __restrict__ assign, int n, int q, int32_t* __restrict__ centroid_count,
+                     int32_t* __restrict__ cluster_size) {
   __shared__ int red[8];
   __shared__ int sh_members;
   const int j = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -42,19 +42,28 @@ cluster_update_kernel(const uint32_t* __restrict__ act_bits, int words, int q, c
   int32_t* cc = centroid_count + (size_t)j * q;
   for (int k = tid; k < q; k += 256) cc[k] = 0;
   if (tid == 0) cluster_size[j] = members;
-  __syncthreads();
-  // a warp per member row, lanes over its words; the set bits are few (K_a per token overall)
-  for (int i = warp; i < n; i += 8) {
-    if (assign[i] != j) continue;
-    const uint32_t* row = act_bits + (size_t)neuron_idx[i] * words;
-    for (int w = lane; w < words; w += 32) {
-      uint32_t bits = row[w];
-      while (bits) {
-        const int b = __ffs(bits) - 1;
-        bits &= bits - 1;
-        const int k = 32 * w + b;
-        if (k < q) atomicAdd(cc + k, 1);
-      }
+}
+
+// Centroid update, second half.  One warp per listed neuron with a cluster: lanes walk its
+// words and add 1 to the cluster's count for every set bit (few: K_a per token over all neurons).
+__global__ void __launch_bounds__(256)
+cluster_accumulate_kernel(const uint32_t* __restrict__ act_bits, int words, int q,
+                          const int32_t* __restrict__ neuron_idx, const int32_t* __restrict__ assign, int n,
+                          int n_clusters, int32_t* __restrict__ centroid_count) {
+  const int lane = threadIdx.x & 31;
+  const int i = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (i >= n) return;
+  const int j = assign[i];
+  if (j < 0 || j >= n_clusters) return;
+  const uint32_t* row = act_bits + (size_t)neuron_idx[i] * words;
+  int32_t* cc = centroid_count + (size_t)j * q;
+  for (int w = lane; w < words; w += 32) {
+    uint32_t bits = row[w];
+    while (bits) {
+      const int b = __ffs(bits) - 1;
+      bits &= bits - 1;
+      const int k = 32 * w + b;
+      if (k < q) atomicAdd(cc + k, 1);
     }
   }
 }

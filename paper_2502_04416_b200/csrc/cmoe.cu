@@ -688,8 +688,11 @@ int cmoe_cluster_update(const uint32_t* act_bits, int32_t words_per_neuron, int3
   if (rc != CMOE_OK) return rc;
   if (!centroid_count || !cluster_size || (n > 0 && !assign))
     return arg_fail(CMOE_ERR_INVALID_ARG, "null assign / centroid_count / cluster_size");
-  cluster_update_kernel<<<n_clusters, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-      act_bits, words_per_neuron, n_tokens, neuron_idx, assign, n, centroid_count, cluster_size);
+  if (n == 0) return CMOE_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cluster_reset_kernel<<<n_clusters, 256, 0, st>>>(assign, n, n_tokens, centroid_count, cluster_size);
+  cluster_accumulate_kernel<<<(n + 7) / 8, 256, 0, st>>>(act_bits, words_per_neuron, n_tokens, neuron_idx, assign, n,
+                                                        n_clusters, centroid_count);
   CU_TRY(cudaGetLastError());
   return CMOE_OK;
 }
