@@ -190,6 +190,50 @@ permute_scatter_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k
   chunk_scatter(topk_idx, n_rows, n_k, n_groups, row, base, warp_cnt, row_token, row_of);
 }
 
+// Scan and scatter in one launch, for count matrices small enough to be re-read by every block
+// (n_chunks * n_groups <= kPermFusedCells): block c adds up, per group, the counts of the chunks
+// before it and of all chunks, scans the group totals itself and places its chunk; block 0 also
+// publishes counts, offsets and the groups' row ranges.  The same integers as the three-kernel
+// form, one launch fewer.
+constexpr int kPermFusedCells = 16384;
+
+__global__ void __launch_bounds__(kPermChunk)
+permute_scan_scatter_kernel(const int32_t* __restrict__ topk_idx, int n_rows, int n_k, int n_groups, int n_chunks,
+                            const int32_t* __restrict__ chunk_cnt, int32_t* __restrict__ counts,
+                            int32_t* __restrict__ offsets, int32_t* __restrict__ row_token,
+                            int32_t* __restrict__ row_of, const GroupPlanOut po) {
+  grid_dep_wait();
+  grid_dep_trigger();
+  extern __shared__ int32_t sm[];
+  int32_t* total = sm;                         // [n_groups]
+  int32_t* offs = total + n_groups;            // [n_groups + 1]
+  int32_t* base = offs + n_groups + 1;         // [n_groups]
+  int32_t* sums = base + n_groups;             // [kPermChunk]
+  int32_t* warp_cnt = sums + kPermChunk;       // [8][n_groups]
+  const int c = blockIdx.x;
+  for (int g = threadIdx.x; g < n_groups; g += blockDim.x) {
+    int before = 0, all = 0;
+    for (int cc = 0; cc < n_chunks; ++cc) {
+      const int v = __ldg(chunk_cnt + (size_t)cc * n_groups + g);
+      before += cc < c ? v : 0;
+      all += v;
+    }
+    total[g] = all;
+    base[g] = before;
+  }
+  __syncthreads();
+  block_scan_groups(total, offs, n_groups, sums);
+  for (int g = threadIdx.x; g < n_groups; g += blockDim.x) base[g] += offs[g];
+  if (c == 0) {
+    for (int g = threadIdx.x; g < n_groups; g += blockDim.x) { counts[g] = total[g]; offsets[g] = offs[g]; }
+    if (threadIdx.x == 0) offsets[n_groups] = offs[n_groups];
+    write_group_rows(po, n_groups, total, offs);
+  }
+  __syncthreads();
+  const int row = c * kPermChunk + threadIdx.x;
+  chunk_scatter(topk_idx, n_rows, n_k, n_groups, row, base, warp_cnt, row_token, row_of);
+}
+
 inline int64_t permute_scratch_bytes(int n_rows, int n_groups) {
   const int64_t n_chunks = (n_rows + kPermChunk - 1) / kPermChunk;
   const int64_t b = n_chunks * n_groups * (int64_t)sizeof(int32_t);
@@ -210,6 +254,12 @@ inline int launch_token_permute(const int32_t* topk_idx, int n_rows, int n_k, in
   const int n_chunks = (n_rows + kPermChunk - 1) / kPermChunk;
   launch_kernel(dep, permute_count_kernel, dim3(n_chunks), dim3(kPermChunk), n_groups * sizeof(int32_t), stream,
                 topk_idx, n_rows, n_k, n_groups, scratch);
+  if ((long long)n_chunks * n_groups <= kPermFusedCells && n_groups <= 1024) {
+    const size_t smem = (size_t)(n_groups * 3 + 1 + kPermChunk + 8 * n_groups) * sizeof(int32_t);
+    launch_kernel(dep, permute_scan_scatter_kernel, dim3(n_chunks), dim3(kPermChunk), smem, stream, topk_idx, n_rows,
+                  n_k, n_groups, n_chunks, (const int32_t*)scratch, counts, offsets, row_token, row_of, po);
+    return 2;
+  }
   launch_kernel(dep, permute_scan_kernel, dim3(1), dim3(1024), 0, stream, scratch, n_chunks, n_groups, counts,
                 offsets, po);
   launch_kernel(dep, permute_scatter_kernel, dim3(n_chunks), dim3(kPermChunk), 9 * n_groups * sizeof(int32_t), stream,
