@@ -107,6 +107,8 @@ struct cmoe_layer {
   Umma2Plan pair;
   float* rsk_part = nullptr;    // split-K router partial sums [slices][64 rows][64]
   int32_t* rsk_ticket = nullptr;
+  float* rt_part = nullptr;     // tcgen05 router: K-slice partial sums and tickets
+  int32_t* rt_ticket = nullptr;
   float* dec_part = nullptr;    // decode GEMMs: K-slice partial sums, tickets per (tile, epilogue warp)
   int32_t* dec_ticket = nullptr;
   float *share = nullptr, *target = nullptr;   // utilisation of the last step / bias-update targets
@@ -232,6 +234,10 @@ void carve_workspace(cmoe_layer* L, char* base) {
     L->dec_ticket = a.take<int32_t>(4 * (t1 > t2 ? t1 : t2));
     L->dec_part = a.take<float>((size_t)kDecMaxSlots * kDecSlotFloats);
   }
+  if (esz == 2 && nr > 0) {
+    L->rt_ticket = a.take<int32_t>(4 * 256);
+    L->rt_part = a.take<float>((size_t)256 * 64 * 128);
+  }
   L->ws_bytes = align_up(a.used + 256, 256);
 }
 
@@ -280,6 +286,7 @@ int finish_layer(cmoe_layer* L, cudaStream_t st) {
     L->umma_ok = (rc == CMOE_OK);
     if (L->umma_ok && !decode_plan_create(&L->umma, &L->decode)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     L->decode.part = L->dec_part; L->decode.ticket = L->dec_ticket;
+    L->umma.rt_part = L->rt_part; L->umma.rt_ticket = L->rt_ticket;
     if (L->umma_ok && !umma2_plan_create(&L->umma, &L->pair)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   }
   CU_TRY(cudaStreamSynchronize(st));

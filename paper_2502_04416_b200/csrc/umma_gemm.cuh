@@ -187,6 +187,9 @@ struct UmmaArgs {
   const bf16* x_rows_ptr;     // mode 1: the outer rows of x (source of the cp.async gather)
   int32_t* err;
   // mode 3 (router)
+  int ksplit;                 // K slices per tile (>= 1): a tile's k range is cut so that more SMs take part
+  float* rt_part;             // ksplit > 1: [unit][2 n_rp columns][128 rows] fp32 partial sums
+  int32_t* rt_ticket;         // ksplit > 1: [tile][4 epilogue warps], zero between launches
   const int32_t* outer_off;   // row ranges of the outer experts, or null (one range [0, n_rows))
   int n_rows, n_rp, n_k;      // n_rp: N_r rounded up to 8 (rows per block of the padded W^R)
   const float* u;
@@ -340,13 +343,16 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int total_tiles = tile_start[n_groups];
+  const int ksplit = MODE == 3 ? max(p.ksplit, 1) : 1;
+  const int total_units = total_tiles * ksplit;
   const int k_blocks_fixed = (p.d + kUmmaBK - 1) / kUmmaBK;      // modes 1 and 3: K = d
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (whole warp)
     uint32_t it = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+    for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+      const int t = u / ksplit, kz = u - t * ksplit;
       const TileCoord c = umma_decode<MODE>(p, tile_start, n_groups, t);
       GroupStatic g;
       if (MODE != 3) g = p.gs[c.g]; else { g.is_shared = 1; g.outer = c.g; g.width = 0; g.w_row0 = 0; }
@@ -382,7 +388,8 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
         k_blocks = k_blocks_fixed;
         b_bytes = 2 * p.n_rp * kUmmaBK * 2;
       }
-      for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+      const int kb_lo = kz * k_blocks / ksplit, kb_hi = (kz + 1) * k_blocks / ksplit;      // this unit's k slice
+      for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
         const uint32_t s = it % kStages, n = it / kStages;
         if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
         const uint32_t fb = full0 + 8 * s;
@@ -408,7 +415,8 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
     if (lane == 0) {
       uint32_t it = 0, tile_n = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_n) {
+      for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++tile_n) {
+        const int t = u / ksplit, kz = u - t * ksplit;
         const TileCoord c = umma_decode<MODE>(p, tile_start, n_groups, t);
         int k_blocks, n_mma;
         if (MODE == 1) {
@@ -424,7 +432,8 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
         if (!mbar_wait(acce0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.err, kErrWaitAccEmpty)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * 256;
-        for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+        const int kb_lo = kz * k_blocks / ksplit, kb_hi = (kz + 1) * k_blocks / ksplit;
+        for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
           const uint32_t s = it % kStages, n = it / kStages;
           if (!mbar_wait(full0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
           if (MODE == 1) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // cp.async-written rows
@@ -433,7 +442,7 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
 #pragma unroll
           for (int k = 0; k < kUmmaBK / 16; ++k)
             umma_bf16(d_tmem, umma_smem_desc(sa + k * 32), umma_smem_desc(sb + k * 32), idesc,
-                      (kb | k) != 0 ? 1u : 0u);
+                      (kb != kb_lo || k != 0) ? 1u : 0u);
           umma_commit(empty0 + 8 * s);         // stage reusable once these MMAs have read it
         }
         if (ok) umma_commit(accf0 + 8 * buf);  // accumulator complete
@@ -490,7 +499,8 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
     const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
     uint32_t tile_n = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_n) {
+    for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++tile_n) {
+      const int t = u / ksplit, kz = u - t * ksplit;
       const TileCoord c = umma_decode<MODE>(p, tile_start, n_groups, t);
       const uint32_t buf = tile_n & 1, use = tile_n >> 1;
       if (!mbar_wait(accf0 + 8 * buf, use & 1, abort_flag, p.err, kErrWaitAccFull)) { ok = false; break; }
@@ -563,7 +573,42 @@ umma_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_con
           tmem_ld16(taddr + p.n_rp + 16, v + 16);
         }
         tmem_ld_wait();
-        if (row_ok) {
+        bool finish_row = true;
+        if (ksplit > 1) {
+          // K slice of a split tile: park this row's partial sums ([column][row]: a warp's store is one
+          // 128-byte line), take the warp's ticket for the tile; the warp that takes the last one adds
+          // the slices in ascending order (a fixed order: deterministic) and goes on to the gate logic
+          const int row128 = quad * 32 + lane;
+          float* mine = p.rt_part + ((size_t)t * ksplit + kz) * (64 * 128) + row128;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            if (j < p.n_rp) { __stcg(mine + (size_t)j * 128, a[j]); __stcg(mine + (size_t)(32 + j) * 128, v[j]); }
+          }
+          __threadfence();
+          __syncwarp();
+          int32_t* tk = p.rt_ticket + (size_t)t * 4 + quad;
+          int last = 0;
+          if (lane == 0) last = atomicAdd(tk, 1) == ksplit - 1;
+          last = __shfl_sync(0xffffffffu, last, 0);
+          finish_row = last != 0;
+          if (finish_row) {
+            __threadfence();
+            const float* all = p.rt_part + (size_t)t * ksplit * (64 * 128) + row128;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) { a[j] = 0.0f; v[j] = 0.0f; }
+            for (int z = 0; z < ksplit; ++z) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                if (j < p.n_rp) {
+                  a[j] += __ldcg(all + (size_t)z * (64 * 128) + (size_t)j * 128);
+                  v[j] += __ldcg(all + (size_t)z * (64 * 128) + (size_t)(32 + j) * 128);
+                }
+              }
+            }
+            if (lane == 0) *tk = 0;            // ready for the next launch
+          }
+        }
+        if (row_ok && finish_row) {
           const size_t row = (size_t)(c.row0 + row_in_group);
           router_row_epilogue(a, v, p.n_r, p.n_k, p.u + c.g * p.n_r, p.b + c.g * p.n_r, c.g * p.n_r,
                               p.scores + row * p.n_r, p.keys + row * p.n_r, p.topk_idx + row * p.n_k,
@@ -614,6 +659,8 @@ struct UmmaPlan {
   UmmaShape shape;
   UmmaBuffers buf;
   int bn_s = 128, bn_r = 128, n_sms = 0, n_groups = 0;
+  float* rt_part = nullptr;                // router K-slice partials: n_sms units x 64 columns x 128 rows (caller's workspace)
+  int32_t* rt_ticket = nullptr;            // [n_sms][4], zeroed once
   bool has_s = false, has_r = false;
   PFN_encodeTiled encode = nullptr;
   CUtensorMap x_rows, x_gather;            // x: 64 x 128 boxes for consecutive rows, 64 x 1 for gather4
@@ -764,8 +811,19 @@ inline int umma_router_forward(UmmaPlan* P, int n_rows, const int32_t* outer_off
                                cudaStream_t st) {
   UmmaArgs a = umma_base_args(P, nullptr, err_word);
   a.outer_off = outer_off; a.n_rows = n_rows;
-  const int tiles = (n_rows + kUmmaBM - 1) / kUmmaBM + P->shape.n_outer;
-  const int grid = tiles < P->n_sms ? tiles : P->n_sms;
+  const int tiles = (n_rows + kUmmaBM - 1) / kUmmaBM + P->shape.n_outer;     // upper bound of the tile count
+  // with few tiles, cut each tile's K range so that up to four times as many SMs stream x
+  int ksplit = 1;
+  if (P->rt_part && P->rt_ticket) {
+    const int kb = (P->shape.d + kUmmaBK - 1) / kUmmaBK;
+    ksplit = P->n_sms / tiles;
+    if (ksplit > 4) ksplit = 4;
+    if (ksplit > kb / 8) ksplit = kb / 8;
+    if (ksplit < 1) ksplit = 1;
+  }
+  a.ksplit = ksplit; a.rt_part = P->rt_part; a.rt_ticket = P->rt_ticket;
+  const int units = tiles * ksplit;
+  const int grid = units < P->n_sms ? units : P->n_sms;
   umma_grouped_kernel<3><<<grid, kUmmaThreads, kUmmaSmemBytes, st>>>(P->x_rows, P->x_rows, P->w_rep, P->w_rep, a);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
