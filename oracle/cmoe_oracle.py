@@ -25,7 +25,9 @@ clustering pieces (Appendix "Balanced Clustering Algorithm"): squared L2 = Hammi
 on binary vectors, a hand-worked mean, brute-force argmin, an exhaustive balanced assignment.
 Parity unpinned (conventions the paper does not fix): the outer router's
 weights for an existing MoE layer (softmax over the selected logits), the
-tie-break between equal keys (lower index wins) and the NaN policy.
+tie-break between equal keys (lower index wins) and the NaN policy; likewise the
+tie-breaks of equal magnitudes in ATopK, of equal activation counts and of equal
+centroid distances (lower index or position wins).
 """
 from __future__ import annotations
 
