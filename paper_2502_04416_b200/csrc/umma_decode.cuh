@@ -63,6 +63,7 @@ struct DecodeArgs {
   int32_t* err;
   float* part;           // [kDecMaxSlots][kDecSlotFloats] slice partials
   int32_t* ticket;       // [tiles][4 epilogue warps], zero between launches
+  int tok_box_rows;      // rows of the token-tile TMA box (16, 32 or 64): no more than the batch needs
 };
 
 // Tile handled by CTA `cta` in its `round`-th turn: even rounds run left to right, odd
@@ -224,7 +225,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         const uint32_t fb = full0 + 8 * s;
         const uint32_t sw = base + s * kStageBytes, sx = sw + kWBytes;
         if (lane == 0) {
-          mbar_expect_tx(fb, kWBytes + kDecXBytes);
+          mbar_expect_tx(fb, kWBytes + p.tok_box_rows * kUmmaBK * 2);
           if (MODE == 4) tma_load_3d(sw, tw, fb, kb * kUmmaBK, g.w_row0 + nt * 128, 0);
           else if (g.is_shared) tma_load_3d(sw, tw, fb, kb * kUmmaBK, nt * 128, g.outer);
           else tma_load_4d(sw, tw, fb, kb * kUmmaBK, nt * 128, j, g.outer);
@@ -382,8 +383,10 @@ struct DecodePlan {
   int32_t* ticket = nullptr;        // zeroed once; the kernels leave it zero
   CUtensorMap w_gu;                 // stacked gate/up rows, box 64 k x 128 rows x 2 planes
   CUtensorMap wd_s, wd_r;           // W_down blocks, 128-channel boxes
-  CUtensorMap x_rows64;             // x, 64-row boxes (bound per forward for a plain layer)
-  CUtensorMap h_s, h_r;             // H, 64-row boxes
+  // token tiles come in boxes of 16, 32 or 64 rows (index 0..2): a launch uses the smallest that holds
+  // its rows, so that a stage carries as little besides weights as possible
+  CUtensorMap x_rows[3];            // x (bound per forward for a plain layer)
+  CUtensorMap h_s[3], h_r[3];       // H
 };
 
 inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
@@ -402,7 +405,9 @@ inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
     const cuuint64_t str[2] = {(cuuint64_t)s.shared_width * 2, d * s.d_ff * 2};
     const cuuint32_t box[3] = {kUmmaBK, 128, 1};
     ok = umma_encode(P, &D->wd_s, buf.w_down, 3, dims, str, box, "shared W_down (decode)") &&
-         umma_encode_rows(P, &D->h_s, buf.h_s, s.max_outer_rows, s.shared_width, kDecMaxRows, "H shared (decode)");
+         umma_encode_rows(P, &D->h_s[0], buf.h_s, s.max_outer_rows, s.shared_width, 16, "H shared (decode)") &&
+         umma_encode_rows(P, &D->h_s[1], buf.h_s, s.max_outer_rows, s.shared_width, 32, "H shared (decode)") &&
+         umma_encode_rows(P, &D->h_s[2], buf.h_s, s.max_outer_rows, s.shared_width, 64, "H shared (decode)");
   }
   if (ok && P->has_r) {
     const cuuint64_t dims[4] = {(cuuint64_t)s.m, d, (cuuint64_t)s.n_r, (cuuint64_t)s.n_outer};
@@ -410,13 +415,19 @@ inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
     const cuuint32_t box[4] = {kUmmaBK, 128, 1, 1};
     ok = umma_encode(P, &D->wd_r, (const bf16*)buf.w_down + (size_t)s.shared_width * d, 4, dims, str, box,
                      "routed W_down (decode)") &&
-         umma_encode_rows(P, &D->h_r, buf.h_r, s.max_routed_rows, s.m, kDecMaxRows, "H routed (decode)");
+         umma_encode_rows(P, &D->h_r[0], buf.h_r, s.max_routed_rows, s.m, 16, "H routed (decode)") &&
+         umma_encode_rows(P, &D->h_r[1], buf.h_r, s.max_routed_rows, s.m, 32, "H routed (decode)") &&
+         umma_encode_rows(P, &D->h_r[2], buf.h_r, s.max_routed_rows, s.m, 64, "H routed (decode)");
   }
   if (ok && buf.x_fixed)
-    ok = umma_encode_rows(P, &D->x_rows64, buf.x_fixed, s.max_outer_rows, d, kDecMaxRows, "outer rows of x (decode)");
+    ok = umma_encode_rows(P, &D->x_rows[0], buf.x_fixed, s.max_outer_rows, d, 16, "outer rows of x (decode)") &&
+         umma_encode_rows(P, &D->x_rows[1], buf.x_fixed, s.max_outer_rows, d, 32, "outer rows of x (decode)") &&
+         umma_encode_rows(P, &D->x_rows[2], buf.x_fixed, s.max_outer_rows, d, 64, "outer rows of x (decode)");
   if (!ok) return false;
-  if (!P->has_r) { D->wd_r = D->wd_s; D->h_r = D->h_s; }
-  if (!P->has_s) { D->wd_s = D->wd_r; D->h_s = D->h_r; }
+  for (int i = 0; i < 3; ++i) {
+    if (!P->has_r) { D->wd_r = D->wd_s; D->h_r[i] = D->h_s[i]; }
+    if (!P->has_s) { D->wd_s = D->wd_r; D->h_s[i] = D->h_r[i]; }
+  }
   cudaError_t e = cudaFuncSetAttribute(umma_decode_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        decode_smem_bytes<4>());
   if (e == cudaSuccess)
@@ -436,9 +447,13 @@ inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
   return true;
 }
 
+// Index of the smallest token box (16 << index rows) that holds n_rows rows.
+inline int decode_box_index(int n_rows) { return n_rows <= 16 ? 0 : (n_rows <= 32 ? 1 : 2); }
+
 inline bool decode_bind_x(UmmaPlan* P, DecodePlan* D, const void* x_rows, int n_rows) {
   if (P->buf.x_fixed) return true;
-  return umma_encode_rows(P, &D->x_rows64, x_rows, (size_t)n_rows, (size_t)P->shape.d, kDecMaxRows, "x (decode)");
+  const int bi = decode_box_index(n_rows);
+  return umma_encode_rows(P, &D->x_rows[bi], x_rows, (size_t)n_rows, (size_t)P->shape.d, 16 << bi, "x (decode)");
 }
 
 // Both decode GEMMs; requires umma_bind_x and decode_bind_x for this forward and n_rows <=
@@ -465,14 +480,16 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n
   a.gs = P->buf.gs_dev; a.gr = gr; a.n_groups = P->n_groups; a.n_outer = s.n_outer; a.n_r = s.n_r;
   a.d = s.d; a.row_token = P->buf.row_token; a.err = err_word;
   a.part = D->part; a.ticket = D->ticket;
+  const int bi = decode_box_index(n_rows);
+  a.tok_box_rows = 16 << bi;
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
   launch_kernel(dep, split1 ? umma_decode_kernel<4, true> : umma_decode_kernel<4, false>, dim3(P->n_sms),
-                dim3(kUmmaThreads), decode_smem_bytes<4>(), st, D->w_gu, D->w_gu, D->x_rows64, D->x_rows64, a);
+                dim3(kUmmaThreads), decode_smem_bytes<4>(), st, D->w_gu, D->w_gu, D->x_rows[bi], D->x_rows[bi], a);
   if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
   if (!gate_up_only)
     launch_kernel(dep, split2 ? umma_decode_kernel<5, true> : umma_decode_kernel<5, false>, dim3(P->n_sms),
-                  dim3(kUmmaThreads), decode_smem_bytes<5>(), st, D->wd_s, D->wd_r, D->h_s, D->h_r, a);
+                  dim3(kUmmaThreads), decode_smem_bytes<5>(), st, D->wd_s, D->wd_r, D->h_s[bi], D->h_r[bi], a);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
     snprintf(P->error, sizeof(P->error), "decode GEMM launch: %s", cudaGetErrorString(e));
