@@ -369,7 +369,9 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
           return arg_fail(CMOE_ERR_CUDA, L->umma.error);
       } else if (R <= kRskMaxRows && d <= kRskMaxSlices * kRskSliceK) {
         perm_fused = G <= kRskFuseGroups;
-        router_splitk_kernel<<<(d + kRskSliceK - 1) / kRskSliceK, kRskThreads, 0, st>>>(
+        const bool sub8 = n_r <= 8 && R > 16;
+        (sub8 ? router_splitk_kernel<true> : router_splitk_kernel<false>)
+            <<<(d + kRskSliceK - 1) / kRskSliceK, kRskThreads, 0, st>>>(
             xo, R, d, n_r, L->n_rp, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->rsk_part,
             L->rsk_ticket, L->scores, L->keys, L->topk_idx, L->topk_gate, perm_fused ? 1 : 0, G, L->counts,
             L->offsets, L->row_token, L->row_of, po);

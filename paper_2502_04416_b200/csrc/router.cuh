@@ -53,6 +53,47 @@ __device__ __forceinline__ void gate_row(int lane, int n_r, int n_k, float a, fl
   }
 }
 
+// The same gate logic with W lanes per row (W = 8, 16 or 32 >= n_r): a warp handles 32 / W rows at
+// once.  `sub` is the lane's position in its W-lane group; every lane of the warp must call it (the
+// shuffles name the full warp), `live_row` = false for groups that hold no row.  The arithmetic and
+// its order per row are those of gate_row with the idle lanes removed, so the results are the same bits.
+template <int W>
+__device__ __forceinline__ void gate_row_sub(int sub, bool live_row, int n_r, int n_k, float a, float v,
+                                             const float* __restrict__ u, const float* __restrict__ b,
+                                             int group_base, float* __restrict__ scores_row,
+                                             float* __restrict__ keys_row, int32_t* __restrict__ idx_row,
+                                             float* __restrict__ gates_row) {
+  const bool live = live_row && sub < n_r;
+  const float s = live ? silu_accurate(a) * v : -INFINITY;
+  float s_max = s;
+#pragma unroll
+  for (int o = W / 2; o > 0; o >>= 1) s_max = fmaxf(s_max, __shfl_xor_sync(0xffffffffu, s_max, o));
+  const float e = live ? expf(s - s_max) : 0.0f;
+  float e_sum = e;
+#pragma unroll
+  for (int o = W / 2; o > 0; o >>= 1) e_sum += __shfl_xor_sync(0xffffffffu, e_sum, o);
+  const float s_prime = e / e_sum;
+  const float key = live ? s_prime + __ldg(b + sub) : -INFINITY;
+  if (live) { scores_row[sub] = s; keys_row[sub] = key; }
+  const float gate = live ? 1.0f + s_prime * __ldg(u + sub) : 0.0f;
+  const float rank_key = (key != key) ? -INFINITY : key;
+  const int lane = threadIdx.x & 31, group0 = lane - sub;
+  bool taken = !live;
+  for (int i = 0; i < n_k; ++i) {
+    float best = taken ? -INFINITY : rank_key;
+    int who = taken ? 64 + sub : sub;
+#pragma unroll
+    for (int o = W / 2; o > 0; o >>= 1) {
+      const float k2 = __shfl_xor_sync(0xffffffffu, best, o);
+      const int i2 = __shfl_xor_sync(0xffffffffu, who, o);
+      if (k2 > best || (k2 == best && i2 < who)) { best = k2; who = i2; }
+    }
+    const float g = __shfl_sync(0xffffffffu, gate, group0 + (who & (W - 1)));
+    if (sub == who) taken = true;
+    if (live_row && sub == 0) { idx_row[i] = group_base + who; gates_row[i] = g; }
+  }
+}
+
 template <typename T, int NACC>
 __global__ void __launch_bounds__(256)
 router_kernel(const T* __restrict__ xo, int n_rows, int d, int n_r, int n_rp, int n_k,

@@ -194,6 +194,9 @@ constexpr int kRskMaxSlices = 64;           // d <= 8192
 constexpr int kRskThreads = 256;
 constexpr int kRskFuseGroups = 64;
 
+// SUB8: the gate logic of the last block runs four rows per warp (8 lanes each; needs n_r <= 8),
+// which pays for batches of more than 16 rows; the plain form is launched otherwise.
+template <bool SUB8>
 __global__ void __launch_bounds__(kRskThreads)
 router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, int n_rp, int n_k,
                      const bf16* __restrict__ w_rep, const float* __restrict__ u, const float* __restrict__ b,
@@ -293,12 +296,26 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
     *reinterpret_cast<float4*>(&total[r][n]) = sum;
   }
   __syncthreads();
-  for (int r = warp; r < n_rows; r += kRskThreads / 32) {
-    const float a = lane < n_r ? total[r][lane] : 0.0f;
-    const float v = lane < n_r ? total[r][n_rp + lane] : 0.0f;
-    const int go = row_group[r];
-    gate_row(lane, n_r, n_k, a, v, u + go * n_r, b + go * n_r, go * n_r, scores + (size_t)r * n_r,
-             keys + (size_t)r * n_r, topk_idx + (size_t)r * n_k, topk_gate + (size_t)r * n_k);
+  if (SUB8) {                                      // four rows per warp at a time, 8 lanes each
+    const int sub = lane & 7, grp = lane >> 3;
+    for (int r0 = warp * 4; r0 < n_rows; r0 += (kRskThreads / 32) * 4) {
+      const int r = r0 + grp;
+      const bool live_row = r < n_rows;
+      const int rr = live_row ? r : 0;
+      const float a = (live_row && sub < n_r) ? total[rr][sub] : 0.0f;
+      const float v = (live_row && sub < n_r) ? total[rr][n_rp + sub] : 0.0f;
+      const int go = row_group[rr];
+      gate_row_sub<8>(sub, live_row, n_r, n_k, a, v, u + go * n_r, b + go * n_r, go * n_r, scores + (size_t)rr * n_r,
+                      keys + (size_t)rr * n_r, topk_idx + (size_t)rr * n_k, topk_gate + (size_t)rr * n_k);
+    }
+  } else {
+    for (int r = warp; r < n_rows; r += kRskThreads / 32) {
+      const float a = lane < n_r ? total[r][lane] : 0.0f;
+      const float v = lane < n_r ? total[r][n_rp + lane] : 0.0f;
+      const int go = row_group[r];
+      gate_row(lane, n_r, n_k, a, v, u + go * n_r, b + go * n_r, go * n_r, scores + (size_t)r * n_r,
+               keys + (size_t)r * n_r, topk_idx + (size_t)r * n_k, topk_gate + (size_t)r * n_k);
+    }
   }
   if (threadIdx.x == 0) *ticket = 0;
   if (!fuse_permute) return;
