@@ -97,10 +97,11 @@ int cmoe_hier_create(int32_t n_outer, int32_t outer_top_k, const void* w_router,
 
 /* out = F_MoE(x) for T tokens (Eq. moe_output with Eq. router and Eq. final_gate).
  *   x   : device, [T, d_model] row-major, 16-byte aligned.
- *   out : device, [T, d_model] row-major, 16-byte aligned, must not overlap x.
+ *   out : device, [T, d_model] row-major, 32-byte aligned (the combine step writes 32 bytes
+ *         per store), must not overlap x.
  * Asynchronous on `stream`; allocates nothing; T == 0 is a no-op.  A layer owns
  * one workspace: do not run two forwards of the same layer concurrently.
- * Errors: INVALID_ARG, CAPACITY (T > max_tokens), CUDA. */
+ * Errors: INVALID_ARG (null, misaligned or overlapping buffers), CAPACITY (T > max_tokens), CUDA. */
 int cmoe_ffn_forward(cmoe_layer* layer, const void* x, int32_t T, void* out, void* stream);
 
 /* Replace the learnable gate scaling u and the selection bias b (Section 4.3).
@@ -145,7 +146,8 @@ int cmoe_layer_update_bias(cmoe_layer* layer, float gamma, const float* target_s
  * Both outputs accumulate: the caller zeroes them before the first chunk.  Asynchronous on
  * `stream`; the buffers belong to the caller.  Errors: INVALID_ARG (layer has routed experts or
  * is hierarchical, k_a outside [1, d_ff], null or misaligned pointers), CAPACITY, UNSUPPORTED
- * (d_ff above 24576 for bf16 or 12288 for fp32: a row's keys are staged in 48 KB of shared memory), CUDA. */
+ * (d_ff above 20352 for bf16 or 10176 for fp32: a row's keys and the candidate arrays share 48 KB
+ * of shared memory), CUDA. */
 int cmoe_profile_activations(cmoe_layer* layer, const void* x, int32_t n_tokens, int32_t k_a, int32_t token0,
                              uint32_t* act_bits, int32_t words_per_neuron, int32_t* act_count, void* stream);
 
@@ -234,8 +236,19 @@ int cmoe_get_routing(cmoe_layer* layer, float* keys, float* scores, int32_t* top
 
 /* Device-side error word of the last forward: 0, or a code written by a kernel whose
  * bounded wait (mbarrier) ran out.  Synchronises the last stream.  Returns
- * CMOE_ERR_DEVICE_TIMEOUT when the word is non-zero. */
+ * CMOE_ERR_DEVICE_TIMEOUT when the word is non-zero; the output of the forward that timed out
+ * is undefined.  Recovery is part of this call: after reporting a timeout it clears the error
+ * word and the K-slice tickets a part-finished kernel may have left taken, so the layer can be
+ * used again (the next status call reports CMOE_OK unless another wait runs out). */
 int cmoe_layer_status(cmoe_layer* layer, int32_t* device_error_word);
+
+/* Self-test of the give-up path (no paper counterpart: failure detection of this library).
+ * Enqueues one warp that waits on a barrier nobody arrives on through the same bounded wait the
+ * tensor-core kernels use, with a limit of limit_cycles SM clock cycles (1e3 .. 2e9; 2e6 is
+ * about a millisecond).  The wait gives up, writes its code to the layer's error word and the
+ * kernel returns normally: nothing traps, no copy is in flight, the context stays usable.
+ * cmoe_layer_status then returns CMOE_ERR_DEVICE_TIMEOUT once.  Asynchronous on `stream`. */
+int cmoe_layer_selftest_wait_timeout(cmoe_layer* layer, int64_t limit_cycles, void* stream);
 
 /* Number of this library's kernels the last forward launched. */
 int cmoe_layer_launch_count(const cmoe_layer* layer, int32_t* n_launches);

@@ -21,7 +21,7 @@ EXPORTS = [
     "cmoe_layer_create", "cmoe_hier_create", "cmoe_ffn_forward", "cmoe_layer_set_gate_params",
     "cmoe_layer_get_gate_params", "cmoe_layer_update_bias", "cmoe_profile_activations", "cmoe_select_shared",
     "cmoe_cluster_update", "cmoe_cluster_distances", "cmoe_cluster_representatives", "cmoe_layer_set_gemm_path", "cmoe_layer_set_launch_chaining",
-    "cmoe_layer_dims", "cmoe_get_routing", "cmoe_layer_status",
+    "cmoe_layer_dims", "cmoe_get_routing", "cmoe_layer_status", "cmoe_layer_selftest_wait_timeout",
     "cmoe_layer_launch_count", "cmoe_layer_enable_stage_timing", "cmoe_layer_stage_times",
     "cmoe_layer_destroy", "cmoe_token_permute_scratch_bytes",
     "cmoe_token_permute", "cmoe_token_permute_static", "cmoe_status_string", "cmoe_last_error",
@@ -70,6 +70,7 @@ def load() -> C.CDLL:
     lib.cmoe_layer_dims.argtypes = [vp] + [C.POINTER(i32)] * 4
     lib.cmoe_get_routing.argtypes = [vp] * 12
     lib.cmoe_layer_status.argtypes = [vp, C.POINTER(i32)]
+    lib.cmoe_layer_selftest_wait_timeout.argtypes = [vp, i64, vp]
     lib.cmoe_layer_launch_count.argtypes = [vp, C.POINTER(i32)]
     lib.cmoe_layer_destroy.argtypes = [vp]
     lib.cmoe_layer_enable_stage_timing.argtypes = [vp, i32]
@@ -237,11 +238,18 @@ class Layer:
         return r
 
     def status(self) -> int:
+        """Device error word of the last forward (0 = none).  A non-zero word is reported once:
+        the call also clears it and the layer's K-slice tickets."""
         w = C.c_int32()
         st = load().cmoe_layer_status(self._h, C.byref(w))
         if st not in (0, -6):
             _check(st, "cmoe_layer_status")
         return w.value
+
+    def selftest_wait_timeout(self, limit_cycles: int = 2_000_000, stream=None) -> None:
+        """cmoe_layer_selftest_wait_timeout: one warp runs a bounded wait to its limit."""
+        _check(load().cmoe_layer_selftest_wait_timeout(self._h, limit_cycles, _stream_ptr(stream)),
+               "cmoe_layer_selftest_wait_timeout")
 
     def launch_count(self) -> int:
         w = C.c_int32()

@@ -111,6 +111,7 @@ struct cmoe_layer {
   int32_t* rt_ticket = nullptr;
   float* dec_part = nullptr;    // decode GEMMs: K-slice partial sums, tickets per (tile, epilogue warp)
   int32_t* dec_ticket = nullptr;
+  size_t n_dec_ticket = 0, n_rt_ticket = 0;    // lengths of the ticket arrays (zeroed again after a device timeout)
   float *share = nullptr, *target = nullptr;   // utilisation of the last step / bias-update targets
 
   cudaStream_t last_stream = nullptr;
@@ -231,11 +232,13 @@ void carve_workspace(cmoe_layer* L, char* base) {
   if (esz == 2) {
     const size_t t1 = (size_t)L->n_outer * ((L->shared_width() + 127) / 128 + nr * ((L->m + 127) / 128));
     const size_t t2 = (size_t)L->n_groups_total() * ((d + 127) / 128);
-    L->dec_ticket = a.take<int32_t>(4 * (t1 > t2 ? t1 : t2));
+    L->n_dec_ticket = 4 * (t1 > t2 ? t1 : t2);
+    L->dec_ticket = a.take<int32_t>(L->n_dec_ticket);
     L->dec_part = a.take<float>((size_t)kDecMaxSlots * kDecSlotFloats);
   }
   if (esz == 2 && nr > 0) {
-    L->rt_ticket = a.take<int32_t>(4 * 256);
+    L->n_rt_ticket = 4 * 256;
+    L->rt_ticket = a.take<int32_t>(L->n_rt_ticket);
     L->rt_part = a.take<float>((size_t)256 * 64 * 128);
   }
   L->ws_bytes = align_up(a.used + 256, 256);
@@ -617,8 +620,9 @@ int cmoe_ffn_forward(cmoe_layer* L, const void* x, int32_t T, void* out, void* s
   if (T == 0) { L->last_T = 0; L->launches = 0; return CMOE_OK; }
   if (!x || !out) return arg_fail(CMOE_ERR_INVALID_ARG, "null x / out");
   if (T > L->cfg.max_tokens) return arg_fail(CMOE_ERR_CAPACITY, "T exceeds max_tokens");
-  if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(out)) & 15)
-    return arg_fail(CMOE_ERR_INVALID_ARG, "x / out must be 16-byte aligned");
+  if (reinterpret_cast<uintptr_t>(x) & 15) return arg_fail(CMOE_ERR_INVALID_ARG, "x must be 16-byte aligned");
+  if (reinterpret_cast<uintptr_t>(out) & 31)      // the combine kernels write 32 bytes per store
+    return arg_fail(CMOE_ERR_INVALID_ARG, "out must be 32-byte aligned");
   {
     const char *xa = (const char*)x, *oa = (const char*)out;
     const size_t bytes = (size_t)T * L->cfg.d_model * L->esz;
@@ -648,8 +652,9 @@ int cmoe_profile_activations(cmoe_layer* L, const void* x, int32_t T, int32_t k_
   L->last_stream = st;
   L->last_T = T;
   const int d_ff = L->cfg.d_ff;
-  if ((size_t)d_ff * L->esz > 48 * 1024)      // the row's keys are staged in (default-sized) shared memory
-    return arg_fail(CMOE_ERR_UNSUPPORTED, "profiling supports d_ff up to 24576 (bf16) / 12288 (fp32)");
+  // a row's keys are staged in dynamic shared memory next to the kernel's static arrays; both must fit 48 KB
+  if ((size_t)d_ff * L->esz + kAtopkStaticSmem > 48 * 1024)
+    return arg_fail(CMOE_ERR_UNSUPPORTED, "profiling supports d_ff up to 20352 (bf16) / 10176 (fp32)");
   int rc;
   if (L->cfg.dtype == CMOE_BF16) {
     rc = forward_impl<bf16>(L, (const bf16*)x, T, nullptr, st, true);
@@ -831,7 +836,27 @@ int cmoe_layer_status(cmoe_layer* L, int32_t* device_error_word) {
   if (!L || !device_error_word) return arg_fail(CMOE_ERR_INVALID_ARG, "null argument");
   CU_TRY(cudaMemcpyAsync(device_error_word, L->err_word, 4, cudaMemcpyDeviceToHost, L->last_stream));
   CU_TRY(cudaStreamSynchronize(L->last_stream));
-  return *device_error_word ? CMOE_ERR_DEVICE_TIMEOUT : CMOE_OK;
+  if (*device_error_word == 0) return CMOE_OK;
+  // A wait gave up: that forward's output is undefined and its K-slice tickets may be left part-taken.
+  // Clear the error word and every ticket so that the next forward starts from a clean state.
+  cudaStream_t st = L->last_stream;
+  CU_TRY(cudaMemsetAsync(L->err_word, 0, 4, st));
+  CU_TRY(cudaMemsetAsync(L->rsk_ticket, 0, 4, st));
+  if (L->dec_ticket) CU_TRY(cudaMemsetAsync(L->dec_ticket, 0, L->n_dec_ticket * 4, st));
+  if (L->rt_ticket) CU_TRY(cudaMemsetAsync(L->rt_ticket, 0, L->n_rt_ticket * 4, st));
+  CU_TRY(cudaStreamSynchronize(st));
+  return CMOE_ERR_DEVICE_TIMEOUT;
+}
+
+int cmoe_layer_selftest_wait_timeout(cmoe_layer* L, int64_t limit_cycles, void* stream) {
+  if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "null layer");
+  if (limit_cycles < 1000 || limit_cycles > 2000000000LL)
+    return arg_fail(CMOE_ERR_INVALID_ARG, "limit_cycles outside [1e3, 2e9]");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  L->last_stream = st;
+  wait_timeout_probe_kernel<<<1, 32, 0, st>>>(L->err_word, (long long)limit_cycles);
+  CU_TRY(cudaGetLastError());
+  return CMOE_OK;
 }
 
 int cmoe_layer_launch_count(const cmoe_layer* L, int32_t* n_launches) {

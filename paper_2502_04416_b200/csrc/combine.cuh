@@ -146,9 +146,11 @@ combine_kernel(const T* __restrict__ y_s, const T* __restrict__ y_r,
 // the next token's routing words are fetched while the current rows are in flight.  The
 // arithmetic and its order are those of combine_kernel, so both give the same bits.
 __device__ __forceinline__ void ld256_stream(const bf16* p, uint32_t (&w)[8]) {
-  asm("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-      : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
-      : "l"(p));
+  // volatile + memory clobber: the load must stay below griddepcontrol.wait (its source is written
+  // by the preceding kernel of a chained launch)
+  asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+               : "l"(p) : "memory");
 }
 
 template <int NK>

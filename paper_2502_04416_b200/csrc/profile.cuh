@@ -44,6 +44,8 @@ __device__ __forceinline__ int block_sum(int v, int* red) {
 }
 
 constexpr int kAtopkCap = 1024;     // candidates ranked directly
+// static shared memory of atopk_kernel: two candidate arrays, two per-warp arrays, two scalars (rounded up)
+constexpr int kAtopkStaticSmem = 2 * kAtopkCap * 4 + 2 * (kAtopkThreads / 32) * 4 + 192;
 
 // One block per token row; the row's magnitude keys are staged once in shared memory.
 // Fast path (K_a small against d_h, the paper's K_a = 10): the K_a-th largest of the 256

@@ -78,7 +78,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait: false if the wait ran out (error word + abort flag set) or another wait
 // of this CTA already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int32_t* err_word, int code) {
+                                          int32_t* err_word, int code, long long limit = kUmmaWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
@@ -86,7 +86,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kUmmaWaitCycles) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1;
       atomicCAS(err_word, 0, code);
       return false;
@@ -170,6 +170,23 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t addr) {
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
 __device__ __forceinline__ uint32_t umma_idesc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kUmmaBM >> 4) << 24);
+}
+
+// One warp waits, with a limit of `limit` SM cycles, on an mbarrier that nobody arrives on, through the
+// same mbar_wait the tensor-core kernels use: the wait gives up, the error word takes the code,
+// the kernel returns normally.  No copy is in flight and no tensor memory is held.
+__global__ void wait_timeout_probe_kernel(int32_t* err_word, long long limit) {
+  __shared__ __align__(8) unsigned long long bar_mem;
+  __shared__ int abort_flag;
+  const uint32_t bar = smem_u32(&bar_mem);
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  if (threadIdx.x == 0) mbar_wait(bar, 0, &abort_flag, err_word, kErrWaitFull, limit);
+  __syncwarp();
 }
 
 // ----------------------------------------------------------------------------- kernel

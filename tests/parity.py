@@ -113,9 +113,10 @@ def check_output(got: np.ndarray, want: np.ndarray):
 
 
 def check_plain_layer(layer: binding.Layer, lay: wl.LayerInputs, x: np.ndarray,
-                      sample_tokens: Optional[np.ndarray] = None) -> dict:
+                      sample_tokens=None) -> dict:
     """One forward of a plain layer on x [T,d], compared stage by stage with the oracle.
-    ``sample_tokens``: compare outputs only on these tokens (large workloads)."""
+    ``sample_tokens``: compare outputs only on these tokens (large workloads); an array, or a
+    callable (n_tok, counts, offsets, row_token) -> token ids such as ``stratified_tokens``."""
     import torch
     s = lay.shape
     n_tok = x.shape[0]
@@ -133,19 +134,82 @@ def check_plain_layer(layer: binding.Layer, lay: wl.LayerInputs, x: np.ndarray,
         cnt = check_permutation(rc.sel_idx, s.n_routed, r["topk_idx"], r)
         stats.update(near_tie=rc.near_tie, differing=rc.differing, counts=cnt.tolist())
         sel, gates = rc.sel_idx, rc.gates
+        if callable(sample_tokens):    # chosen from the oracle's own (patched) permutation
+            _, off, row_token, _ = oracle.token_permutation(sel, s.n_routed)
+            sample_tokens = sample_tokens(n_tok, cnt, off, row_token)
     else:
         sel = np.zeros((n_tok, 0), np.int32)
         gates = np.zeros((n_tok, 0))
+        if callable(sample_tokens):
+            sample_tokens = sample_tokens(n_tok, [], [0], [])
     want = oracle.moe_forward(x, lay.w_gate, lay.w_up, lay.w_down, lay.neuron_perm, s.n_experts,
                               s.n_shared, sel, gates, token_ids=sample_tokens)
     if sample_tokens is not None:
         got = got[sample_tokens]
+        stats["sampled"] = len(sample_tokens)
     stats["max_rel"], stats["mean_rel"] = check_output(got, want)
     return stats
 
 
+def check_outer_routing(gpu_outer_idx: np.ndarray, gpu_outer_w: np.ndarray, x: np.ndarray,
+                        w_router: np.ndarray, outer_top_k: int):
+    """Outer level of a hierarchical layer (Section 4.4), the same rule as the inner level: the
+    selected sets must equal the oracle's except on tokens whose outer_top_k-th and next logit are
+    within MARGIN; there the CUDA choice may only trade experts whose logit is within MARGIN of the
+    cut, the oracle's selection is replaced by it and the weights (softmax over the selected
+    logits) are recomputed for that selection.  Pure numpy: no device is touched.
+    Returns (outer_idx, outer_w, near-tie tokens, differing tokens) after patching."""
+    o_idx, o_w, logits = oracle.outer_router(x, w_router, outer_top_k)
+    n_tok, n_outer = logits.shape
+    assert gpu_outer_idx.min() >= 0 and gpu_outer_idx.max() < n_outer
+    srt = -np.sort(-logits, axis=1)
+    cut = srt[:, outer_top_k - 1]
+    near = (cut - srt[:, outer_top_k]) < MARGIN if outer_top_k < n_outer else np.zeros(n_tok, bool)
+    differ = ~(np.sort(gpu_outer_idx, 1) == np.sort(o_idx, 1)).all(axis=1)
+    assert not (differ & ~near).any(), \
+        f"{int((differ & ~near).sum())} tokens pick other outer experts with margin >= {MARGIN}"
+    for t in np.nonzero(differ)[0]:
+        assert len(set(gpu_outer_idx[t])) == outer_top_k
+        traded = set(gpu_outer_idx[t]) ^ set(o_idx[t])
+        assert all(abs(logits[t, e] - cut[t]) < MARGIN for e in traded), f"token {t}: inadmissible outer choice"
+        order = sorted(gpu_outer_idx[t], key=lambda e: (-logits[t, e], e))     # descending logit, like the oracle
+        o_idx[t] = order
+        o_w[t] = oracle.softmax(logits[t, order][None, :])[0]
+    go, oo = np.argsort(gpu_outer_idx, 1), np.argsort(o_idx, 1)
+    np.testing.assert_allclose(np.take_along_axis(gpu_outer_w, go, 1),
+                               np.take_along_axis(o_w, oo, 1), rtol=1e-4, atol=1e-6)
+    return o_idx, o_w, int(near.sum()), int(differ.sum())
+
+
+def stratified_tokens(n_tok: int, counts, offsets, row_token, seed: int, n_random: int = 48,
+                      tile: int = 128) -> np.ndarray:
+    """Tokens at which a large workload's output is compared: first and last token, the tokens
+    on both sides of the first and last tile edge of the token-ordered (shared) rows, for every
+    routed group the tokens of its first and last row, for the largest and the smallest non-empty
+    group the tokens on both sides of every ``tile``-row edge, plus a seeded random sample.
+    ``counts/offsets/row_token`` are the oracle's permutation (after near-tie patching)."""
+    ids = {0, n_tok - 1}
+    for e in (tile, (n_tok - 1) // tile * tile):
+        ids.update(t for t in (e - 1, e) if 0 <= t < n_tok)
+    counts = np.asarray(counts)
+    live = np.nonzero(counts > 0)[0]
+    for g in live:
+        ids.add(int(row_token[offsets[g]]))
+        ids.add(int(row_token[offsets[g + 1] - 1]))
+    if live.size:
+        big = live[np.argmax(counts[live])]
+        small = live[np.argmin(counts[live])]
+        for g in {int(big), int(small)}:
+            for e in range(tile, int(counts[g]), tile):
+                ids.add(int(row_token[offsets[g] + e - 1]))
+                ids.add(int(row_token[offsets[g] + e]))
+    rng = np.random.default_rng(seed)
+    ids.update(int(t) for t in rng.choice(n_tok, size=min(n_random, n_tok), replace=False))
+    return np.array(sorted(ids), dtype=np.int64)
+
+
 def check_hier_layer(layer: binding.Layer, inputs: wl.WorkloadInputs, x: np.ndarray,
-                     sample_tokens: Optional[np.ndarray] = None) -> dict:
+                     sample_tokens=None) -> dict:
     """Hierarchical layer: outer routing, per-outer-expert inner routing, flattened
     permutation over n_outer*N_r groups, output."""
     import torch
@@ -158,22 +222,14 @@ def check_hier_layer(layer: binding.Layer, inputs: wl.WorkloadInputs, x: np.ndar
     got = to_host(out)
     r = layer.routing(n_tok, nr)
     # --- outer level
-    o_idx, o_w, logits = oracle.outer_router(x, inputs.w_router, ok)
-    srt = -np.sort(-logits, axis=1)
-    near_outer = (srt[:, ok - 1] - srt[:, ok]) < MARGIN if ok < n_outer else np.zeros(n_tok, bool)
-    differ = ~(np.sort(r["outer_idx"], 1) == np.sort(o_idx, 1)).all(axis=1)
-    assert not (differ & ~near_outer).any()
-    assert not differ.any(), "outer near-tie patching is not implemented; pick another seed"
-    go, oo = np.argsort(r["outer_idx"], 1), np.argsort(o_idx, 1)
-    np.testing.assert_allclose(np.take_along_axis(r["outer_w"], go, 1),
-                               np.take_along_axis(o_w, oo, 1), rtol=1e-4, atol=1e-6)
+    o_idx, o_w, near_o, diff_o = check_outer_routing(r["outer_idx"], r["outer_w"], x, inputs.w_router, ok)
     _, o_off, o_row_token, _ = oracle.token_permutation(o_idx, n_outer)
     np.testing.assert_array_equal(r["outer_row_token"], o_row_token)
     # --- inner level, outer expert by outer expert (rows are grouped by outer expert)
     R = n_tok * ok
     sel_global = np.zeros((R, k), np.int32)
     gates_all = np.zeros((R, k))
-    near = diff = 0
+    near, diff = near_o, diff_o
     for i, lay in enumerate(inputs.layers):
         rows = np.arange(o_off[i], o_off[i + 1])
         if rows.size == 0:
@@ -187,8 +243,11 @@ def check_hier_layer(layer: binding.Layer, inputs: wl.WorkloadInputs, x: np.ndar
         gates_all[rows] = rc.gates
         near += rc.near_tie
         diff += rc.differing
-    check_permutation(sel_global, n_outer * nr, r["topk_idx"], r)
+    cnt = check_permutation(sel_global, n_outer * nr, r["topk_idx"], r)
     # --- output on the sampled tokens
+    if callable(sample_tokens):        # chosen from the permutation: routed rows hold outer rows, those hold tokens
+        _, off_in, row_tok_in, _ = oracle.token_permutation(sel_global, n_outer * nr)
+        sample_tokens = sample_tokens(n_tok, cnt, off_in, o_row_token[row_tok_in])
     keep = np.arange(n_tok) if sample_tokens is None else np.asarray(sample_tokens)
     want = np.zeros((len(keep), s.d_model))
     row_of_tok = {(int(o_row_token[rr]), int(i)): rr for i in range(n_outer)
@@ -205,8 +264,8 @@ def check_hier_layer(layer: binding.Layer, inputs: wl.WorkloadInputs, x: np.ndar
         wt = np.array([o_w[t, list(o_idx[t]).index(i)] for t in toks])
         want[pos] += wt[:, None] * y
     max_rel, mean_rel = check_output(got[keep], want)
-    return dict(tokens=n_tok, near_tie=near, differing=diff, max_rel=max_rel, mean_rel=mean_rel,
-                launches=layer.launch_count())
+    return dict(tokens=n_tok, near_tie=near, differing=diff, outer_near_tie=near_o, outer_differing=diff_o,
+                sampled=len(keep), max_rel=max_rel, mean_rel=mean_rel, launches=layer.launch_count())
 
 
 # ------------------------------------------------------------ activation profiling

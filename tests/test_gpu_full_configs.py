@@ -1,7 +1,10 @@
 """-m gpu: the five full-size workloads in the launch configuration bench.py times.
 Routing, counts, offsets and the permutation are compared for every token (bit-exact
-outside the near-tie margin); outputs on a seeded sample of tokens that the oracle
-evaluates one expert batch at a time."""
+outside the near-tie margin); outputs on a stratified sample of a few hundred tokens
+(batch ends, tile edges of the shared rows, first and last row of every routed group,
+every 128-row tile edge of the largest and the smallest group, plus a seeded random
+draw) that the oracle evaluates one expert batch at a time."""
+import functools
 import numpy as np
 import pytest
 
@@ -11,16 +14,12 @@ from tests import parity
 
 pytestmark = pytest.mark.gpu
 
-N_SAMPLE = 48
 
 
 def _sample(n_tok, seed):
-    if n_tok <= N_SAMPLE:
+    if n_tok <= 64:
         return None
-    rng = np.random.default_rng(seed)
-    ids = np.sort(rng.choice(n_tok, size=N_SAMPLE, replace=False))
-    ids[0], ids[-1] = 0, n_tok - 1                      # first and last row of the batch
-    return ids
+    return functools.partial(parity.stratified_tokens, seed=seed)
 
 
 @pytest.mark.parametrize("name", ["c2_llama2_7b", "c3_llama3_8b", "c5_skew_13b"])
@@ -35,7 +34,7 @@ def test_plain_workloads_full_size(name):
         st = parity.check_plain_layer(layer, lay, inputs.x[:t], sample_tokens=_sample(t, t))
         assert st["differing"] <= st["near_tie"]
         assert sum(st["counts"]) == t * w.shape.top_k
-        print(name, t, {k: st[k] for k in ("near_tie", "differing", "max_rel", "mean_rel")},
+        print(name, t, {k: st.get(k) for k in ("near_tie", "differing", "sampled", "max_rel", "mean_rel")},
               "counts", st["counts"])
         if w.zipf_s:                                     # the load really is skewed as designed
             share = np.array(st["counts"]) / sum(st["counts"])

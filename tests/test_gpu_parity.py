@@ -1,6 +1,7 @@
 """-m gpu: the CUDA path, called through the C-ABI, against the CPU oracle on the
 same seeded inputs.  Small shapes keep each expert's ragged tile tails (m = 1376,
 448, 864 ...) and token counts that are not multiples of any tile."""
+import ctypes as C
 import dataclasses
 
 import numpy as np
@@ -87,6 +88,27 @@ def test_hierarchical_small(path):
     layer.destroy()
 
 
+def test_hierarchical_outer_near_ties():
+    """Outer logits within the 1e-3 margin (Section 4.4's top-level router): two pairs of outer
+    experts get router rows that differ in one coordinate by 2^-27, so whenever such a pair
+    straddles the outer cut the fp32 logits cannot tell its members apart while the fp64 oracle
+    can.  The CUDA choice must then be an admissible trade and everything downstream (outer
+    permutation, inner routing, output) must agree once the oracle takes that choice."""
+    inp = _inputs("c4_hier_8x7b", d_model=256, tokens=(600,), m=64)
+    w_r = inp.w_router
+    for a, b_, col in ((1, 4, 3), (2, 6, 100)):
+        w_r[b_] = w_r[a]
+        w_r[a, col] = np.float32(2.0 ** -20)
+        w_r[b_, col] = np.float32(2.0 ** -20 * (1 + 2.0 ** -7))       # both exact in bf16
+    inners = [parity.gpu_layer(lay, 8) for lay in inp.layers]
+    layer = binding.Layer.create_hier(parity.to_device(w_r, "bf16"), inners, 2, 600)
+    st = parity.check_hier_layer(layer, inp, inp.x)
+    print("outer near-ties:", st["outer_near_tie"], "differing:", st["outer_differing"])
+    assert st["outer_near_tie"] >= 50                    # the planted pairs straddle the cut often
+    assert st["outer_differing"] <= st["outer_near_tie"]
+    layer.destroy()
+
+
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
 def test_degenerate_structures(path):
     base = wl.shrunk(wl.WORKLOADS["c2_llama2_7b"], d_model=128, tokens=(70,), m=80)
@@ -121,6 +143,9 @@ def test_call_contract():
     with pytest.raises(binding.CmoeError) as e:
         layer.forward(x[:8], x[:8])                               # aliasing
     assert e.value.status == -1
+    with pytest.raises(binding.CmoeError) as e:                   # out 16- but not 32-byte aligned: refused on the
+        layer.forward(x[:8], out.view(-1)[8:8 + 8 * 128].view(8, 128))   # host, nothing is launched
+    assert e.value.status == -1
     a = layer.forward(x[:32]).clone()
     b = layer.forward(x[:32]).clone()
     torch.cuda.synchronize()
@@ -130,6 +155,30 @@ def test_call_contract():
     layer.set_gate_params(gate_scale_u=u)
     lay.gate_scale_u = u
     parity.check_plain_layer(layer, lay, inp.x[:32])
+    layer.destroy()
+
+
+def test_wait_timeout_is_reported_and_recovered():
+    """The give-up path of the bounded device-side waits: a wait that nothing ends runs to its
+    (millisecond) limit, the kernel returns normally, the layer's error word carries the code,
+    cmoe_layer_status maps it to the timeout status once and clears it, and the layer then
+    computes correct results again (tensor path: decode, mid-size and large batches)."""
+    import torch
+    inp = _inputs("c2_llama2_7b", d_model=256, tokens=(700,), m=160)
+    lay = inp.layers[0]
+    layer = parity.gpu_layer(lay, 700)
+    parity.check_plain_layer(layer, lay, inp.x[:700])
+    assert layer.status() == 0
+    layer.selftest_wait_timeout(2_000_000)
+    torch.cuda.synchronize()
+    w = C.c_int32()
+    assert binding.load().cmoe_layer_status(layer._h, C.byref(w)) == -6      # CMOE_ERR_DEVICE_TIMEOUT
+    assert w.value == 1                                                       # the wait's own code
+    assert layer.status() == 0                                                # reported once, then cleared
+    for t in (1, 64, 300, 700):
+        parity.check_plain_layer(layer, lay, inp.x[:t])
+    with pytest.raises(binding.CmoeError):
+        layer.selftest_wait_timeout(10)                                       # limit below the documented range
     layer.destroy()
 
 

@@ -259,6 +259,44 @@ def pin_bias_update_rule(o):
     np.testing.assert_allclose(got, [-0.4, 0.7, 0.8, -0.1], rtol=0, atol=1e-15)
 
 
+def pin_fit_select_bias(o):
+    """The iterated bias rule of Section 4.3 on scores small enough to follow by hand.
+    Three experts, top-1, 24 rows whose softmax values are given outright (s = ln p).
+    Row r gives expert 0 the value p_0 = 0.40 + 0.01 r and splits the rest between experts 1 and 2
+    in a proportion that varies from row to row; with b = 0 expert 0 wins all 24 rows."""
+    rows = 24
+    r = np.arange(rows)
+    p0 = 0.40 + 0.01 * r
+    f = 0.35 + 0.0125 * ((7 * r) % 24)
+    p = np.stack([p0, (1 - p0) * f, (1 - p0) * (1 - f)], axis=1)
+    assert np.all(p[:, 0] > p[:, 1:].max(axis=1))
+    s = np.log(p)
+    # (1) a target that b = 0 already meets is left alone: no update is applied
+    b, counts = o.fit_select_bias(s, 1, [1.0, 0.0, 0.0], tol=1e-9)
+    assert np.all(b == 0.0) and list(counts) == [24, 0, 0]
+    # (2) the step decays geometrically from gamma_hi to gamma_lo: with a tolerance that is never
+    # met and three iterations, expert 0 (always over its target) loses hi + sqrt(hi*lo) + lo and
+    # expert 2 (always under) gains the same
+    hi, lo = 4e-3, 1e-3
+    b, _ = o.fit_select_bias(s, 1, [0.0, 0.5, 0.5], iters=3, gamma_hi=hi, gamma_lo=lo, tol=0.0)
+    total = hi + math.sqrt(hi * lo) + lo
+    np.testing.assert_allclose(b, [-total, total, total], rtol=1e-12)
+    # (3) a reachable target is reached on EVERY expert: recount the selections with the returned b
+    # by a scalar loop.  Shares move in steps of 1/24 > tol, so only the exact split 12/8/4 passes; on
+    # the way there the split 12/9/3 has expert 0 on target and a mean deviation under tol, so a
+    # stopping test on one expert or on the mean ends too early.
+    target = np.array([12, 8, 4]) / 24.0
+    tol = 0.03
+    b, counts = o.fit_select_bias(s, 1, target, iters=4000, gamma_hi=2e-2, gamma_lo=1e-4, tol=tol)
+    recount = [0, 0, 0]
+    for r in range(rows):
+        keys = [p[r, j] + b[j] for j in range(3)]
+        recount[max(range(3), key=lambda j: (keys[j], -j))] += 1
+    assert list(counts) == recount
+    assert max(abs(recount[j] / rows - target[j]) for j in range(3)) <= tol
+    assert b[0] < 0 < b[2]                     # the overloaded expert was pushed down, the starved one up
+
+
 # ---------------------------------------------------------------- hierarchical
 def hier_case(seed=12, n_outer=4, top_k=None):
     shape = wl.LayerShape(20, 8 * 5, 8, 2, 2, "fp32")
@@ -460,7 +498,7 @@ def pin_initial_centroids_and_assignment(o):
 PINS = [pin_dense_closed_form, pin_dense_library, pin_dense_per_neuron_brute_force,
         pin_all_experts_on_is_dense, pin_reconstruction_error_identity, pin_shared_always_on,
         pin_router_is_representative_activation, pin_gate_closed_forms, pin_topk_brute_force,
-        pin_moe_linear_in_gates, pin_permutation, pin_logit_margin, pin_bias_update_rule,
+        pin_moe_linear_in_gates, pin_permutation, pin_logit_margin, pin_bias_update_rule, pin_fit_select_bias,
         pin_hierarchical_all_on_is_original_moe, pin_hierarchical_is_weighted_sum_of_layers,
         pin_atopk_brute_force, pin_atopk_invariants, pin_activation_rates_and_shared, pin_profile_pipeline,
         pin_distance_is_hamming_on_binary, pin_cluster_update_and_representatives,
@@ -502,6 +540,13 @@ MUTATIONS = {
     "offsets_inclusive": ("off[e + 1] = off[e] + cnt[e]", "off[e + 1] = off[e] + cnt[e] + (e == 0)"),
     "outer_weights_unnormalised": ("outer_w = softmax(sel_logits)", "outer_w = np.exp(sel_logits)"),
     "bias_rule_sign": ("b[p > target] -= gamma", "b[p > target] += gamma"),
+    "fit_step_grows": ("gamma = gamma_hi * (gamma_lo / gamma_hi) ** (it / max(iters - 1, 1))",
+                       "gamma = gamma_hi * (gamma_hi / gamma_lo) ** (it / max(iters - 1, 1))"),
+    "fit_step_constant": ("gamma = gamma_hi * (gamma_lo / gamma_hi) ** (it / max(iters - 1, 1))", "gamma = gamma_hi"),
+    "fit_stops_on_mean": ("if np.abs(counts / counts.sum() - target).max() <= tol:",
+                          "if np.abs(counts / counts.sum() - target).mean() <= tol:"),
+    "fit_stops_on_first_expert": ("if np.abs(counts / counts.sum() - target).max() <= tol:",
+                                  "if np.abs(counts / counts.sum() - target)[0] <= tol:"),
     "atopk_signed": ("mag = np.abs(_f64(h))\n    order", "mag = _f64(h)\n    order"),
     "atopk_smallest": ("order = np.argsort(-mag, axis=1, kind=\"stable\")[:, :k_a]",
                        "order = np.argsort(mag, axis=1, kind=\"stable\")[:, :k_a]"),
