@@ -164,12 +164,17 @@ def prepare_inputs(name: str):
     return inputs
 
 
-# DRAM bytes (read + write) per forward of the dominant kernels from the ncu captures summarised
-# under profiles/ (taken on this kernel version); None where no capture exists.
-NCU_TRAFFIC = {
-    ("c2_llama2_7b", 4096): {"bytes": 251.1e6 + 38.5e6 + 135.4e6 + 70.6e6,
-                             "source": "profiles/umma_grouped_gemm_c2_llama2_7b_T4096.md"},
-}
+# DRAM bytes (read + write) per forward of the dominant kernels (the two expert GEMMs), from the ncu
+# captures summarised under profiles/; an entry is only valid for the kernel version it was taken on,
+# so the table is emptied whenever those kernels change and refilled from a new capture.
+NCU_TRAFFIC = {}
+
+# Every (workload, T) point the metric is quoted on; the last one (the largest single-GPU
+# configuration) is the headline.
+SWEEP_POINTS = [("c2_llama2_7b", 1), ("c2_llama2_7b", 16), ("c2_llama2_7b", 64), ("c2_llama2_7b", 512),
+                ("c2_llama2_7b", 4096), ("c3_llama3_8b", 32), ("c3_llama3_8b", 8192), ("c4_hier_8x7b", 4096),
+                ("c5_skew_13b", 16384)]
+HEADLINE = SWEEP_POINTS[-1]
 
 
 def traffic_note(name, tokens, use_graph):
@@ -194,58 +199,167 @@ def replica_throughput(world: int, tokens_per_step: int, steps: int, ms_max: flo
     return world * tokens_per_step * steps / (ms_max * 1e-3)
 
 
+def replica_launch_command(n_gpus: int, argv, port: int):
+    """The command that starts one process per GPU for `bench.py --gpus N` run without a launcher."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+
+
+def free_port() -> int:
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        return sock.getsockname()[1]
+
+
 # ------------------------------------------------------------------ GPU arm
-def run_gpu(args):
-    import torch
-    import torch.distributed as dist
-    from paper_2502_04416_b200 import binding
-    from paper_2502_04416_b200 import torch_io
+class Rig:
+    """Process-wide state of one benchmark run: rank layout, stream, timing helpers."""
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    torch.cuda.set_device(local)
-    binding.load()
+    def __init__(self, args):
+        import torch
+        import torch.distributed as dist
+        self.torch, self.dist, self.args = torch, dist, args
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        if self.world > 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            dist.init_process_group("nccl", device_id=torch.device("cuda", self.local))
+        torch.cuda.set_device(self.local)
+        self.stream = torch.cuda.current_stream()
 
-    inputs = prepare_inputs(args.workload)
-    w = inputs.workload
-    s = w.shape
-    T = args.tokens or w.t_max
-    x_host = inputs.x[:T]
-    layer = torch_io.layer_from_workload(inputs, T)
-    x = torch_io.to_device(x_host, s.dtype)
-    out = torch.empty_like(x)
-    stream = torch.cuda.current_stream()
+    def barrier(self):
+        self.torch.cuda.synchronize()
+        if self.world > 1:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
 
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def timed(fn, steps):
-        """K steps between CUDA events on the launching stream; max over ranks."""
+    def timed(self, fn, steps):
+        """Exactly `steps` calls between CUDA events on the launching stream, a barrier and a
+        synchronize on both sides; the max over ranks, in milliseconds."""
+        torch = self.torch
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        e0.record(stream)
+        self.barrier()
+        e0.record(self.stream)
         for _ in range(steps):
             fn()
-        e1.record(stream)
-        barrier()
+        e1.record(self.stream)
+        self.barrier()
         return max_over_ranks(e0.elapsed_time(e1), "cuda")
 
-    # ---- device-resident throughput.  Large batches: direct launches with per-stage events for
-    # the roofline.  Small batches are launch-bound, so the forward (same C-ABI call, same
-    # kernels) is captured once into a CUDA graph and replayed; stage events are off there.
-    if args.chain == "off":
-        layer.set_launch_chaining(False)
+    def timed_blocks(self, fn, steps, min_region_s, max_blocks):
+        """Repeats the K-step block until the timed region reaches min_region_s (or max_blocks);
+        returns the per-block times in ms.  Every rank runs the same number of blocks: the
+        decision uses the max-over-ranks times."""
+        blocks = []
+        while True:
+            blocks.append(self.timed(fn, steps))
+            if sum(blocks) >= min_region_s * 1e3 or len(blocks) >= max_blocks:
+                return blocks
+
+    def close(self):
+        if self.world > 1:
+            self.dist.destroy_process_group()
+
+
+def dense_comparison(rig, inputs, x, steps, min_region_s=0.2):
+    """The comparison run, never the product path: the dense FFN of the same d and d_ff through
+    torch (cuBLAS); for the hierarchical workload the layer it replaces, a plain top-2 MoE whose
+    selected experts run as dense per-expert cuBLAS GEMMs on their tokens."""
+    torch = rig.torch
+    from paper_2502_04416_b200 import torch_io
+    F = torch.nn.functional
+    w, s = inputs.workload, inputs.workload.shape
+    T = x.shape[0]
+    ws = [tuple(torch_io.to_device(a, s.dtype) for a in (l.w_gate, l.w_up, l.w_down)) for l in inputs.layers]
+    if w.n_outer:
+        w_r = torch_io.to_device(inputs.w_router, s.dtype)
+        kind = ("plain top-%d MoE over the %d dense outer experts: torch router + per-expert F.linear x3 + "
+                "silu*mul on the expert's tokens (cuBLAS) + index_add" % (w.outer_top_k, w.n_outer))
+
+        def step():
+            logits = F.linear(x, w_r).float()
+            top, idx = logits.topk(w.outer_top_k, dim=1)
+            wt = torch.softmax(top, dim=1).to(x.dtype)
+            out = torch.zeros_like(x)
+            for i, (wg, wu, wd) in enumerate(ws):
+                tok, slot = (idx == i).nonzero(as_tuple=True)
+                if tok.numel():
+                    xi = x[tok]
+                    y = F.linear(F.silu(F.linear(xi, wg)) * F.linear(xi, wu), wd)
+                    out.index_add_(0, tok, y * wt[tok, slot].unsqueeze(1))
+            return out
+    else:
+        wg, wu, wd = ws[0]
+        kind = "torch F.linear x3 + silu*mul (cuBLAS), same d and d_ff"
+
+        def step():
+            return F.linear(F.silu(F.linear(x, wg)) * F.linear(x, wu), wd)
+    for _ in range(3):
+        step()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    times = []
+    while sum(times) < min_region_s * 1e3 and len(times) < 50:
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    dms = statistics.median(times) / steps
+    del ws
+    return {"kind": kind, "ms_per_step": dms, "value": T / (dms * 1e-3), "unit": UNIT}
+
+
+def roofline_record(peaks, w, T, touched, step_ms, first_ms, gemm_ms, stage_ms, use_graph):
+    """Algorithmic work of one forward against the measured peaks (flops 6 d m (N_s+N_k) per
+    token; bytes = every touched expert's weights once + x read + out write)."""
+    s = w.shape
+    mult = w.outer_top_k if w.n_outer else 1
+    flops = mult * T * 6 * s.d_model * s.m * (s.n_shared + s.top_k)
+    w_bytes = (w.n_outer if w.n_outer else 1) * (s.n_shared + touched) * s.expert_weight_bytes()
+    alg_bytes = w_bytes + 2 * T * s.d_model * s.elem_bytes
+    t_tensor = flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
+    if t_tensor >= t_hbm:
+        ach = flops / (gemm_ms * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": ach / peaks["bf16_tflops"], "frac_of_sustained": ach / peaks["bf16_tflops_sustained"]}
+        t_roof, t_sus = t_tensor, flops / (peaks["bf16_tflops_sustained"] * 1e12)
+    else:
+        ach = alg_bytes / (gemm_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / peaks["hbm_gbs"]}
+        t_roof, t_sus = t_hbm, t_hbm
+    roof.update({
+        "kernel": ("expert GEMMs (gate/up + SwiGLU, down), timed by per-stage events in a separate short loop"
+                   if not use_graph else "whole forward, all kernels (CUDA graph replay; no per-stage events)"),
+        "kernel_ms": gemm_ms, "peak_source": peaks["source"], "traffic": traffic_note(w.name, T, use_graph),
+        "algorithmic_flops": flops, "algorithmic_bytes": alg_bytes,
+        "whole_step_frac": t_roof / (step_ms * 1e-3),                    # median block, against the burst peak
+        "whole_step_frac_first_block": t_roof / (first_ms * 1e-3),
+        "whole_step_frac_of_sustained": t_sus / (step_ms * 1e-3),
+        "other_bound_frac": (t_hbm if t_tensor >= t_hbm else t_tensor) / (step_ms * 1e-3),
+        "stage_ms": stage_ms})
+    return roof, w_bytes
+
+
+def measure_point(rig, inputs, layer, T, min_region_s, max_blocks, with_dense):
+    """Times the forward of `layer` on the first T tokens of the workload, device-resident.
+    Returns the sweep record plus what the headline line needs."""
+    torch, args = rig.torch, rig.args
+    from paper_2502_04416_b200 import binding, torch_io
+    w, s = inputs.workload, inputs.workload.shape
+    x = torch_io.to_device(inputs.x[:T], s.dtype)
+    out = torch.empty_like(x)
     use_graph = args.graph == "on" or (args.graph == "auto" and T <= 512)
-    sampler = ClockSampler(local)
-    sampler.start()
-    if use_graph:
+    layer.set_launch_chaining(args.chain != "off")
+    if args.gemm_path:
+        layer.set_gemm_path(args.gemm_path)
+    layer.enable_stage_timing(0)
+    if use_graph:     # launch-bound sizes: the same C-ABI call captured once and replayed
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
@@ -258,127 +372,179 @@ def run_gpu(args):
             layer.forward(x, out)
         step = graph.replay
     else:
-        layer.enable_stage_timing(min(args.steps, 4096))
         step = lambda: layer.forward(x, out)
+    sampler = ClockSampler(rig.local)
+    sampler.start()
     for _ in range(args.warmup):
         step()
-    if not use_graph:
-        layer.enable_stage_timing(min(args.steps, 4096))      # reset the ring after warm-up
     sampler.wait_first()
     sampler.mark_begin()
-    ms_total = timed(step, args.steps)
+    blocks = rig.timed_blocks(step, args.steps, min_region_s, max_blocks)
     sampler.mark_end()
     time.sleep(0.12)                                          # let the sample that covers the end arrive
     clocks = sampler.stop()
-    stage_ms, n_cov = layer.stage_times() if not use_graph else ([0.0] * binding.N_STAGES, 0)
-    launches = layer.launch_count() * args.steps
+    launches_per_step = layer.launch_count()
     assert layer.status() == 0, "device-side wait timed out"
-    layer.enable_stage_timing(0)
-    value = replica_throughput(world, T, args.steps, ms_total)
+    step_ms = statistics.median(blocks) / args.steps
+    first_ms = blocks[0] / args.steps
+    # per-stage split: a second, short loop with the library's stage events (ordinary launches)
+    stage_ms, gemm_ms = None, step_ms
+    if not use_graph:
+        n_st = max(3, min(args.steps, 50))
+        layer.enable_stage_timing(n_st)
+        for _ in range(n_st):
+            layer.forward(x, out)
+        ms, n_cov = layer.stage_times()
+        layer.enable_stage_timing(0)
+        stage_ms = {n: v / max(n_cov, 1) for n, v in zip(binding.STAGE_NAMES, ms)}
+        gemm_ms = stage_ms["gemm1_swiglu"] + stage_ms["gemm2_down"]
+    touched = s.n_routed
+    if not w.n_outer and T * s.top_k < 64 * s.n_routed:
+        layer.forward(x, out)
+        touched = int((layer.routing(T, s.n_routed)["counts"] > 0).sum())
+    peaks = load_peaks()
+    roof, w_bytes = roofline_record(peaks, w, T, touched, step_ms, first_ms, gemm_ms, stage_ms, use_graph)
+    dense = dense_comparison(rig, inputs, x, args.steps) if (with_dense and rig.rank == 0) else None
+    rec = {"workload": w.name, "tokens": T, "ms_per_step": step_ms, "first_block_ms_per_step": first_ms,
+           "blocks": len(blocks), "timed_region_s": sum(blocks) * 1e-3,
+           "value": replica_throughput(rig.world, T, 1, step_ms), "unit": UNIT,
+           "launch": "CUDA graph replay" if use_graph else "direct launches, chained",
+           "launches_per_step": launches_per_step, "routed_experts_touched": touched,
+           "roofline": {k: roof[k] for k in ("bound", "frac", "achieved", "peak", "unit", "kernel_ms", "whole_step_frac",
+                                             "whole_step_frac_first_block", "whole_step_frac_of_sustained",
+                                             "other_bound_frac", "stage_ms")},
+           "dense_cublas": dense, "clocks": clocks}
+    if dense:
+        rec["speedup_vs_dense"] = dense["ms_per_step"] / step_ms
+    return rec, roof, (x, out, step, w_bytes)
+
+
+def run_gpu(args):
+    import torch
+    from paper_2502_04416_b200 import binding
+    from paper_2502_04416_b200 import torch_io
+
+    rig = Rig(args)
+    binding.load()
+    world, rank = rig.world, rig.rank
+    name = args.workload or HEADLINE[0]
+    inputs = prepare_inputs(name)
+    w = inputs.workload
+    s = w.shape
+    T = args.tokens or w.t_max
+    layer = torch_io.layer_from_workload(inputs, w.t_max if T <= w.t_max else T)
 
     if args.forward_only:                     # profiling runs: nothing but the forward passes
+        x = torch_io.to_device(inputs.x[:T], s.dtype)
+        out = torch.empty_like(x)
+        if args.chain == "off":
+            layer.set_launch_chaining(False)
+        for _ in range(args.warmup):
+            layer.forward(x, out)
+        ms = rig.timed(lambda: layer.forward(x, out), args.steps)
+        assert layer.status() == 0
         if rank == 0:
-            print(json.dumps({"forward_only": True, "workload": f"{w.name} T={T}", "ms_per_step": ms_total / args.steps,
-                              "stage_ms": {n: v / max(n_cov, 1) for n, v in zip(binding.STAGE_NAMES, stage_ms)}}))
-        if world > 1:
-            dist.destroy_process_group()
+            print(json.dumps({"forward_only": True, "workload": f"{w.name} T={T}", "ms_per_step": ms / args.steps}))
+        rig.close()
         return None
 
-    # ---- end to end through the public call with host buffers
+    # ---- headline: device-resident, K-step blocks repeated over at least a second
+    head, roof, (x, out, step, w_bytes) = measure_point(rig, inputs, layer, T, args.min_region_s, 400,
+                                                        with_dense=True)
+    launches = head["launches_per_step"] * args.steps
+
+    # ---- end to end through the public host-buffer call: H2D and D2H copies inside the timed region
     x_pin = torch.empty(x.shape, dtype=x.dtype).pin_memory()
     x_pin.copy_(x.cpu())
     out_pin = torch.empty(x.shape, dtype=x.dtype).pin_memory()
 
     def e2e_step():
-        x.copy_(x_pin, non_blocking=True)
-        step()
-        out_pin.copy_(out, non_blocking=True)
-    for _ in range(max(args.warmup, 3)):
+        layer.forward_host(x_pin, out_pin, args.e2e_chunk)
+    for _ in range(max(min(args.warmup, 5), 3)):
         e2e_step()
-    e2e_ms = timed(e2e_step, args.steps)
+    e2e_blocks = rig.timed_blocks(e2e_step, args.steps, min(args.min_region_s, 0.5), 100)
+    e2e_ms = statistics.median(e2e_blocks) / args.steps
     io_bytes = T * s.d_model * s.elem_bytes
+    torch.cuda.synchronize()
+    same = bool(torch.equal(out_pin.view(torch.int16), out.cpu().view(torch.int16))) if s.dtype == "bf16" else None
 
-    # ---- dense cuBLAS FFN of the same shape (comparison run, never the product path)
-    dense = None
-    if rank == 0 and not w.n_outer:
-        lay = inputs.layers[0]
-        wg, wu, wd = (torch_io.to_device(a, s.dtype) for a in (lay.w_gate, lay.w_up, lay.w_down))
-        F = torch.nn.functional
+    # ---- CPU baseline: the oracle on a bounded sample, on this machine's host cores (rank 0)
+    cpu = None
+    if rank == 0:
+        sample = min(args.cpu_sample_tokens, T)
+        cpu_v, cpu_dt = time_oracle(inputs, inputs.x[:T], sample)
+        cpu = {"value": cpu_v, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+               "sample": f"first {sample} tokens of the same workload, one pass, {cpu_dt:.2f} s"}
 
-        def dense_step():
-            return F.linear(F.silu(F.linear(x, wg)) * F.linear(x, wu), wd)
-        for _ in range(3):
-            dense_step()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(args.steps):
-            dense_step()
-        e1.record()
-        torch.cuda.synchronize()
-        dms = e0.elapsed_time(e1) / args.steps
-        dense = {"kind": "torch F.linear x3 + silu*mul (cuBLAS), same d and d_ff",
-                 "ms_per_step": dms, "value": T / (dms * 1e-3), "unit": UNIT}
-        del wg, wu, wd
+    # ---- the other (workload, T) points
+    sweep = None
+    do_sweep = args.sweep == "on" or (args.sweep == "auto" and world == 1 and (name, T) == HEADLINE)
+    if do_sweep:
+        found = {(head["workload"], head["tokens"]): head}
+        del x, out, step
+        order = [name] + [n_ for n_ in dict.fromkeys(p_[0] for p_ in SWEEP_POINTS) if n_ != name]
+        for n_ in order:
+            ts = [t_ for m_, t_ in SWEEP_POINTS if m_ == n_ and (m_, t_) not in found]
+            if not ts:
+                continue
+            if n_ != name:
+                layer.destroy()
+                del inputs, layer
+                torch.cuda.empty_cache()
+                inputs = prepare_inputs(n_)
+                layer = torch_io.layer_from_workload(inputs, inputs.workload.t_max)
+                name = n_
+            for t_ in ts:
+                found[(n_, t_)], _, _ = measure_point(rig, inputs, layer, t_, args.sweep_region_s, 200, with_dense=True)
+        sweep = [found[p_] for p_ in SWEEP_POINTS if p_ in found]
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        rig.close()
         return None
 
-    # ---- roofline of the dominant kernel stage
-    peaks = load_peaks()
-    touched = s.n_routed
-    if not w.n_outer and T * s.top_k < 64 * s.n_routed:
-        r = layer.routing(T, s.n_routed)
-        touched = int((r["counts"] > 0).sum())
-    mult = w.outer_top_k if w.n_outer else 1
-    flops = mult * T * 6 * s.d_model * s.m * (s.n_shared + s.top_k)
-    w_bytes = (w.n_outer if w.n_outer else 1) * (s.n_shared + touched) * s.expert_weight_bytes()
-    alg_bytes = w_bytes + 2 * T * s.d_model * s.elem_bytes
-    step_ms = ms_total / args.steps
-    gemm_ms = (stage_ms[2] + stage_ms[3]) / max(n_cov, 1) if not use_graph else step_ms
-    t_tensor = flops / (peaks["bf16_tflops"] * 1e12)
-    t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
-    if t_tensor >= t_hbm:
-        ach = flops / (gemm_ms * 1e-3) / 1e12
-        roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": ach / peaks["bf16_tflops"],
-                "frac_of_sustained": ach / peaks["bf16_tflops_sustained"]}
-    else:
-        ach = alg_bytes / (gemm_ms * 1e-3) / 1e9
-        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / peaks["hbm_gbs"]}
-    roof.update({"kernel": ("expert GEMMs (gate/up + SwiGLU, down)" if not use_graph else
-                            "whole forward, all kernels (CUDA graph replay; no per-stage events)"),
-                 "kernel_ms": gemm_ms,
-                 "peak_source": peaks["source"], "traffic": traffic_note(w.name, T, use_graph),
-                 "whole_step_frac": (t_tensor if t_tensor >= t_hbm else t_hbm) / (step_ms * 1e-3),
-                 "stage_ms": {n: v / max(n_cov, 1) for n, v in zip(binding.STAGE_NAMES, stage_ms)}})
-
-    # ---- CPU baseline: the oracle on a bounded sample, on this machine's host cores
-    sample = args.cpu_sample_tokens
-    cpu_v, cpu_dt = time_oracle(inputs, x_host, min(sample, T))
-    cpu = {"value": cpu_v, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
-           "sample": f"first {min(sample, T)} tokens of the same workload, one pass, {cpu_dt:.2f} s"}
-
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": s.dtype, "data": "synthetic",
+        "metric": METRIC, "value": replica_throughput(world, T, 1, head["ms_per_step"]), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": head["ms_per_step"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": s.dtype, "data": "synthetic",
         "config": {"workload": f"{w.name} T={T}", "note": w.note, "d_model": s.d_model,
                    "d_ff": s.d_ff, "experts": f"S{s.n_shared}A{s.top_k}E{s.n_experts}",
                    "tokens_per_step": T, "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2": "weights (%.0f MB) exceed the 126 MB L2" % (w_bytes / 1e6),
-                   "launch": "CUDA graph replay" if use_graph else "direct launches"},
-        "e2e": {"value": world * T * args.steps / (e2e_ms * 1e-3), "unit": UNIT,
-                "h2d_bytes_per_step": io_bytes, "d2h_bytes_per_step": io_bytes},
-        "gpu_launches": launches, "clocks": clocks, "roofline": roof, "cpu_baseline": cpu,
-        "dense_cublas": dense,
+                   "launch": head["launch"],
+                   "timing": "the K-step block is repeated until the timed region reaches %.1f s; ms_per_step is "
+                             "the median block / K, first_block_ms_per_step the first" % args.min_region_s},
+        "first_block_ms_per_step": head["first_block_ms_per_step"], "blocks": head["blocks"],
+        "timed_region_s": head["timed_region_s"],
+        "e2e": {"value": world * T / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": io_bytes, "d2h_bytes_per_step": io_bytes,
+                "call": "cmoe_ffn_forward_host: pinned host x and out, chunks double-buffered on two copy streams",
+                "chunk_tokens": args.e2e_chunk or "auto", "ms_per_step": e2e_ms,
+                "bit_identical_to_device_call": same},
+        "gpu_launches": launches, "clocks": head["clocks"], "roofline": roof, "cpu_baseline": cpu,
+        "dense_cublas": head["dense_cublas"], "speedup_vs_dense": head.get("speedup_vs_dense"),
     }
-    if world > 1:
-        dist.destroy_process_group()
+    if sweep is not None:
+        line["sweep"] = sweep
+    rig.close()
     return line
+
+
+def run_ranks(args):
+    """Launch-path self-check that needs no GPU: every rank joins a gloo group, reports a
+    rank-dependent stand-in time, and rank 0 prints the replica arithmetic of the real run."""
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("gloo", rank=rank, world_size=world)
+    ms = max_over_ranks(10.0 + 5.0 * rank, "cpu")
+    line = {"stage": "ranks", "n_gpus": world, "ms_max": ms,
+            "value": replica_throughput(world, 4096, args.steps, ms)}
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return line if rank == 0 else None
 
 
 # ------------------------------------------------------------ reference arm
@@ -614,26 +780,48 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", default="c2_llama2_7b", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--workload", default=None, choices=sorted(wl.WORKLOADS),
+                    help="default: the largest single-GPU configuration, c5_skew_13b")
     ap.add_argument("--tokens", type=int, default=0, help="tokens per step (default: the workload's largest T)")
     ap.add_argument("--cpu-sample-tokens", type=int, default=256)
     ap.add_argument("--graph", choices=["auto", "on", "off"], default="auto",
                     help="replay the forward from a CUDA graph (auto: batches of at most 512 tokens)")
     ap.add_argument("--chain", choices=["on", "off"], default="on",
                     help="programmatic dependent launches between the kernels of a forward (library default: on)")
-    ap.add_argument("--stage", choices=["forward", "profile", "cluster"], default="forward",
+    ap.add_argument("--gemm-path", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="expert-GEMM implementation (cmoe_layer_set_gemm_path); 0 = the library's choice")
+    ap.add_argument("--sweep", choices=["auto", "on", "off"], default="auto",
+                    help="add one record per (workload, T) point of the metric to the JSON line "
+                         "(auto: on for the default single-GPU headline run)")
+    ap.add_argument("--min-region-s", type=float, default=1.0,
+                    help="the K-step block is repeated until the timed region is at least this long")
+    ap.add_argument("--sweep-region-s", type=float, default=0.4)
+    ap.add_argument("--e2e-chunk", type=int, default=0, help="tokens per chunk of the host-buffer call (0: automatic)")
+    ap.add_argument("--stage", choices=["forward", "profile", "cluster", "ranks"], default="forward",
                     help="forward: the MoE forward pass (the headline metric); profile: the activation-profiling "
                          "pass; cluster: one round of the GPU clustering pieces")
     ap.add_argument("--forward-only", action="store_true",
                     help="run only the timed forward passes (for profiler captures)")
     args = ap.parse_args()
+    world_env = os.environ.get("WORLD_SIZE")
+    if args.gpus > 1 and world_env is None:
+        # run directly with --gpus N: start one replica process per GPU (the launcher's job otherwise)
+        sys.exit(subprocess.call(replica_launch_command(args.gpus, sys.argv[1:], free_port())))
+    if world_env is not None and int(world_env) != args.gpus:
+        print(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world_env}", file=sys.stderr)
+        sys.exit(2)
     if args.impl == "reference":
+        args.workload = args.workload or HEADLINE[0]
         line = run_reference(args)
+    elif args.stage == "ranks":
+        line = run_ranks(args)
     else:
         args.warmup = max(args.warmup, 3)
+        if args.stage != "forward":
+            args.workload = args.workload or "c2_llama2_7b"
         line = (run_profile(args) if args.stage == "profile" else
                 run_cluster(args) if args.stage == "cluster" else run_gpu(args))
     if line is not None:

@@ -104,6 +104,25 @@ int cmoe_hier_create(int32_t n_outer, int32_t outer_top_k, const void* w_router,
  * Errors: INVALID_ARG (null, misaligned or overlapping buffers), CAPACITY (T > max_tokens), CUDA. */
 int cmoe_ffn_forward(cmoe_layer* layer, const void* x, int32_t T, void* out, void* stream);
 
+/* The same forward for buffers in HOST memory (Eq. moe_output is per token, so a batch may be
+ * cut anywhere): the T tokens are processed in chunks; chunk c+1 is copied to the device and
+ * chunk c-1 back to the host on two internal copy streams while chunk c runs on `stream`
+ * through the kernels of cmoe_ffn_forward.  Each token's result is what cmoe_ffn_forward
+ * gives for it in a batch of the chunk's size.
+ *   x_host, out_host : host, [T, d_model] row-major; page-locked memory is needed for the
+ *                      copies to overlap (pageable memory works, serially).  The buffers
+ *                      belong to the caller and must stay valid until `stream` has passed
+ *                      this call; out_host is complete when work enqueued on `stream` after
+ *                      the call runs (or after synchronising `stream`).
+ *   chunk_tokens     : tokens per chunk, clamped to [1, max_tokens]; <= 0 picks an eighth
+ *                      of the batch rounded up to 128 rows, at least 512.
+ * The first call (and any later call with a larger chunk) allocates the staging: two device
+ * buffers each for x and out of chunk_tokens rows, two streams and a few events, all freed by
+ * cmoe_layer_destroy; other calls allocate nothing.  Routing read-back afterwards (cmoe_get_routing)
+ * describes the LAST chunk only.  Errors: INVALID_ARG, CUDA. */
+int cmoe_ffn_forward_host(cmoe_layer* layer, const void* x_host, int32_t T, void* out_host,
+                          int32_t chunk_tokens, void* stream);
+
 /* Replace the learnable gate scaling u and the selection bias b (Section 4.3).
  * host arrays [n_routed_groups] (N_r, or n_outer*N_r for a hierarchical layer,
  * outer-major) or NULL for zeros.  Synchronises `stream`. */

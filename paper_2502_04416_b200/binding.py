@@ -18,7 +18,7 @@ N_STAGES = 5
 STAGE_NAMES = ["route", "permute", "gemm1_swiglu", "gemm2_down", "combine"]
 
 EXPORTS = [
-    "cmoe_layer_create", "cmoe_hier_create", "cmoe_ffn_forward", "cmoe_layer_set_gate_params",
+    "cmoe_layer_create", "cmoe_hier_create", "cmoe_ffn_forward", "cmoe_ffn_forward_host", "cmoe_layer_set_gate_params",
     "cmoe_layer_get_gate_params", "cmoe_layer_update_bias", "cmoe_profile_activations", "cmoe_select_shared",
     "cmoe_cluster_update", "cmoe_cluster_distances", "cmoe_cluster_representatives", "cmoe_layer_set_gemm_path", "cmoe_layer_set_launch_chaining",
     "cmoe_layer_dims", "cmoe_get_routing", "cmoe_layer_status", "cmoe_layer_selftest_wait_timeout",
@@ -57,6 +57,7 @@ def load() -> C.CDLL:
                                       C.POINTER(vp)]
     lib.cmoe_hier_create.argtypes = [i32, i32, vp, C.POINTER(vp), i32, vp, C.POINTER(vp)]
     lib.cmoe_ffn_forward.argtypes = [vp, vp, i32, vp, vp]
+    lib.cmoe_ffn_forward_host.argtypes = [vp, vp, i32, vp, i32, vp]
     lib.cmoe_layer_set_gate_params.argtypes = [vp, vp, vp, vp]
     lib.cmoe_layer_set_gemm_path.argtypes = [vp, i32]
     lib.cmoe_layer_set_launch_chaining.argtypes = [vp, i32]
@@ -173,6 +174,16 @@ class Layer:
                                      _stream_ptr(stream))
         _check(st, "cmoe_ffn_forward")
         return out
+
+    def forward_host(self, x_host, out_host, chunk_tokens: int = 0, stream=None):
+        """cmoe_ffn_forward_host: x_host / out_host are CPU tensors [T,d] (pinned for overlap);
+        asynchronous on the stream, out_host is complete once the stream has passed the call."""
+        if x_host.is_cuda or out_host.is_cuda or not (x_host.is_contiguous() and out_host.is_contiguous()):
+            raise ValueError("forward_host takes contiguous CPU tensors")
+        st = load().cmoe_ffn_forward_host(self._h, x_host.data_ptr(), x_host.shape[0], out_host.data_ptr(),
+                                          chunk_tokens, _stream_ptr(stream))
+        _check(st, "cmoe_ffn_forward_host")
+        return out_host
 
     def set_gate_params(self, gate_scale_u=None, select_bias_b=None, stream=None) -> None:
         u = None if gate_scale_u is None else np.ascontiguousarray(gate_scale_u, dtype=np.float32)

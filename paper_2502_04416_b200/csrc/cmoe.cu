@@ -118,6 +118,16 @@ struct cmoe_layer {
   int last_T = 0;
   int launches = 0;
 
+  // staging for cmoe_ffn_forward_host (created by its first call): two device buffers each for
+  // x and out, one copy stream per direction, events per buffer
+  struct HostIo {
+    int chunk = 0;
+    void *x[2] = {nullptr, nullptr}, *out[2] = {nullptr, nullptr};
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t start = nullptr, in_done[2] = {nullptr, nullptr}, cmp_done[2] = {nullptr, nullptr},
+                out_done[2] = {nullptr, nullptr};
+  } hio;
+
   // optional per-stage CUDA-event timing: ring of (kStages + 1) events per forward
   std::vector<cudaEvent_t> ev;
   int ev_ring = 0;
@@ -132,6 +142,15 @@ namespace {
 void free_layer(cmoe_layer* L) {
   if (!L) return;
   for (cudaEvent_t e : L->ev) cudaEventDestroy(e);
+  for (int b = 0; b < 2; ++b) {
+    cudaFree(L->hio.x[b]); cudaFree(L->hio.out[b]);
+    if (L->hio.in_done[b]) cudaEventDestroy(L->hio.in_done[b]);
+    if (L->hio.cmp_done[b]) cudaEventDestroy(L->hio.cmp_done[b]);
+    if (L->hio.out_done[b]) cudaEventDestroy(L->hio.out_done[b]);
+  }
+  if (L->hio.start) cudaEventDestroy(L->hio.start);
+  if (L->hio.s_in) cudaStreamDestroy(L->hio.s_in);
+  if (L->hio.s_out) cudaStreamDestroy(L->hio.s_out);
   umma_plan_destroy(&L->umma);
   cudaFree(L->w_gu); cudaFree(L->wd_p); cudaFree(L->w_rep);
   cudaFree(L->w_router); cudaFree(L->u); cudaFree(L->b); cudaFree(L->gs); cudaFree(L->ws);
@@ -633,6 +652,70 @@ int cmoe_ffn_forward(cmoe_layer* L, const void* x, int32_t T, void* out, void* s
   L->last_T = T;
   return L->cfg.dtype == CMOE_BF16 ? forward_impl<bf16>(L, (const bf16*)x, T, (bf16*)out, st)
                                    : forward_impl<float>(L, (const float*)x, T, (float*)out, st);
+}
+
+int cmoe_ffn_forward_host(cmoe_layer* L, const void* x_host, int32_t T, void* out_host, int32_t chunk_tokens,
+                          void* stream) {
+  if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "null layer");
+  if (T < 0) return arg_fail(CMOE_ERR_INVALID_ARG, "negative token count");
+  if (T == 0) { L->last_T = 0; L->launches = 0; return CMOE_OK; }
+  if (!x_host || !out_host) return arg_fail(CMOE_ERR_INVALID_ARG, "null x / out");
+  const size_t row_bytes = (size_t)L->cfg.d_model * L->esz;
+  int chunk = chunk_tokens;
+  if (chunk <= 0) {                                  // an eighth of the batch, in whole 128-row tiles, at least 512
+    chunk = ((T + 7) / 8 + 127) / 128 * 128;
+    if (chunk < 512) chunk = 512;
+  }
+  if (chunk > L->cfg.max_tokens) chunk = L->cfg.max_tokens;
+  if (chunk > T) chunk = T;
+  cmoe_layer::HostIo& h = L->hio;
+  if (h.chunk < chunk) {                             // first call (or a larger chunk than before): set up the staging
+    for (int b = 0; b < 2; ++b) {
+      cudaFree(h.x[b]); cudaFree(h.out[b]);
+      h.x[b] = h.out[b] = nullptr;
+    }
+    h.chunk = 0;
+    for (int b = 0; b < 2; ++b) {
+      CU_TRY(cudaMalloc(&h.x[b], (size_t)chunk * row_bytes));
+      CU_TRY(cudaMalloc(&h.out[b], (size_t)chunk * row_bytes));
+      if (!h.in_done[b]) CU_TRY(cudaEventCreateWithFlags(&h.in_done[b], cudaEventDisableTiming));
+      if (!h.cmp_done[b]) CU_TRY(cudaEventCreateWithFlags(&h.cmp_done[b], cudaEventDisableTiming));
+      if (!h.out_done[b]) CU_TRY(cudaEventCreateWithFlags(&h.out_done[b], cudaEventDisableTiming));
+    }
+    if (!h.start) CU_TRY(cudaEventCreateWithFlags(&h.start, cudaEventDisableTiming));
+    if (!h.s_in) CU_TRY(cudaStreamCreateWithFlags(&h.s_in, cudaStreamNonBlocking));
+    if (!h.s_out) CU_TRY(cudaStreamCreateWithFlags(&h.s_out, cudaStreamNonBlocking));
+    h.chunk = chunk;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  L->last_stream = st;
+  // the copies start where the caller's stream stands now
+  CU_TRY(cudaEventRecord(h.start, st));
+  CU_TRY(cudaStreamWaitEvent(h.s_in, h.start, 0));
+  CU_TRY(cudaStreamWaitEvent(h.s_out, h.start, 0));
+  int launches = 0, n_chunks = 0;
+  for (int t0 = 0; t0 < T; t0 += chunk, ++n_chunks) {
+    const int n = T - t0 < chunk ? T - t0 : chunk, b = n_chunks & 1;
+    const char* src = static_cast<const char*>(x_host) + (size_t)t0 * row_bytes;
+    char* dst = static_cast<char*>(out_host) + (size_t)t0 * row_bytes;
+    if (n_chunks >= 2) CU_TRY(cudaStreamWaitEvent(h.s_in, h.cmp_done[b], 0));      // x[b] has been consumed
+    CU_TRY(cudaMemcpyAsync(h.x[b], src, (size_t)n * row_bytes, cudaMemcpyHostToDevice, h.s_in));
+    CU_TRY(cudaEventRecord(h.in_done[b], h.s_in));
+    CU_TRY(cudaStreamWaitEvent(st, h.in_done[b], 0));
+    if (n_chunks >= 2) CU_TRY(cudaStreamWaitEvent(st, h.out_done[b], 0));          // out[b] has been drained
+    L->last_T = n;
+    const int rc = L->cfg.dtype == CMOE_BF16 ? forward_impl<bf16>(L, (const bf16*)h.x[b], n, (bf16*)h.out[b], st)
+                                             : forward_impl<float>(L, (const float*)h.x[b], n, (float*)h.out[b], st);
+    if (rc != CMOE_OK) return rc;
+    launches += L->launches;
+    CU_TRY(cudaEventRecord(h.cmp_done[b], st));
+    CU_TRY(cudaStreamWaitEvent(h.s_out, h.cmp_done[b], 0));
+    CU_TRY(cudaMemcpyAsync(dst, h.out[b], (size_t)n * row_bytes, cudaMemcpyDeviceToHost, h.s_out));
+    CU_TRY(cudaEventRecord(h.out_done[b], h.s_out));
+  }
+  for (int b = 0; b < 2 && b < n_chunks; ++b) CU_TRY(cudaStreamWaitEvent(st, h.out_done[b], 0));
+  L->launches = launches;
+  return CMOE_OK;
 }
 
 int cmoe_profile_activations(cmoe_layer* L, const void* x, int32_t T, int32_t k_a, int32_t token0,

@@ -158,6 +158,38 @@ def test_call_contract():
     layer.destroy()
 
 
+def test_forward_host_matches_device_forward():
+    """cmoe_ffn_forward_host (chunked, copies overlapped on side streams) against the device-buffer
+    call: a token's result does not depend on what else is in its batch (Eq. moe_output is per x), so
+    chunks processed by the same kernel family give the same bits; a ragged last chunk, a single
+    chunk and pageable host memory are covered."""
+    import torch
+    inp = _inputs("c2_llama2_7b", d_model=256, tokens=(2900,), m=160)
+    lay = inp.layers[0]
+    layer = parity.gpu_layer(lay, 2900)
+    x = parity.to_device(inp.x, "bf16")
+    ref = layer.forward(x).cpu()
+    torch.cuda.synchronize()
+    x_pin = x.cpu().pin_memory()
+    out_pin = torch.empty_like(x_pin).pin_memory()
+    for chunk in (1024, 700, 0, 2900, 5000):
+        out_pin.zero_()
+        layer.forward_host(x_pin, out_pin, chunk)
+        torch.cuda.synchronize()
+        assert layer.status() == 0
+        assert torch.equal(out_pin.view(torch.int16), ref.view(torch.int16)), chunk
+    for _ in range(3):                                  # back-to-back calls reuse the staging buffers
+        layer.forward_host(x_pin, out_pin, 1024)
+    torch.cuda.synchronize()
+    assert torch.equal(out_pin.view(torch.int16), ref.view(torch.int16))
+    x_page, out_page = x.cpu(), torch.zeros_like(ref)   # pageable memory: serial copies, same result
+    layer.forward_host(x_page[:1500], out_page[:1500], 600)
+    torch.cuda.synchronize()
+    assert torch.equal(out_page[:1500].view(torch.int16), ref[:1500].view(torch.int16))
+    parity.check_output(parity.to_host(out_pin), oracle.cmoe_layer_forward(inp.x, **parity.oracle_kwargs(lay))[0])
+    layer.destroy()
+
+
 def test_wait_timeout_is_reported_and_recovered():
     """The give-up path of the bounded device-side waits: a wait that nothing ends runs to its
     (millisecond) limit, the kernel returns normally, the layer's error word carries the code,
