@@ -351,7 +351,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
   // Plain bf16 layers on the tensor path chain their kernels by programmatic dependent launch
   // (every kernel after the router may become resident early and waits on the device for its
   // predecessor); per-stage events, the hierarchical prologue and CTA pairs use ordinary launches.
-  const bool dep = use_umma && !L->hier && !ev && L->gemm_path != 3 && L->chain_launches;
+  const bool dep = use_umma && !L->hier && !ev && L->chain_launches;
 
   if (L->hier) {
     if constexpr (std::is_same<T, bf16>::value) {
@@ -420,22 +420,51 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
     ++launches;
   }
   // The tensor path gathers routed rows inside the gate/up GEMM (decode: not at all; a few rows:
-  // TMA gather4; otherwise cp.async by dedicated warps); only CTA pairs and the SIMT path read a
-  // permuted copy of x.
-  const bool pairs = use_umma && !decode && R >= kPairMinRows && L->gemm_path == 3;
+  // TMA gather4; otherwise cp.async by dedicated warps); only the SIMT path reads a permuted copy of x.
+  // CTA pairs (cta_group::2, 256-row tiles) move a third less operand data per flop but round every
+  // group up to an even number of 128-row tiles.  Path 3 forces them; the automatic choice takes them
+  // per GEMM when the padding expected for evenly loaded experts stays small (thresholds measured on
+  // the paper-shaped workloads: the down GEMM gains more from pairs than the gate/up GEMM, except
+  // when its K extent, the expert width, is only a few k blocks).
+  int pair_mask = 0;                               // bit 0: gate/up on pairs, bit 1: down on pairs
+  if (use_umma && !decode && R >= kPairMinRows) {
+    if (L->gemm_path == 3) {
+      pair_mask = 3;
+    } else if (L->gemm_path == 0) {
+      auto pad = [](double rows) {                 // tile slots on pairs / tiles on single CTAs
+        const int mt = (int)((rows + 127) / 128);
+        return mt > 0 ? (double)(2 * ((mt + 1) / 2)) / mt : 1.0;
+      };
+      const double rows_s = (double)R / L->n_outer, rows_r = G > 0 ? (double)P / G : 0.0;
+      const double w_s = (double)R * L->cfg.n_shared, w_r = (double)P;
+      const double ratio = (w_s + w_r) > 0 ? (pad(rows_s) * w_s + pad(rows_r) * w_r) / (w_s + w_r) : 1.0;
+      if (ratio <= 1.03) pair_mask |= 1;
+      if (ratio <= 1.08 && L->m >= 512) pair_mask |= 2;
+    }
+  }
   const int gather_mode = P <= kTmaGatherMaxRows ? 1 : 2;
-  if (P > 0 && (!use_umma || pairs)) {
+  if (P > 0 && !use_umma) {
     gather_rows_kernel<<<P, 256, 0, st>>>((const uint4*)xo, L->row_token, P, row_vec, (uint4*)L->x_perm);
     ++launches;
   }
 
   mark(2);
   if (use_umma) {
-    // CTA pairs (cta_group::2, 256-row tiles) on request: measured equal to single-CTA tiles on
-    // even groups and slower on ragged ones (an odd m-tile count idles half a pair)
-    const int n = decode ? decode_forward(&L->umma, &L->decode, L->gr, R, L->err_word, st, ev ? ev[3] : nullptr, dep, gate_up_only)
-                : pairs  ? umma2_forward(&L->umma, &L->pair, &L->decode, L->gr, L->err_word, st, ev ? ev[3] : nullptr)
-                         : umma_forward(&L->umma, L->gr, gather_mode, xo, L->err_word, st, ev ? ev[3] : nullptr, dep, gate_up_only);
+    cudaEvent_t mid = ev ? ev[3] : nullptr;
+    int n;
+    if (decode) {
+      n = decode_forward(&L->umma, &L->decode, L->gr, R, L->err_word, st, mid, dep, gate_up_only);
+    } else {
+      const int todo = gate_up_only ? 1 : 3;
+      n = 0;
+      for (int bit = 1; bit <= 2 && n >= 0; bit <<= 1) {          // gate/up, then down, each on its chosen tile shape
+        if (!(todo & bit)) continue;
+        const int k = (pair_mask & bit)
+            ? umma2_forward(&L->umma, &L->pair, &L->decode, L->gr, 2, xo, L->err_word, st, mid, dep, bit)
+            : umma_forward(&L->umma, L->gr, gather_mode, xo, L->err_word, st, mid, dep, bit);
+        n = k < 0 ? -1 : n + k;
+      }
+    }
     if (n < 0) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
     launches += n;
   } else {

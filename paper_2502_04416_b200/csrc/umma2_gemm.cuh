@@ -10,10 +10,18 @@
 //   MODE 2, down:    each CTA stages 128 of the tile's 256 output channels.
 // The two 128-row halves are two m-tiles of the same group and n-tile; a group with an odd
 // number of m-tiles leaves one half computing rows that are never stored.
+// Routed groups of the gate/up GEMM gather their A rows straight from x (no permuted copy):
+// four extra warps per CTA copy the CTA's 128 rows of each k block with 16-byte cp.async into the
+// swizzled layout and arrive, copy-completion-bound, on a barrier of their own CTA; a relay
+// thread per CTA forwards each completed block to the leader's full barrier.  (Waiting for the
+// copies in the gather threads themselves, cp.async.wait_group + proxy fence per block, drained
+// the copies in flight at every block and ran three times slower.)
 //
 // Synchronisation (all waits bounded):
 //   full[s]      leader's barrier; the leader's producer arrives with the byte count of BOTH
-//                CTAs' copies, and both CTAs' TMA copies complete on it.
+//                CTAs' TMA copies, which complete on it; in the gate/up kernel each CTA's relay
+//                thread arrives on it as well (2 more arrivals).
+//   afull[s]     gate/up only, one per CTA: its 128 gather threads, then its relay waits on it.
 //   empty[s]     one per CTA; the leader's tcgen05.commit is multicast to both.
 //   acc_full[b]  one per CTA, multicast commit;  acc_empty[b]: leader's, 8 arrivals (the
 //                four epilogue warps of each CTA, the peer's arriving remotely).
@@ -29,6 +37,7 @@ constexpr int kU2ABytes = kUmmaBM * kUmmaBK * 2;        // 16 KB: this CTA's 128
 constexpr int kU2BBytes = 128 * kUmmaBK * 2;            // 16 KB: this CTA's half of B
 constexpr int kU2StageBytes = kU2ABytes + kU2BBytes;
 constexpr int kU2SmemBytes = 1024 + kU2Stages * kU2StageBytes + 256 + (kUmmaMaxGroups + 1) * 4;
+constexpr int kU2Threads1 = kUmmaThreads + kUmmaGatherThreads + 32;   // gate/up: + 4 gather warps + 1 relay warp
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -43,6 +52,13 @@ __device__ __forceinline__ uint32_t mapa_shared(uint32_t local, uint32_t rank) {
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Arrive on a barrier of a cluster CTA with the default (CTA-scope release) semantics: the data
+// the arrival stands for was written by cp.async and fenced towards the async proxy, and is read
+// only by tcgen05.mma.  (Cluster-scope acquire / release on this per-k-block path cost more than
+// the MMAs of the block.)
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
@@ -119,10 +135,12 @@ __device__ __forceinline__ Pair2Coord umma2_decode(const UmmaArgs& p, const int3
 }
 
 template <int MODE>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kUmmaThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MODE == 1 ? kU2Threads1 : kUmmaThreads, 1)
 umma2_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_constant__ CUtensorMap tm_a_r,
                      const __grid_constant__ CUtensorMap tm_b_s, const __grid_constant__ CUtensorMap tm_b_r,
                      const UmmaArgs p) {
+  grid_dep_wait();
+  grid_dep_trigger();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -130,7 +148,7 @@ umma2_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_co
   const uint32_t bars = base + kU2Stages * kU2StageBytes;
   uint8_t* bars_gen = gen + kU2Stages * kU2StageBytes;
   // barrier block: full[8] empty[8] acc_full[2] acc_empty[2], tmem slot, abort flag
-  const uint32_t full0 = bars, empty0 = bars + 64, accf0 = bars + 128, acce0 = bars + 144;
+  const uint32_t full0 = bars, empty0 = bars + 64, accf0 = bars + 128, acce0 = bars + 144, afull0 = bars + 192;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_gen + 160);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
   int32_t* tile_start = reinterpret_cast<int32_t*>(bars_gen + 256);
@@ -141,7 +159,10 @@ umma2_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_co
   const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kU2Stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    const uint32_t full_count = MODE == 1 ? 3 : 1;      // gate/up: plus one relay arrival per CTA
+    for (int s = 0; s < kU2Stages; ++s) {
+      mbar_init(full0 + 8 * s, full_count); mbar_init(empty0 + 8 * s, 1); mbar_init(afull0 + 8 * s, kUmmaGatherThreads);
+    }
     for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 8); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -177,6 +198,7 @@ umma2_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_co
         const int row = c.row0 + (2 * c.mp + (int)rank) * kUmmaBM;     // this CTA's m-tile
         const CUtensorMap* ta = g.is_shared ? &tm_a_s : &tm_a_r;
         const CUtensorMap* tb = g.is_shared ? &tm_b_s : &tm_b_r;
+        const bool by_threads = MODE == 1 && !g.is_shared && p.use_gather == 2;   // the gather warps fill A
         int k_blocks, b_half, b_row, j = 0;
         if (MODE == 1) {
           const int bn = g.is_shared ? p.bn_s : p.bn_r;
@@ -195,8 +217,8 @@ umma2_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_co
           const uint32_t fb_local = full0 + 8 * s;
           const uint32_t fb = mapa_shared(fb_local, 0);               // the leader's barrier
           const uint32_t sa = base + s * kU2StageBytes, sb = sa + kU2ABytes;
-          if (leader) mbar_expect_tx(fb_local, 2 * (kU2ABytes + b_half));
-          tma2_load_2d(sa, ta, fb, kb * kUmmaBK, row);
+          if (leader) mbar_expect_tx(fb_local, 2 * ((by_threads ? 0 : kU2ABytes) + b_half));
+          if (!by_threads) tma2_load_2d(sa, ta, fb, kb * kUmmaBK, row);
           if (MODE == 1) tma2_load_3d(sb, tb, fb, kb * kUmmaBK, b_row, (int)rank);   // plane 0 gate, 1 up
           else if (g.is_shared) tma2_load_3d(sb, tb, fb, kb * kUmmaBK, b_row, g.outer);
           else tma2_load_4d(sb, tb, fb, kb * kUmmaBK, b_row, j, g.outer);
@@ -223,6 +245,7 @@ umma2_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_co
         for (int kb = 0; kb < k_blocks; ++kb, ++it) {
           const uint32_t s = it % kU2Stages, n = it / kU2Stages;
           if (!mbar_wait(full0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
+          if (MODE == 1) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           tc_fence_after();
           const uint32_t sa = base + s * kU2StageBytes, sb = sa + kU2ABytes;
 #pragma unroll
@@ -234,6 +257,67 @@ umma2_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_co
         if (ok) umma2_commit_both(accf0 + 8 * buf);
       }
     }
+  } else if (MODE == 1 && warp == 10) {
+    // ------------------------------------------------------------ relay (gate/up, warp 10, both CTAs)
+    // Waits until this CTA's 128 gather threads have landed a k block (local barrier), fences
+    // those generic-proxy writes towards the async proxy and arrives on the leader's full barrier.
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = pair_id; t < total_tiles && ok; t += n_pairs) {
+        for (int kb = 0; kb < k_blocks_fixed; ++kb, ++it) {
+          const uint32_t s = it % kU2Stages, n = it / kU2Stages;
+          if (!mbar_wait(afull0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          mbar_arrive_remote(mapa_shared(full0 + 8 * s, 0));
+        }
+      }
+    }
+  } else if (MODE == 1 && warp >= 6) {
+    // ------------------------------------------------------------ A-row gather (gate/up, warps 6..9, both CTAs)
+    // Eight consecutive threads cover one 128-byte row segment, 16 rows per pass, 8 passes; 16-byte
+    // chunk c of row r goes to the swizzled chunk c ^ (r & 7).  Each thread's arrival on the CTA's
+    // local barrier is tied to the completion of its copies (cp.async.mbarrier.arrive.noinc).
+    const int gt = threadIdx.x - kUmmaThreads;
+    const int ch = gt & 7, r_sub = gt >> 3;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = pair_id; t < total_tiles && ok; t += n_pairs) {
+      const Pair2Coord c = umma2_decode(p, tile_start, t);
+      const GroupStatic g = p.gs[c.g];
+      const bool mine = !g.is_shared && p.use_gather == 2;
+      const bf16* src_row[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        src_row[i] = nullptr;
+        if (mine) {                                   // rows past the group repeat its last row
+          const int r = c.row0 + min((2 * c.mp + (int)rank) * kUmmaBM + i * 16 + r_sub, c.count - 1);
+          src_row[i] = p.x_rows_ptr + (size_t)__ldg(p.row_token + r) * p.d;
+        }
+      }
+      for (int kb = 0; kb < k_blocks_fixed; ++kb, ++it) {
+        const uint32_t s = it % kU2Stages, n = it / kU2Stages;
+        if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
+        const uint32_t ab = afull0 + 8 * s;
+        if (mine) {
+          const int k = kb * kUmmaBK + ch * 8;
+          const uint32_t bytes = k < p.d ? 16u : 0u;                        // zero-fill past the end of the row
+          const int k_src = k < p.d ? k : 0;
+          const uint32_t sa = base + s * kU2StageBytes;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int r = i * 16 + r_sub;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                         ::"r"(sa + r * 128 + ((ch ^ (r & 7)) << 4)), "l"(src_row[i] + k_src), "r"(bytes)
+                         : "memory");
+          }
+          asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(ab) : "memory");
+        } else {
+          mbar_arrive(ab);
+        }
+      }
+    }
+    if (!ok) asm volatile("cp.async.wait_all;" ::: "memory");
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
     const int quad = warp & 3;
@@ -347,7 +431,7 @@ inline bool umma2_plan_create(UmmaPlan* P, Umma2Plan* Q) {
   // persistent grid: as many pairs as the device can hold at once (GPCs with an odd SM count leave one SM out)
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(P->n_sms & ~1, 1, 1);
-  cfg.blockDim = dim3(kUmmaThreads, 1, 1);
+  cfg.blockDim = dim3(kU2Threads1, 1, 1);
   cfg.dynamicSmemBytes = kU2SmemBytes;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -364,26 +448,33 @@ inline bool umma2_plan_create(UmmaPlan* P, Umma2Plan* Q) {
   return true;
 }
 
-// Gate/up and down GEMM on CTA pairs; routed rows come from the permuted copy of x.
+// Gate/up and down GEMM on CTA pairs.  gather_mode 2: routed rows are gathered from x_rows inside
+// the gate/up kernel; 0: they come from the permuted copy of x by TMA.
 // `D` supplies the 128-channel W_down maps (shared with the decode path).  Requires
-// umma_bind_x for this forward.  Returns launches or -1.
-inline int umma2_forward(UmmaPlan* P, Umma2Plan* Q, DecodePlan* D, const GroupRows* gr, int32_t* err_word,
-                         cudaStream_t st, cudaEvent_t mid) {
+// umma_bind_x for this forward.  which: bit 0 the gate/up GEMM, bit 1 the down GEMM.  Returns launches or -1.
+inline int umma2_forward(UmmaPlan* P, Umma2Plan* Q, DecodePlan* D, const GroupRows* gr, int gather_mode,
+                         const void* x_rows, int32_t* err_word, cudaStream_t st, cudaEvent_t mid, bool dep = false,
+                         int which = 3) {
   const UmmaShape& s = P->shape;
   UmmaArgs a = umma_base_args(P, gr, err_word);
   const int grid = Q->grid;
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
-  umma2_grouped_kernel<1><<<grid, kUmmaThreads, kU2SmemBytes, st>>>(
-      P->x_rows, P->has_r ? P->x_perm : P->x_rows, Q->b1_s, Q->b1_r, a);
-  if (mid) cudaEventRecord(mid, st);
+  a.use_gather = gather_mode;
+  a.x_rows_ptr = (const bf16*)x_rows;
+  if (which & 1)
+    launch_kernel(dep, umma2_grouped_kernel<1>, dim3(grid), dim3(kU2Threads1), kU2SmemBytes, st,
+                  P->x_rows, P->has_r ? P->x_perm : P->x_rows, Q->b1_s, Q->b1_r, a);
+  if (mid && (which & 1)) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
-  umma2_grouped_kernel<2><<<grid, kUmmaThreads, kU2SmemBytes, st>>>(P->a2_s, P->a2_r, D->wd_s, D->wd_r, a);
+  if (which & 2)
+    launch_kernel(dep, umma2_grouped_kernel<2>, dim3(grid), dim3(kUmmaThreads), kU2SmemBytes, st, P->a2_s, P->a2_r,
+                  D->wd_s, D->wd_r, a);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
     snprintf(P->error, sizeof(P->error), "CTA-pair GEMM launch: %s", cudaGetErrorString(e));
     return -1;
   }
-  return 2;
+  return (which & 1) + ((which >> 1) & 1);
 }
 
 }  // namespace cmoe

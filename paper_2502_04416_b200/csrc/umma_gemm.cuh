@@ -852,19 +852,21 @@ inline int umma_router_forward(UmmaPlan* P, int n_rows, const int32_t* outer_off
 
 // Enqueues the gate/up and the down GEMM over all groups.  gather_mode: how routed groups get
 // their rows of x (0 permuted copy, 1 TMA gather4, 2 cp.async gather).  Requires umma_bind_x for this
-// forward.  Returns the number of kernels launched, or -1 (P->error).
+// forward.  which: bit 0 the gate/up GEMM, bit 1 the down GEMM.  Returns the number of kernels
+// launched, or -1 (P->error).
 inline int umma_forward(UmmaPlan* P, const GroupRows* gr, int gather_mode, const void* x_rows, int32_t* err_word,
-                        cudaStream_t st, cudaEvent_t mid, bool dep = false, bool gate_up_only = false) {
+                        cudaStream_t st, cudaEvent_t mid, bool dep = false, int which = 3) {
   const UmmaShape& s = P->shape;
   UmmaArgs a = umma_base_args(P, gr, err_word);
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
   a.use_gather = gather_mode;
   a.x_rows_ptr = (const bf16*)x_rows;
-  launch_kernel(dep, umma_grouped_kernel<1>, dim3(P->n_sms), dim3(kUmmaThreads + kUmmaGatherThreads), kUmmaSmemBytes,
-                st, P->x_rows, (gather_mode != 0 || !P->has_r) ? P->x_gather : P->x_perm, P->b1_s, P->b1_r, a);
-  if (mid) cudaEventRecord(mid, st);
+  if (which & 1)
+    launch_kernel(dep, umma_grouped_kernel<1>, dim3(P->n_sms), dim3(kUmmaThreads + kUmmaGatherThreads), kUmmaSmemBytes,
+                  st, P->x_rows, (gather_mode != 0 || !P->has_r) ? P->x_gather : P->x_perm, P->b1_s, P->b1_r, a);
+  if (mid && (which & 1)) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
-  if (!gate_up_only)
+  if (which & 2)
     launch_kernel(dep, umma_grouped_kernel<2>, dim3(P->n_sms), dim3(kUmmaThreads), kUmmaSmemBytes, st, P->a2_s,
                   P->a2_r, P->b2_s, P->b2_r, a);
   const cudaError_t e = cudaGetLastError();
@@ -872,7 +874,7 @@ inline int umma_forward(UmmaPlan* P, const GroupRows* gr, int gather_mode, const
     snprintf(P->error, sizeof(P->error), "tensor-core GEMM launch: %s", cudaGetErrorString(e));
     return -1;
   }
-  return gate_up_only ? 1 : 2;
+  return (which & 1) + ((which >> 1) & 1);
 }
 
 }  // namespace cmoe
