@@ -22,12 +22,17 @@ all-on = the original MoE layer (Section 4.4); for the activation profiling
 stage (Appendix "Complete Activation Analysis Pipeline"): scalar brute force,
 row/column invariants, sign and scale invariance of ATopK, a hand-worked case; for the
 clustering pieces (Appendix "Balanced Clustering Algorithm"): squared L2 = Hamming distance
-on binary vectors, a hand-worked mean, brute-force argmin, an exhaustive balanced assignment.
+on binary vectors, a hand-worked mean, brute-force argmin, an exhaustive balanced assignment;
+for the FP8 weight quantisation (Section 6): the E4M3 format's defining values, exhaustive
+round trip, hand-worked ties, brute-force nearest-value search, scale-1 and power-of-two
+scale cases, the rounding error bound, all-experts-on = dense FFN of the dequantised weights.
 Parity unpinned (conventions the paper does not fix): the outer router's
 weights for an existing MoE layer (softmax over the selected logits), the
 tie-break between equal keys (lower index wins) and the NaN policy; likewise the
 tie-breaks of equal magnitudes in ATopK, of equal activation counts and of equal
-centroid distances (lower index or position wins).
+centroid distances (lower index or position wins); the quantisation format itself (E4M3 codes,
+one power-of-two scale per output channel, router left unquantised) is a reading, the paper
+names none.
 """
 from __future__ import annotations
 
@@ -410,3 +415,122 @@ def balanced_assignment(d, m: int) -> np.ndarray:
     assign = np.empty(n, dtype=np.int64)
     assign[rows] = cols // m
     return assign
+
+
+# ------------------- Section 6 "Compatibility with Other Efficiency Techniques"
+# Post-training weight quantisation of the restructured experts.  The paper only states that
+# the restructured FFN composes with post-training quantisation and fixes no format; the
+# reading taken here: weight-only FP8 in the OCP E4M3 encoding (1 sign, 4 exponent bits with
+# bias 7, 3 mantissa bits, subnormals, largest finite value 448, no infinities; S.1111.111 is
+# NaN) with ONE POWER-OF-TWO scale per output channel, as in the OCP microscaling formats'
+# E8M0 scales.  Output channel = a neuron's row of W_gate / W_up, and a row of an expert's
+# block of W_down^T (one scale per (expert, model dimension); the N_s shared experts form one
+# block).  Activations, the router's representative rows and all arithmetic stay as they are.
+# Because the scale is a power of two, w / scale is exact in any binary format, so the code
+# chosen by round-to-nearest-even does not depend on the precision it is computed in, and the
+# dequantised weight code * scale is again exact (also in bf16).
+
+E4M3_MAX = 448.0
+
+
+def fp8_e4m3_decode(codes) -> np.ndarray:
+    """Value of each E4M3 code byte: (-1)^s * 2^(E-7) * (1 + M/8) for E > 0,
+    (-1)^s * 2^-6 * (M/8) for E = 0; codes 0x7F / 0xFF are NaN."""
+    c = np.asarray(codes, dtype=np.uint8).astype(np.int64)
+    s, e, m = c >> 7, (c >> 3) & 0xF, c & 0x7
+    mag = np.where(e > 0, np.ldexp(1.0 + m / 8.0, e - 7), np.ldexp(m / 8.0, -6))
+    mag = np.where((e == 15) & (m == 7), np.nan, mag)
+    return np.where(s == 1, -mag, mag)
+
+
+def fp8_e4m3_encode(v) -> np.ndarray:
+    """Nearest E4M3 code of each value, ties to the even mantissa, magnitudes beyond 448
+    saturate to +-448 (no infinities in this format); NaN -> 0x7F."""
+    v = _f64(v)
+    a = np.abs(v)
+    out = np.zeros(v.shape, dtype=np.uint8)
+    fin = ~np.isnan(v)
+    a_f = np.where(fin, np.minimum(a, E4M3_MAX), 0.0)
+    # spacing of representable values around a: 2^(e-3) in the binade 2^e, 2^-9 below 2^-6
+    _, p = np.frexp(a_f)                       # a = f * 2^p, f in [0.5, 1)  =>  binade exponent p - 1
+    e = np.maximum(p - 1, -6)
+    q = np.rint(np.ldexp(a_f, 3 - e))          # a / 2^(e-3), rounded half to even; in [0, 16]
+    # q = 16 means the value rounded up into the next binade
+    bump = q >= 16
+    e = np.where(bump, e + 1, e)
+    q = np.where(bump, 8.0, q)
+    normal = q >= 8                            # q in [8, 15]: 1.M with M = q - 8; below: subnormal, M = q
+    field_e = np.where(normal, e + 7, 0).astype(np.int64)
+    field_m = np.where(normal, q - 8, q).astype(np.int64)
+    code = (field_e << 3) | field_m
+    code = np.where(code > 0x7E, 0x7E, code)   # cannot exceed 448 after the clamp; kept as a guard
+    sign = (np.signbit(v) & fin).astype(np.int64) << 7
+    out = np.where(fin, code | sign, 0x7F).astype(np.uint8)
+    return out
+
+
+def pow2_scale_exponent(amax) -> np.ndarray:
+    """Smallest integer e with amax * 2^-e <= 448 (so that the channel's largest weight uses the
+    top of the E4M3 range); 0 for an all-zero channel."""
+    amax = _f64(amax)
+    f, p = np.frexp(amax)                      # amax = f * 2^p, f in [0.5, 1);  448 = 0.875 * 2^9
+    e = np.where(f <= 0.875, p - 9, p - 8)
+    return np.where(amax > 0, e, 0).astype(np.int64)
+
+
+def quantise_rows_fp8(w):
+    """Per-row (output-channel) power-of-two scale and E4M3 codes of a weight matrix [rows, k].
+    Returns (codes uint8 [rows, k], scale_exponent int64 [rows]); weight ~ decode(code) * 2^e."""
+    w = _f64(w)
+    e = pow2_scale_exponent(np.abs(w).max(axis=1)) if w.shape[1] else np.zeros(w.shape[0], np.int64)
+    codes = fp8_e4m3_encode(np.ldexp(w, -e[:, None]))
+    return codes, e
+
+
+def dequantise_rows_fp8(codes, scale_exponent) -> np.ndarray:
+    return np.ldexp(fp8_e4m3_decode(codes), np.asarray(scale_exponent, dtype=np.int64)[:, None])
+
+
+def quantise_expert_weights(w_gate, w_up, w_down, neuron_perm, n_experts: int, n_shared: int):
+    """FP8 weight-only quantisation of a restructured layer.  W_gate and W_up: one scale per
+    neuron (row).  W_down: one scale per (expert block, model dimension), the block being the
+    expert's slice of neurons (all shared experts together form block 0).  Returns a dict with
+    the dequantised matrices in the original layout (``w_gate``, ``w_up``, ``w_down``: what a
+    forward pass of the quantised layer multiplies by) and the codes / scale exponents:
+    ``gate_codes, gate_exp, up_codes, up_exp`` by original neuron, ``down_codes`` [d, d_ff] by
+    original neuron column, ``down_exp`` [1 + N_r, d] by block."""
+    w_down = _f64(w_down)
+    d_ff = len(neuron_perm)
+    m = d_ff // n_experts
+    n_r = n_experts - n_shared
+    g_codes, g_exp = quantise_rows_fp8(w_gate)
+    u_codes, u_exp = quantise_rows_fp8(w_up)
+    blocks = []
+    if n_shared > 0:
+        blocks.append(np.asarray(neuron_perm[:n_shared * m], dtype=np.int64))
+    for j in range(n_r):
+        blocks.append(expert_neurons(neuron_perm, n_experts, n_shared + j))
+    d_codes = np.zeros(w_down.shape, dtype=np.uint8)
+    d_exp = np.zeros((len(blocks), w_down.shape[0]), dtype=np.int64)
+    w_down_q = np.zeros_like(w_down)
+    for b, neurons in enumerate(blocks):
+        codes, e = quantise_rows_fp8(w_down[:, neurons])
+        d_codes[:, neurons] = codes
+        d_exp[b] = e
+        w_down_q[:, neurons] = dequantise_rows_fp8(codes, e)
+    return dict(w_gate=dequantise_rows_fp8(g_codes, g_exp), w_up=dequantise_rows_fp8(u_codes, u_exp),
+                w_down=w_down_q, gate_codes=g_codes, gate_exp=g_exp, up_codes=u_codes, up_exp=u_exp,
+                down_codes=d_codes, down_exp=d_exp, has_shared_block=n_shared > 0)
+
+
+def cmoe_layer_forward_fp8(x, w_gate, w_up, w_down, neuron_perm, rep_idx, n_experts: int,
+                           n_shared: int, top_k: int, gate_scale_u=None, select_bias_b=None):
+    """Forward of the layer with FP8-quantised expert weights: the router (Eq. router) reads the
+    ORIGINAL representative rows, so the routing is that of the unquantised layer; the experts
+    (Eq. moe_output) multiply by the dequantised weights.  Returns what cmoe_layer_forward does."""
+    q = quantise_expert_weights(w_gate, w_up, w_down, neuron_perm, n_experts, n_shared)
+    s = router_scores(x, w_gate, w_up, rep_idx)
+    sel_idx, gates, s_prime, keys = gate_logic(s, top_k, gate_scale_u, select_bias_b)
+    out = moe_forward(x, q["w_gate"], q["w_up"], q["w_down"], neuron_perm, n_experts, n_shared,
+                      sel_idx, gates)
+    return out, sel_idx, gates, s, s_prime, keys

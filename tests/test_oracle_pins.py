@@ -495,6 +495,98 @@ def pin_initial_centroids_and_assignment(o):
     assert abs(sum(d[i, got[i]] for i in range(6)) - best) < 1e-12
 
 
+# ------------------------------------------------------- FP8 weight quantisation
+def pin_fp8_format(o):
+    """OCP E4M3 as its definition gives it: bias 7, 3 mantissa bits, subnormals below 2^-6,
+    largest finite value 448, S.1111.111 = NaN; round to nearest, ties to even, saturating."""
+    dec = o.fp8_e4m3_decode
+    np.testing.assert_array_equal(dec([0x00, 0x01, 0x07, 0x08, 0x38, 0x3C, 0x40, 0x77, 0x7E]),
+                                  [0.0, 2.0 ** -9, 7 * 2.0 ** -9, 2.0 ** -6, 1.0, 1.5, 2.0, 240.0, 448.0])
+    assert dec([0xB8])[0] == -1.0 and np.isnan(dec([0x7F, 0xFF])).all()
+    codes = np.array([c for c in range(256) if c & 0x7F != 0x7F], dtype=np.uint8)
+    vals = dec(codes)
+    np.testing.assert_array_equal(o.fp8_e4m3_encode(vals), codes)            # every value is its own code
+    # hand-worked roundings: 1.0625 and 1.1875 are ties in the binade of 1 (spacing 1/8)
+    enc = o.fp8_e4m3_encode([1.0625, 1.1875, 1.07, 2.0 ** -10, 1.5 * 2.0 ** -9, 2.0 ** -6 - 2.0 ** -11, 460.0, 1e6, -1e6])
+    np.testing.assert_array_equal(enc, [0x38, 0x3A, 0x39, 0x00, 0x02, 0x08, 0x7E, 0x7E, 0xFE])
+    # brute force: nearest representable value by exhaustive search over the 253 finite magnitudes
+    rng = np.random.default_rng(21)
+    x = np.concatenate([rng.normal(scale=s, size=400) for s in (300.0, 3.0, 0.02, 0.004)])
+    pos = np.array(sorted(set(np.abs(vals))))
+    pos_code = {v: c for c, v in zip(codes, vals) if c < 0x80}
+    for xi, ci in zip(x, o.fp8_e4m3_encode(x)):
+        a = min(abs(xi), 448.0)
+        dist = np.abs(pos - a)
+        best = np.nonzero(dist == dist.min())[0]
+        cand = [pos_code[pos[i]] for i in best]
+        want = cand[0] if len(cand) == 1 else [c for c in cand if c % 2 == 0][0]
+        assert ci == (want | (0x80 if xi < 0 else 0)), (xi, hex(ci), hex(want))
+
+
+def pin_fp8_row_scales(o):
+    """One power-of-two scale per output channel, the smallest that brings the channel's largest
+    weight to at most 448."""
+    rng = np.random.default_rng(22)
+    w = rng.normal(scale=0.02, size=(9, 40))
+    w[3] = 0.0
+    w[4, 7] = 448.0                      # scale 1: the codes are the plain encoding
+    w[4, :7] = [1.0, 1.5, -2.0, 0.25, 1.0625, 240.0, -448.0]
+    codes, e = o.quantise_rows_fp8(w)
+    assert e[4] == 0 and e[3] == 0 and not codes[3].any()
+    np.testing.assert_array_equal(codes[4, :8], [0x38, 0x3C, 0xC0, 0x28, 0x38, 0x77, 0xFE, 0x7E])
+    amax = np.abs(w).max(axis=1)
+    scaled = amax * 2.0 ** (-e.astype(np.float64))
+    live = amax > 0
+    assert np.all(scaled[live] <= 448.0) and np.all(scaled[live] > 224.0)
+    # a power-of-two multiple of a row has the same codes and a shifted exponent
+    codes2, e2 = o.quantise_rows_fp8(w * np.array([2.0 ** k for k in (-3, 0, 5, 1, -7, 2, 9, -1, 4)])[:, None])
+    np.testing.assert_array_equal(codes2, codes)
+    np.testing.assert_array_equal((e2 - e)[live], np.array([-3, 0, 5, 1, -7, 2, 9, -1, 4])[live])
+    # error bound of round-to-nearest with 3 mantissa bits: half a unit in the last place
+    wq = o.dequantise_rows_fp8(codes, e)
+    normal = np.abs(w) >= np.ldexp(1.0, -6 + e)[:, None]
+    assert np.all(np.abs(wq - w)[normal] <= np.abs(w)[normal] * 2.0 ** -4)
+    assert np.all(np.abs(wq - w) <= np.ldexp(1.0, -10 + e)[:, None] + np.abs(w) * 2.0 ** -4)
+    # dequantised values are exactly representable in bf16 (8 significant bits suffice)
+    np.testing.assert_array_equal(wl.round_to_storage(wq.astype(np.float32), "bf16"), wq.astype(np.float32))
+
+
+def pin_fp8_layer(o):
+    """Quantised layer: W_gate / W_up scaled per neuron, W_down per (expert block, model dimension);
+    the router reads the original weights; all experts on with unit gates = the dense FFN of the
+    dequantised weights."""
+    shape, x, lay = small_layer(seed=23, d=24, m=6, n_tok=29)
+    kw = layer_kwargs(shape, lay)
+    q = o.quantise_expert_weights(lay.w_gate, lay.w_up, lay.w_down, lay.neuron_perm, shape.n_experts, shape.n_shared)
+    m, n_s = shape.m, shape.n_shared
+    # per-neuron scales of W_gate: row n's largest code sits in the top binade (scaled amax in (224, 448])
+    top = np.abs(o.fp8_e4m3_decode(q["gate_codes"])).max(axis=1)
+    assert np.all((top >= 224) & (top <= 448))       # the scaled maximum lies in (224, 448] before rounding
+    # W_down: one scale per (block, c); block 0 = all shared neurons together
+    blocks = [lay.neuron_perm[:n_s * m]] + [lay.neuron_perm[(n_s + j) * m:(n_s + j + 1) * m] for j in range(shape.n_routed)]
+    assert q["down_exp"].shape == (len(blocks), shape.d_model)
+    for b, neurons in enumerate(blocks):
+        sub = np.abs(lay.w_down[:, neurons]).max(axis=1)
+        np.testing.assert_array_equal(q["down_exp"][b], o.pow2_scale_exponent(sub))
+        top = np.abs(o.fp8_e4m3_decode(q["down_codes"][:, neurons])).max(axis=1)
+        assert np.all((top >= 224) & (top <= 448))       # the scaled maximum lies in (224, 448] before rounding
+        np.testing.assert_array_equal(q["w_down"][:, neurons],
+                                      o.fp8_e4m3_decode(q["down_codes"][:, neurons]) * 2.0 ** q["down_exp"][b][:, None])
+    assert len({tuple(e) for e in q["down_exp"]}) > 1                       # the blocks really have their own scales
+    # forward: routing of the unquantised layer, experts on the dequantised weights
+    out, sel, gates, s, _, _ = o.cmoe_layer_forward_fp8(x, **kw)
+    ref_out, ref_sel, ref_gates, ref_s, _, _ = o.cmoe_layer_forward(x, **kw)
+    np.testing.assert_array_equal(sel, ref_sel)
+    np.testing.assert_array_equal(s, ref_s)
+    kq = dict(kw, w_gate=q["w_gate"], w_up=q["w_up"], w_down=q["w_down"])
+    want = o.moe_forward(x, q["w_gate"], q["w_up"], q["w_down"], lay.neuron_perm, shape.n_experts, shape.n_shared, ref_sel, ref_gates)
+    np.testing.assert_allclose(out, want, rtol=1e-13, atol=1e-15)
+    rel = np.abs(out - ref_out).sum() / np.abs(ref_out).sum()
+    assert 1e-3 < rel < 0.1                                                  # quantisation changes the output, a little
+    all_on, *_ = o.cmoe_layer_forward_fp8(x, **dict(kw, top_k=shape.n_routed))
+    np.testing.assert_allclose(all_on, o.dense_ffn(x, q["w_gate"], q["w_up"], q["w_down"]), rtol=1e-10, atol=1e-13)
+
+
 PINS = [pin_dense_closed_form, pin_dense_library, pin_dense_per_neuron_brute_force,
         pin_all_experts_on_is_dense, pin_reconstruction_error_identity, pin_shared_always_on,
         pin_router_is_representative_activation, pin_gate_closed_forms, pin_topk_brute_force,
@@ -502,7 +594,7 @@ PINS = [pin_dense_closed_form, pin_dense_library, pin_dense_per_neuron_brute_for
         pin_hierarchical_all_on_is_original_moe, pin_hierarchical_is_weighted_sum_of_layers,
         pin_atopk_brute_force, pin_atopk_invariants, pin_activation_rates_and_shared, pin_profile_pipeline,
         pin_distance_is_hamming_on_binary, pin_cluster_update_and_representatives,
-        pin_initial_centroids_and_assignment]
+        pin_initial_centroids_and_assignment, pin_fp8_format, pin_fp8_row_scales, pin_fp8_layer]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda p: p.__name__)
@@ -563,6 +655,17 @@ MUTATIONS = {
     "centroids_include_shared": ("if int(i) not in shared]", "]"),
     "assignment_unbalanced": ("rows, cols = linear_sum_assignment(np.repeat(d, m, axis=1))",
                               "rows, cols = np.arange(n), np.argmin(d, axis=1) * m"),
+    "fp8_truncates": ("q = np.rint(np.ldexp(a_f, 3 - e))", "q = np.floor(np.ldexp(a_f, 3 - e))"),
+    "fp8_ties_away": ("q = np.rint(np.ldexp(a_f, 3 - e))", "q = np.floor(np.ldexp(a_f, 3 - e) + 0.5)"),
+    "fp8_bias_8": ("mag = np.where(e > 0, np.ldexp(1.0 + m / 8.0, e - 7), np.ldexp(m / 8.0, -6))",
+                   "mag = np.where(e > 0, np.ldexp(1.0 + m / 8.0, e - 8), np.ldexp(m / 8.0, -7))"),
+    "fp8_no_subnormals": ("e = np.maximum(p - 1, -6)", "e = np.maximum(p - 1, -9)"),
+    "fp8_scale_one_binade_high": ("e = np.where(f <= 0.875, p - 9, p - 8)", "e = np.where(f <= 0.875, p - 8, p - 7)"),
+    "fp8_scale_ignores_mantissa": ("e = np.where(f <= 0.875, p - 9, p - 8)", "e = p - 9"),
+    "fp8_down_one_scale_per_row": ("codes, e = quantise_rows_fp8(w_down[:, neurons])",
+                                   "codes, e = quantise_rows_fp8(w_down); codes = codes[:, neurons]"),
+    "fp8_router_on_quantised": ("    s = router_scores(x, w_gate, w_up, rep_idx)\n    sel_idx, gates, s_prime, keys = gate_logic(s, top_k, gate_scale_u, select_bias_b)\n    out = moe_forward(x, q[",
+                                "    s = router_scores(x, q[\"w_gate\"], q[\"w_up\"], rep_idx)\n    sel_idx, gates, s_prime, keys = gate_logic(s, top_k, gate_scale_u, select_bias_b)\n    out = moe_forward(x, q["),
     "pack_bit_order": ("np.uint64(1) << np.arange(32, dtype=np.uint64)", "np.uint64(1) << np.arange(31, -1, -1, dtype=np.uint64)"),
 }
 
