@@ -123,6 +123,34 @@ int cmoe_ffn_forward(cmoe_layer* layer, const void* x, int32_t T, void* out, voi
 int cmoe_ffn_forward_host(cmoe_layer* layer, const void* x_host, int32_t T, void* out_host,
                           int32_t chunk_tokens, void* stream);
 
+/* FP8 weight-only quantisation of the expert weights (the paper's Section 6, "Compatibility with
+ * Other Efficiency Techniques", states that the restructured FFN composes with post-training
+ * quantisation and names no format; this library's format is: OCP E4M3 codes — 1 sign, 4 exponent
+ * bits with bias 7, 3 mantissa bits, subnormals, largest value 448 — with one power-of-two scale
+ * per output channel, code = round-to-nearest-even(w / scale), scale = the smallest power of two
+ * with max|w| / scale <= 448, 1 for an all-zero channel).
+ *
+ * cmoe_quantise_rows_fp8: the stand-alone operation on a matrix.
+ *   w           : device, bf16 [rows, cols] row-major; a row is an output channel.
+ *   codes       : device, uint8 [rows, cols], receives the E4M3 codes.
+ *   scale       : device, float [rows], receives the power-of-two scales.
+ *   dequantised : device, bf16 [rows, cols] or NULL; receives code * scale (exact in bf16); may be w itself.
+ * Asynchronous on `stream`, allocates nothing.  Errors: INVALID_ARG, CUDA. */
+int cmoe_quantise_rows_fp8(const void* w, int32_t rows, int32_t cols, uint8_t* codes, float* scale,
+                           void* dequantised, void* stream);
+
+/* cmoe_layer_quantise_fp8: quantise a bf16 layer's expert weights in that format.  Output channels:
+ * a neuron's row of W_gate and of W_up; a model dimension's row of each expert's block of W_down
+ * (the N_s shared experts form one block), so W_down has one scale per (expert, model dimension).
+ * The router's representative rows keep their original values, so the routing does not change.
+ * Afterwards every forward of the layer computes with the dequantised weights code * scale:
+ * batches of at most 64 rows stream the FP8 codes (half the weight bytes of bf16) and expand
+ * them to bf16 on the fly, larger batches read bf16 copies holding exactly the same values.
+ * The layer then owns 1.5x the weight memory.  Plain and hierarchical layers; needs d_model, the
+ * expert width and the shared width to be multiples of 16.  Allocates (a set-up call, like create)
+ * and synchronises `stream`.  Idempotent.  Errors: INVALID_ARG, UNSUPPORTED (fp32 layer, shape), CUDA. */
+int cmoe_layer_quantise_fp8(cmoe_layer* layer, void* stream);
+
 /* Replace the learnable gate scaling u and the selection bias b (Section 4.3).
  * host arrays [n_routed_groups] (N_r, or n_outer*N_r for a hierarchical layer,
  * outer-major) or NULL for zeros.  Synchronises `stream`. */

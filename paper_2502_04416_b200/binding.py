@@ -19,6 +19,7 @@ STAGE_NAMES = ["route", "permute", "gemm1_swiglu", "gemm2_down", "combine"]
 
 EXPORTS = [
     "cmoe_layer_create", "cmoe_hier_create", "cmoe_ffn_forward", "cmoe_ffn_forward_host", "cmoe_layer_set_gate_params",
+    "cmoe_quantise_rows_fp8", "cmoe_layer_quantise_fp8",
     "cmoe_layer_get_gate_params", "cmoe_layer_update_bias", "cmoe_profile_activations", "cmoe_select_shared",
     "cmoe_cluster_update", "cmoe_cluster_distances", "cmoe_cluster_representatives", "cmoe_layer_set_gemm_path", "cmoe_layer_set_launch_chaining",
     "cmoe_layer_dims", "cmoe_get_routing", "cmoe_layer_status", "cmoe_layer_selftest_wait_timeout",
@@ -58,6 +59,8 @@ def load() -> C.CDLL:
     lib.cmoe_hier_create.argtypes = [i32, i32, vp, C.POINTER(vp), i32, vp, C.POINTER(vp)]
     lib.cmoe_ffn_forward.argtypes = [vp, vp, i32, vp, vp]
     lib.cmoe_ffn_forward_host.argtypes = [vp, vp, i32, vp, i32, vp]
+    lib.cmoe_quantise_rows_fp8.argtypes = [vp, i32, i32, vp, vp, vp, vp]
+    lib.cmoe_layer_quantise_fp8.argtypes = [vp, vp]
     lib.cmoe_layer_set_gate_params.argtypes = [vp, vp, vp, vp]
     lib.cmoe_layer_set_gemm_path.argtypes = [vp, i32]
     lib.cmoe_layer_set_launch_chaining.argtypes = [vp, i32]
@@ -185,6 +188,10 @@ class Layer:
         _check(st, "cmoe_ffn_forward_host")
         return out_host
 
+    def quantise_fp8(self, stream=None) -> None:
+        """cmoe_layer_quantise_fp8: FP8 (E4M3, power-of-two scale per output channel) expert weights."""
+        _check(load().cmoe_layer_quantise_fp8(self._h, _stream_ptr(stream)), "cmoe_layer_quantise_fp8")
+
     def set_gate_params(self, gate_scale_u=None, select_bias_b=None, stream=None) -> None:
         u = None if gate_scale_u is None else np.ascontiguousarray(gate_scale_u, dtype=np.float32)
         b = None if select_bias_b is None else np.ascontiguousarray(select_bias_b, dtype=np.float32)
@@ -288,6 +295,19 @@ class Layer:
             self.destroy()
         except Exception:
             pass
+
+
+def quantise_rows_fp8(w, want_dequantised: bool = False, stream=None):
+    """cmoe_quantise_rows_fp8 on a CUDA bf16 tensor [rows, cols]: (codes uint8, scale float32[, dequantised bf16])."""
+    import torch
+    rows, cols = w.shape
+    codes = torch.empty((rows, cols), dtype=torch.uint8, device=w.device)
+    scale = torch.empty(rows, dtype=torch.float32, device=w.device)
+    deq = torch.empty_like(w) if want_dequantised else None
+    _check(load().cmoe_quantise_rows_fp8(w.data_ptr(), rows, cols, codes.data_ptr(), scale.data_ptr(),
+                                         deq.data_ptr() if deq is not None else None, _stream_ptr(stream)),
+           "cmoe_quantise_rows_fp8")
+    return (codes, scale, deq) if want_dequantised else (codes, scale)
 
 
 def token_permute_scratch_bytes(n_rows: int, n_groups: int) -> int:

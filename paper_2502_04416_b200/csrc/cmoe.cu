@@ -16,6 +16,7 @@
 #include "balance.cuh"
 #include "cluster.cuh"
 #include "combine.cuh"
+#include "fp8.cuh"
 #include "common.cuh"
 #include "permute.cuh"
 #include "profile.cuh"
@@ -85,6 +86,10 @@ struct cmoe_layer {
   void* w_router = nullptr; // [n_outer, d] (hierarchical)
   float* u = nullptr;       // [n_outer*N_r]
   float* b = nullptr;
+  // FP8 copy of the expert weights (cmoe_layer_quantise_fp8): codes in the packed layouts, scales
+  uint8_t *w_gu8 = nullptr, *wd8 = nullptr;
+  float *scale_gu = nullptr, *scale_d = nullptr;
+  bool fp8 = false;
   GroupStatic* gs = nullptr;
   std::vector<GroupStatic> gs_host;
 
@@ -152,6 +157,7 @@ void free_layer(cmoe_layer* L) {
   if (L->hio.s_in) cudaStreamDestroy(L->hio.s_in);
   if (L->hio.s_out) cudaStreamDestroy(L->hio.s_out);
   umma_plan_destroy(&L->umma);
+  cudaFree(L->w_gu8); cudaFree(L->wd8); cudaFree(L->scale_gu); cudaFree(L->scale_d);
   cudaFree(L->w_gu); cudaFree(L->wd_p); cudaFree(L->w_rep);
   cudaFree(L->w_router); cudaFree(L->u); cudaFree(L->b); cudaFree(L->gs); cudaFree(L->ws);
   delete L;
@@ -744,6 +750,49 @@ int cmoe_ffn_forward_host(cmoe_layer* L, const void* x_host, int32_t T, void* ou
   }
   for (int b = 0; b < 2 && b < n_chunks; ++b) CU_TRY(cudaStreamWaitEvent(st, h.out_done[b], 0));
   L->launches = launches;
+  return CMOE_OK;
+}
+
+int cmoe_quantise_rows_fp8(const void* w, int32_t rows, int32_t cols, uint8_t* codes, float* scale, void* dequantised,
+                           void* stream) {
+  if (rows < 0 || cols < 0) return arg_fail(CMOE_ERR_INVALID_ARG, "negative size");
+  if (rows == 0) return CMOE_OK;
+  if (!w || !scale || (cols > 0 && !codes)) return arg_fail(CMOE_ERR_INVALID_ARG, "null w / codes / scale");
+  quantise_rows_fp8_kernel<<<rows, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      (const bf16*)w, rows, cols, cols, codes, cols, scale, (bf16*)dequantised);
+  CU_TRY(cudaGetLastError());
+  return CMOE_OK;
+}
+
+int cmoe_layer_quantise_fp8(cmoe_layer* L, void* stream) {
+  if (!L) return arg_fail(CMOE_ERR_INVALID_ARG, "null layer");
+  if (L->fp8) return CMOE_OK;
+  if (L->cfg.dtype != CMOE_BF16 || !L->umma_ok)
+    return arg_fail(CMOE_ERR_UNSUPPORTED, "FP8 weights need a bf16 layer on the tensor-core path");
+  if (L->cfg.d_model % 16 || L->m % 16 || L->shared_width() % 16)
+    return arg_fail(CMOE_ERR_UNSUPPORTED, "FP8 weights need d_model, the expert width and the shared width to be multiples of 16");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t d = L->cfg.d_model, rows_w = (size_t)L->n_outer * L->cfg.d_ff;
+  CU_TRY(cudaMalloc(&L->w_gu8, 2 * rows_w * d));
+  CU_TRY(cudaMalloc(&L->wd8, rows_w * d));
+  CU_TRY(cudaMalloc(&L->scale_gu, 2 * rows_w * sizeof(float)));
+  CU_TRY(cudaMalloc(&L->scale_d, (size_t)L->n_groups_total() * d * sizeof(float)));
+  // gate and up planes: one scale per neuron row; the bf16 rows are replaced by the dequantised values
+  quantise_rows_fp8_kernel<<<(unsigned)(2 * rows_w), 256, 0, st>>>((const bf16*)L->w_gu, (int)(2 * rows_w), (int)d, (long long)d,
+                                                                 L->w_gu8, (long long)d, L->scale_gu, (bf16*)L->w_gu);
+  // W_down: every group's block [d, width] has one scale per output channel
+  for (size_t g = 0; g < L->gs_host.size(); ++g) {
+    const GroupStatic& gs = L->gs_host[g];
+    if (gs.width <= 0) continue;
+    bf16* blk = (bf16*)L->wd_p + gs.wd_offset;
+    quantise_rows_fp8_kernel<<<(unsigned)d, 256, 0, st>>>(blk, (int)d, gs.width, (long long)gs.width, L->wd8 + gs.wd_offset,
+                                                         (long long)gs.width, L->scale_d + g * d, blk);
+  }
+  CU_TRY(cudaGetLastError());
+  CU_TRY(cudaStreamSynchronize(st));
+  if (!decode_plan_attach_fp8(&L->umma, &L->decode, L->w_gu8, L->wd8, L->scale_gu, L->scale_d))
+    return arg_fail(CMOE_ERR_CUDA, L->umma.error);
+  L->fp8 = true;
   return CMOE_OK;
 }
 

@@ -23,8 +23,14 @@
 // finishes the tile.  Units are dealt to the persistent CTAs in snake order (left to right,
 // then right to left), which balances long shared-expert units against short routed ones.
 // Same warp roles, bounded waits and teardown as the token-major kernels.
+//
+// W8 = true streams FP8 (E4M3) weights, half the bytes: TMA lands the codes of a k block in a
+// raw ring (unswizzled, 64 bytes per weight row), eight converter warps expand them to bf16 in
+// the 128-byte-swizzled layout of a short second ring (exact, see fp8.cuh), the MMAs read that,
+// and the epilogue multiplies each weight row's sums by its power-of-two scale.
 #pragma once
 
+#include "fp8.cuh"
 #include "umma_gemm.cuh"
 
 namespace cmoe {
@@ -42,13 +48,21 @@ constexpr int kDecSlotFloats = 128 * 2 * kDecMaxRows;      // 128 weight rows x 
 struct DecGroup { int32_t unit0, tile0, slot0; int16_t z, kb; };
 constexpr int kDecInvOff = 256 + ((kUmmaMaxGroups + 1) * (int)sizeof(DecGroup) + 15) / 16 * 16;   // per-warp token tables
 
-template <int MODE> struct DecodeCfg;
-template <> struct DecodeCfg<4> { static constexpr int kWBytes = 2 * 128 * kUmmaBK * 2, kStages = 5; };
-template <> struct DecodeCfg<5> { static constexpr int kWBytes = 128 * kUmmaBK * 2, kStages = 8; };
+constexpr int kDecCvtWarps = 8;            // W8: warps that expand FP8 codes to bf16
+constexpr int kDecThreadsW8 = kUmmaThreads + 32 * kDecCvtWarps;
 
-template <int MODE>
+// kWBytes: bf16 weight tile(s) of one k block (what the MMAs read); kRawBytes: what TMA lands per
+// stage (the same tile for bf16 weights, the FP8 codes for W8); kConv: bf16 tiles of the W8 ring.
+template <int MODE, bool W8> struct DecodeCfg;
+template <> struct DecodeCfg<4, false> { static constexpr int kWBytes = 2 * 128 * kUmmaBK * 2, kRawBytes = kWBytes, kStages = 5, kConv = 0; };
+template <> struct DecodeCfg<5, false> { static constexpr int kWBytes = 128 * kUmmaBK * 2, kRawBytes = kWBytes, kStages = 8, kConv = 0; };
+template <> struct DecodeCfg<4, true> { static constexpr int kWBytes = 2 * 128 * kUmmaBK * 2, kRawBytes = kWBytes / 2, kStages = 5, kConv = 2; };
+template <> struct DecodeCfg<5, true> { static constexpr int kWBytes = 128 * kUmmaBK * 2, kRawBytes = kWBytes / 2, kStages = 8, kConv = 3; };
+
+template <int MODE, bool W8 = false>
 constexpr int decode_smem_bytes() {
-  return 1024 + DecodeCfg<MODE>::kStages * (DecodeCfg<MODE>::kWBytes + kDecXBytes) + kDecInvOff + 4 * 64 * 4;
+  using C = DecodeCfg<MODE, W8>;
+  return 1024 + C::kStages * (C::kRawBytes + kDecXBytes) + C::kConv * C::kWBytes + kDecInvOff + 4 * 64 * 4;
 }
 
 struct DecodeArgs {
@@ -64,6 +78,10 @@ struct DecodeArgs {
   float* part;           // [kDecMaxSlots][kDecSlotFloats] slice partials
   int32_t* ticket;       // [tiles][4 epilogue warps], zero between launches
   int tok_box_rows;      // rows of the token-tile TMA box (16, 32 or 64): no more than the batch needs
+  // W8: power-of-two scales of the FP8 weight rows
+  const float* scale_gu; // [2][rows_w]: gate plane, then up plane, packed neuron order
+  const float* scale_d;  // [n_groups][d]: per group and output channel
+  long long rows_w;      // n_outer * d_ff
 };
 
 // Tile handled by CTA `cta` in its `round`-th turn: even rounds run left to right, odd
@@ -75,24 +93,29 @@ __device__ __forceinline__ int snake_tile(int round, int cta, int n_ctas, int to
 
 // SPLIT = false is the plain form (one unit per tile, no scratch); the host picks SPLIT = true
 // only when even the largest possible set of active experts leaves tiles to split.
-template <int MODE, bool SPLIT>
-__global__ void __launch_bounds__(kUmmaThreads, 1)
+template <int MODE, bool SPLIT, bool W8 = false>
+__global__ void __launch_bounds__(W8 ? kDecThreadsW8 : kUmmaThreads, 1)
 umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_constant__ CUtensorMap tm_w_r,
                    const __grid_constant__ CUtensorMap tm_x_s, const __grid_constant__ CUtensorMap tm_x_r,
                    const DecodeArgs p) {
   grid_dep_wait();
   grid_dep_trigger();
-  constexpr int kStages = DecodeCfg<MODE>::kStages;
-  constexpr int kWBytes = DecodeCfg<MODE>::kWBytes;
-  constexpr int kStageBytes = kWBytes + kDecXBytes;
+  using Cfg = DecodeCfg<MODE, W8>;
+  constexpr int kStages = Cfg::kStages;
+  constexpr int kWBytes = Cfg::kWBytes;
+  constexpr int kRawBytes = Cfg::kRawBytes;
+  constexpr int kConv = Cfg::kConv;
+  constexpr int kStageBytes = kRawBytes + kDecXBytes;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
-  const uint32_t bars = base + kStages * kStageBytes;
-  uint8_t* bars_gen = gen + kStages * kStageBytes;
-  // barrier block: full[8] empty[8] acc_full[2] acc_empty[2], tmem slot, abort flag
+  const uint32_t conv0 = base + kStages * kStageBytes;           // W8: ring of converted bf16 tiles
+  const uint32_t bars = conv0 + kConv * kWBytes;
+  uint8_t* bars_gen = gen + kStages * kStageBytes + kConv * kWBytes;
+  // barrier block: full[8] empty[8] acc_full[2] acc_empty[2], tmem slot, abort flag, W8: conv_full[4] conv_empty[4]
   const uint32_t full0 = bars, empty0 = bars + 64, accf0 = bars + 128, acce0 = bars + 144;
+  const uint32_t cfull0 = bars + 192, cempty0 = bars + 224;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_gen + 160);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
   DecGroup* grp = reinterpret_cast<DecGroup*>(bars_gen + 256);       // SPLIT: [n_groups + 1]
@@ -104,6 +127,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 4); }
+    for (int c = 0; c < kConv; ++c) { mbar_init(cfull0 + 8 * c, kDecCvtWarps); mbar_init(cempty0 + 8 * c, 1); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -223,9 +247,9 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         const uint32_t s = it % kStages, n = it / kStages;
         if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
         const uint32_t fb = full0 + 8 * s;
-        const uint32_t sw = base + s * kStageBytes, sx = sw + kWBytes;
+        const uint32_t sw = base + s * kStageBytes, sx = sw + kRawBytes;
         if (lane == 0) {
-          mbar_expect_tx(fb, kWBytes + p.tok_box_rows * kUmmaBK * 2);
+          mbar_expect_tx(fb, kRawBytes + p.tok_box_rows * kUmmaBK * 2);
           if (MODE == 4) tma_load_3d(sw, tw, fb, kb * kUmmaBK, g.w_row0 + nt * 128, 0);
           else if (g.is_shared) tma_load_3d(sw, tw, fb, kb * kUmmaBK, nt * 128, g.outer);
           else tma_load_4d(sw, tw, fb, kb * kUmmaBK, nt * 128, j, g.outer);
@@ -255,9 +279,17 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         const int k_end = SPLIT ? un.kb1 : ((MODE == 4 ? p.d : g.width) + kUmmaBK - 1) / kUmmaBK;
         for (int kb = un.kb0; kb < k_end; ++kb, ++it) {
           const uint32_t s = it % kStages, n = it / kStages;
-          if (!mbar_wait(full0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
+          uint32_t sw = base + s * kStageBytes;
+          const uint32_t sx = sw + kRawBytes;
+          if constexpr (W8) {
+            // the converters waited for the stage's bytes (weights and tokens) before converting
+            const uint32_t c = it % kConv, cn = it / kConv;
+            if (!mbar_wait(cfull0 + 8 * c, cn & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
+            sw = conv0 + c * kWBytes;
+          } else {
+            if (!mbar_wait(full0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
+          }
           tc_fence_after();
-          const uint32_t sw = base + s * kStageBytes, sx = sw + kWBytes;
 #pragma unroll
           for (int k = 0; k < kUmmaBK / 16; ++k) {
             const uint32_t acc = (kb != un.kb0 || k != 0) ? 1u : 0u;
@@ -267,8 +299,55 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
                         umma_smem_desc(sx + k * 32), idesc, acc);
           }
           umma_commit(empty0 + 8 * s);
+          if constexpr (W8) umma_commit(cempty0 + 8 * (it % kConv));
         }
         if (ok) umma_commit(accf0 + 8 * buf);
+      }
+    }
+  } else if (W8 && warp >= 6) {
+    // ------------------------------------------------------------ FP8 -> bf16 converters (W8, warps 6..13)
+    // A pass of one warp expands 8 weight rows x 64 codes (512 contiguous raw bytes, 16 per lane)
+    // into 8 rows x 128 bytes of the swizzled bf16 tile: lane l holds codes 16c..16c+15 of row l/4
+    // (c = l % 4) and writes the row's 16-byte chunks 2c and 2c+1 at positions (chunk ^ (row & 7)).
+    constexpr int kRows = kRawBytes / kUmmaBK;                    // weight rows per k block (gate + up planes)
+    constexpr int kPasses = kRows / 8 / kDecCvtWarps;
+    const int cw = warp - 6;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int round = 0; ok; ++round) {
+      const int t = snake_tile(round, cta, n_ctas, total_units);
+      if (t < 0) break;
+      const Unit un = find_unit(t);
+      const GroupStatic g = p.gs[un.gi];
+      const int k_end = SPLIT ? un.kb1 : ((MODE == 4 ? p.d : g.width) + kUmmaBK - 1) / kUmmaBK;
+      for (int kb = un.kb0; kb < k_end; ++kb, ++it) {
+        const uint32_t s = it % kStages, n = it / kStages;
+        const uint32_t c = it % (kConv > 0 ? kConv : 1), cn = it / (kConv > 0 ? kConv : 1);
+        if (!mbar_wait(full0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
+        if (!mbar_wait(cempty0 + 8 * c, (cn & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
+        const uint32_t src = base + s * kStageBytes, dstb = conv0 + c * kWBytes;
+#pragma unroll
+        for (int ps = 0; ps < kPasses; ++ps) {
+          const int row = (cw * kPasses + ps) * 8 + (lane >> 2);          // 0 .. kRows-1 (plane = row / 128)
+          const int ch = lane & 3;
+          uint32_t w0, w1, w2, w3;
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3) : "r"(src + row * kUmmaBK + ch * 16));
+          uint32_t o[8];
+          e4m3x4_to_bf16x4(w0, o[0], o[1]);
+          e4m3x4_to_bf16x4(w1, o[2], o[3]);
+          e4m3x4_to_bf16x4(w2, o[4], o[5]);
+          e4m3x4_to_bf16x4(w3, o[6], o[7]);
+          const uint32_t rb = dstb + row * 128;                           // planes are 128 rows x 128 bytes apart
+          const int sw7 = row & 7;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                       ::"r"(rb + (((2 * ch) ^ sw7) << 4)), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                       ::"r"(rb + (((2 * ch + 1) ^ sw7) << 4)), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> tcgen05.mma reads
+        __syncwarp();
+        if (lane == 0) mbar_arrive(cfull0 + 8 * c);
       }
     }
   } else {
@@ -305,10 +384,22 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         __syncwarp();
       }
       const bool row_live = wr < span;
+      float sc_a = 1.0f, sc_b = 1.0f;                    // W8: power-of-two scales of this thread's weight row(s)
+      if constexpr (W8) {
+        if (row_live) {
+          if (MODE == 4) {
+            sc_a = __ldg(p.scale_gu + g.w_row0 + wr);
+            sc_b = __ldg(p.scale_gu + p.rows_w + g.w_row0 + wr);
+          } else {
+            sc_a = __ldg(p.scale_d + (size_t)gi * p.d + wr);
+          }
+        }
+      }
       auto finish = [&](int c, float a, float b) {       // accumulator column c of this thread's weight row
         if (row_live && c < n_cols) {
           const int pos = lookup ? inv[c] : c;
           if (pos >= 0) {
+            if constexpr (W8) { a *= sc_a; b *= sc_b; }
             const float v = MODE == 4 ? a / (1.0f + __expf(-a)) * b : a;
             dst[(size_t)pos * ld] = __float2bfloat16_rn(v);
           }
@@ -387,6 +478,10 @@ struct DecodePlan {
   // its rows, so that a stage carries as little besides weights as possible
   CUtensorMap x_rows[3];            // x (bound per forward for a plain layer)
   CUtensorMap h_s[3], h_r[3];       // H
+  // FP8 weights (set by decode_plan_attach_fp8): codes in the packed layouts, 64-byte x 128-row boxes
+  bool fp8 = false;
+  CUtensorMap w_gu8, wd8_s, wd8_r;
+  const float *scale_gu = nullptr, *scale_d = nullptr;
 };
 
 inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
@@ -447,6 +542,64 @@ inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
   return true;
 }
 
+// Tensor maps over the FP8 codes of the packed weights (same shapes as the bf16 maps, one byte per
+// element, no swizzle: the converter warps read the raw tile linearly).  Needs d, m and the shared
+// width to be multiples of 16 (TMA strides).
+inline bool decode_plan_attach_fp8(UmmaPlan* P, DecodePlan* D, const void* w_gu8, const void* wd8,
+                                   const float* scale_gu, const float* scale_d) {
+  const UmmaShape& s = P->shape;
+  const size_t d = s.d, rows_w = (size_t)s.n_outer * s.d_ff;
+  auto encode8 = [&](CUtensorMap* tm, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* str,
+                     const cuuint32_t* box, const char* what) {
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    const CUresult r = P->encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), dims, str,
+                                 box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+      snprintf(P->error, sizeof(P->error), "cuTensorMapEncodeTiled(%s) failed with CUresult %d", what, (int)r);
+      return false;
+    }
+    return true;
+  };
+  bool ok = true;
+  {
+    const cuuint64_t dims[3] = {d, rows_w, 2};
+    const cuuint64_t str[2] = {d, rows_w * d};
+    const cuuint32_t box[3] = {kUmmaBK, 128, 2};
+    ok = encode8(&D->w_gu8, w_gu8, 3, dims, str, box, "FP8 gate/up weights");
+  }
+  if (ok && P->has_s) {
+    const cuuint64_t dims[3] = {(cuuint64_t)s.shared_width, d, (cuuint64_t)s.n_outer};
+    const cuuint64_t str[2] = {(cuuint64_t)s.shared_width, d * s.d_ff};
+    const cuuint32_t box[3] = {kUmmaBK, 128, 1};
+    ok = encode8(&D->wd8_s, wd8, 3, dims, str, box, "FP8 shared W_down");
+  }
+  if (ok && P->has_r) {
+    const cuuint64_t dims[4] = {(cuuint64_t)s.m, d, (cuuint64_t)s.n_r, (cuuint64_t)s.n_outer};
+    const cuuint64_t str[3] = {(cuuint64_t)s.m, d * s.m, d * s.d_ff};
+    const cuuint32_t box[4] = {kUmmaBK, 128, 1, 1};
+    ok = encode8(&D->wd8_r, (const uint8_t*)wd8 + (size_t)s.shared_width * d, 4, dims, str, box, "FP8 routed W_down");
+  }
+  if (!ok) return false;
+  if (!P->has_r) D->wd8_r = D->wd8_s;
+  if (!P->has_s) D->wd8_s = D->wd8_r;
+  cudaError_t e = cudaSuccess;
+  auto attr = [&](auto kernel, int bytes) {
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  };
+  attr(umma_decode_kernel<4, false, true>, decode_smem_bytes<4, true>());
+  attr(umma_decode_kernel<4, true, true>, decode_smem_bytes<4, true>());
+  attr(umma_decode_kernel<5, false, true>, decode_smem_bytes<5, true>());
+  attr(umma_decode_kernel<5, true, true>, decode_smem_bytes<5, true>());
+  if (e != cudaSuccess) {
+    snprintf(P->error, sizeof(P->error), "cudaFuncSetAttribute (FP8 decode): %s", cudaGetErrorString(e));
+    return false;
+  }
+  D->scale_gu = scale_gu; D->scale_d = scale_d;
+  D->fp8 = true;
+  return true;
+}
+
 // Index of the smallest token box (16 << index rows) that holds n_rows rows.
 inline int decode_box_index(int n_rows) { return n_rows <= 16 ? 0 : (n_rows <= 32 ? 1 : 2); }
 
@@ -482,12 +635,22 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n
   a.part = D->part; a.ticket = D->ticket;
   const int bi = decode_box_index(n_rows);
   a.tok_box_rows = 16 << bi;
+  a.scale_gu = D->scale_gu; a.scale_d = D->scale_d; a.rows_w = (long long)s.n_outer * s.d_ff;
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
-  launch_kernel(dep, split1 ? umma_decode_kernel<4, true> : umma_decode_kernel<4, false>, dim3(P->n_sms),
-                dim3(kUmmaThreads), decode_smem_bytes<4>(), st, D->w_gu, D->w_gu, D->x_rows[bi], D->x_rows[bi], a);
+  if (D->fp8)       // the layer holds FP8 codes of its expert weights: stream those (half the bytes)
+    launch_kernel(dep, split1 ? umma_decode_kernel<4, true, true> : umma_decode_kernel<4, false, true>, dim3(P->n_sms),
+                  dim3(kDecThreadsW8), decode_smem_bytes<4, true>(), st, D->w_gu8, D->w_gu8, D->x_rows[bi],
+                  D->x_rows[bi], a);
+  else
+    launch_kernel(dep, split1 ? umma_decode_kernel<4, true> : umma_decode_kernel<4, false>, dim3(P->n_sms),
+                  dim3(kUmmaThreads), decode_smem_bytes<4>(), st, D->w_gu, D->w_gu, D->x_rows[bi], D->x_rows[bi], a);
   if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
-  if (!gate_up_only)
+  if (gate_up_only) {
+  } else if (D->fp8)
+    launch_kernel(dep, split2 ? umma_decode_kernel<5, true, true> : umma_decode_kernel<5, false, true>, dim3(P->n_sms),
+                  dim3(kDecThreadsW8), decode_smem_bytes<5, true>(), st, D->wd8_s, D->wd8_r, D->h_s[bi], D->h_r[bi], a);
+  else
     launch_kernel(dep, split2 ? umma_decode_kernel<5, true> : umma_decode_kernel<5, false>, dim3(P->n_sms),
                   dim3(kUmmaThreads), decode_smem_bytes<5>(), st, D->wd_s, D->wd_r, D->h_s[bi], D->h_r[bi], a);
   const cudaError_t e = cudaGetLastError();

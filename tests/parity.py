@@ -113,10 +113,12 @@ def check_output(got: np.ndarray, want: np.ndarray):
 
 
 def check_plain_layer(layer: binding.Layer, lay: wl.LayerInputs, x: np.ndarray,
-                      sample_tokens=None) -> dict:
+                      sample_tokens=None, expert_weights: Optional[dict] = None) -> dict:
     """One forward of a plain layer on x [T,d], compared stage by stage with the oracle.
     ``sample_tokens``: compare outputs only on these tokens (large workloads); an array, or a
-    callable (n_tok, counts, offsets, row_token) -> token ids such as ``stratified_tokens``."""
+    callable (n_tok, counts, offsets, row_token) -> token ids such as ``stratified_tokens``.
+    ``expert_weights``: w_gate / w_up / w_down the experts multiply by when they differ from the
+    layer's original weights (a quantised layer: the router still reads the originals)."""
     import torch
     s = lay.shape
     n_tok = x.shape[0]
@@ -142,7 +144,8 @@ def check_plain_layer(layer: binding.Layer, lay: wl.LayerInputs, x: np.ndarray,
         gates = np.zeros((n_tok, 0))
         if callable(sample_tokens):
             sample_tokens = sample_tokens(n_tok, [], [0], [])
-    want = oracle.moe_forward(x, lay.w_gate, lay.w_up, lay.w_down, lay.neuron_perm, s.n_experts,
+    ew = expert_weights or dict(w_gate=lay.w_gate, w_up=lay.w_up, w_down=lay.w_down)
+    want = oracle.moe_forward(x, ew["w_gate"], ew["w_up"], ew["w_down"], lay.neuron_perm, s.n_experts,
                               s.n_shared, sel, gates, token_ids=sample_tokens)
     if sample_tokens is not None:
         got = got[sample_tokens]
