@@ -175,6 +175,7 @@ SWEEP_POINTS = [("c2_llama2_7b", 1), ("c2_llama2_7b", 16), ("c2_llama2_7b", 64),
                 ("c2_llama2_7b", 4096), ("c3_llama3_8b", 32), ("c3_llama3_8b", 8192), ("c4_hier_8x7b", 4096),
                 ("c5_skew_13b", 16384)]
 HEADLINE = SWEEP_POINTS[-1]
+SWEEP_POINTS_FP8 = [("c2_llama2_7b", 1), ("c2_llama2_7b", 16), ("c2_llama2_7b", 64), ("c3_llama3_8b", 32)]
 
 
 def traffic_note(name, tokens, use_graph):
@@ -313,13 +314,15 @@ def dense_comparison(rig, inputs, x, steps, min_region_s=0.2):
     return {"kind": kind, "ms_per_step": dms, "value": T / (dms * 1e-3), "unit": UNIT}
 
 
-def roofline_record(peaks, w, T, touched, step_ms, first_ms, gemm_ms, stage_ms, use_graph):
+def roofline_record(peaks, w, T, touched, step_ms, first_ms, gemm_ms, stage_ms, use_graph, weight_bytes=None):
     """Algorithmic work of one forward against the measured peaks (flops 6 d m (N_s+N_k) per
     token; bytes = every touched expert's weights once + x read + out write)."""
     s = w.shape
     mult = w.outer_top_k if w.n_outer else 1
     flops = mult * T * 6 * s.d_model * s.m * (s.n_shared + s.top_k)
     w_bytes = (w.n_outer if w.n_outer else 1) * (s.n_shared + touched) * s.expert_weight_bytes()
+    if weight_bytes is not None:               # quantised weights: bytes per weight instead of the storage type's
+        w_bytes = w_bytes // s.elem_bytes * weight_bytes
     alg_bytes = w_bytes + 2 * T * s.d_model * s.elem_bytes
     t_tensor = flops / (peaks["bf16_tflops"] * 1e12)
     t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
@@ -346,7 +349,7 @@ def roofline_record(peaks, w, T, touched, step_ms, first_ms, gemm_ms, stage_ms, 
     return roof, w_bytes
 
 
-def measure_point(rig, inputs, layer, T, min_region_s, max_blocks, with_dense):
+def measure_point(rig, inputs, layer, T, min_region_s, max_blocks, with_dense, fp8=False):
     """Times the forward of `layer` on the first T tokens of the workload, device-resident.
     Returns the sweep record plus what the headline line needs."""
     torch, args = rig.torch, rig.args
@@ -403,9 +406,11 @@ def measure_point(rig, inputs, layer, T, min_region_s, max_blocks, with_dense):
         layer.forward(x, out)
         touched = int((layer.routing(T, s.n_routed)["counts"] > 0).sum())
     peaks = load_peaks()
-    roof, w_bytes = roofline_record(peaks, w, T, touched, step_ms, first_ms, gemm_ms, stage_ms, use_graph)
+    roof, w_bytes = roofline_record(peaks, w, T, touched, step_ms, first_ms, gemm_ms, stage_ms, use_graph,
+                                    weight_bytes=1 if (fp8 and T <= 64) else None)
     dense = dense_comparison(rig, inputs, x, args.steps) if (with_dense and rig.rank == 0) else None
-    rec = {"workload": w.name, "tokens": T, "ms_per_step": step_ms, "first_block_ms_per_step": first_ms,
+    rec = {"workload": w.name, "tokens": T, "expert_weights": "fp8 e4m3 + per-channel 2^k scale" if fp8 else s.dtype,
+           "ms_per_step": step_ms, "first_block_ms_per_step": first_ms,
            "blocks": len(blocks), "timed_region_s": sum(blocks) * 1e-3,
            "value": replica_throughput(rig.world, T, 1, step_ms), "unit": UNIT,
            "launch": "CUDA graph replay" if use_graph else "direct launches, chained",
@@ -433,6 +438,8 @@ def run_gpu(args):
     s = w.shape
     T = args.tokens or w.t_max
     layer = torch_io.layer_from_workload(inputs, w.t_max if T <= w.t_max else T)
+    if args.fp8:
+        layer.quantise_fp8()
 
     if args.forward_only:                     # profiling runs: nothing but the forward passes
         x = torch_io.to_device(inputs.x[:T], s.dtype)
@@ -450,7 +457,7 @@ def run_gpu(args):
 
     # ---- headline: device-resident, K-step blocks repeated over at least a second
     head, roof, (x, out, step, w_bytes) = measure_point(rig, inputs, layer, T, args.min_region_s, 400,
-                                                        with_dense=True)
+                                                        with_dense=True, fp8=args.fp8)
     launches = head["launches_per_step"] * args.steps
 
     # ---- end to end through the public host-buffer call: H2D and D2H copies inside the timed region
@@ -497,6 +504,20 @@ def run_gpu(args):
             for t_ in ts:
                 found[(n_, t_)], _, _ = measure_point(rig, inputs, layer, t_, args.sweep_region_s, 200, with_dense=True)
         sweep = [found[p_] for p_ in SWEEP_POINTS if p_ in found]
+        # decode points again with FP8 expert weights (quantising a layer is permanent, so these come last)
+        for n_ in dict.fromkeys(p_[0] for p_ in SWEEP_POINTS_FP8):
+            if n_ != name:
+                layer.destroy()
+                del inputs, layer
+                torch.cuda.empty_cache()
+                inputs = prepare_inputs(n_)
+                layer = torch_io.layer_from_workload(inputs, 64)
+                name = n_
+            layer.quantise_fp8()
+            for m_, t_ in SWEEP_POINTS_FP8:
+                if m_ == n_:
+                    rec, _, _ = measure_point(rig, inputs, layer, t_, args.sweep_region_s, 200, with_dense=False, fp8=True)
+                    sweep.append(rec)
 
     if rank != 0:
         rig.close()
@@ -793,6 +814,7 @@ def main():
                     help="programmatic dependent launches between the kernels of a forward (library default: on)")
     ap.add_argument("--gemm-path", type=int, default=0, choices=[0, 1, 2, 3],
                     help="expert-GEMM implementation (cmoe_layer_set_gemm_path); 0 = the library's choice")
+    ap.add_argument("--fp8", action="store_true", help="quantise the expert weights to FP8 (cmoe_layer_quantise_fp8) first")
     ap.add_argument("--sweep", choices=["auto", "on", "off"], default="auto",
                     help="add one record per (workload, T) point of the metric to the JSON line "
                          "(auto: on for the default single-GPU headline run)")

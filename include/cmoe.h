@@ -243,10 +243,11 @@ int cmoe_cluster_representatives(const int64_t* scaled_sq_dist, const int32_t* n
                                  int32_t n, int32_t n_clusters, int32_t* rep_neuron, void* stream);
 
 /* Choose the expert-GEMM implementation: 0 = automatic (tensor-core path when the
- * dtype is bf16 and the shape allows, else the plain SIMT path; for batches of at least 1024
- * rows each of the two GEMMs runs on CTA pairs when the padding of the expert groups to
- * 256-row tiles is expected to stay small), 1 = always SIMT, 2 = tensor-core with single-CTA
- * tiles only, 3 = tensor-core on CTA pairs (cta_group::2) for batches of at least 1024 rows;
+ * dtype is bf16 and the shape allows, else the plain SIMT path; for batches of at least 256
+ * rows each of the two GEMMs may run on CTA pairs: below 1024 rows because a pair fetches a third
+ * less operand data per SM, from 1024 rows when the padding of the expert groups to 256-row
+ * tiles is expected to stay small), 1 = always SIMT, 2 = tensor-core with single-CTA tiles
+ * only, 3 = tensor-core on CTA pairs (cta_group::2) for batches of at least 256 rows;
  * 2 and 3 return CMOE_ERR_INVALID_ARG if the layer cannot take the tensor-core path. */
 int cmoe_layer_set_gemm_path(cmoe_layer* layer, int32_t path);
 

@@ -50,7 +50,7 @@ int arg_fail(int code, const char* what) {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-constexpr int kPairMinRows = 1024;       // outer rows from which the expert GEMMs run on CTA pairs
+constexpr int kPairMinRows = 256;        // outer rows from which the expert GEMMs may run on CTA pairs
 constexpr int kTmaGatherMaxRows = 512;   // routed rows up to which gather4 replaces the permuted copy of x
 
 // Bump allocator over one device allocation (base == nullptr: measure only).
@@ -234,10 +234,10 @@ void carve_workspace(cmoe_layer* L, char* base) {
   L->perm_scratch = a.take<int32_t>(permute_scratch_bytes((int)R, (int)(G ? G : 1)) / 4);
   L->gr = a.take<GroupRows>(L->n_groups_total());
   L->err_word = a.take<int32_t>(1);
-  L->rsk_ticket = a.take<int32_t>(1);
+  L->rsk_ticket = a.take<int32_t>(kRskMaxChunks);
   L->share = a.take<float>(G ? G : 1);
   L->target = a.take<float>(G ? G : 1);
-  L->rsk_part = a.take<float>((size_t)kRskMaxSlices * kRskMaxRows * 64);
+  L->rsk_part = a.take<float>((size_t)kRskMaxChunks * kRskMaxSlices * kRskMaxRows * 64);
   L->x_perm = a.take<char>(P * d * esz);
   L->h_s = a.take<char>(R * L->shared_width() * esz);
   L->h_r = a.take<char>(P * L->m * esz);
@@ -392,14 +392,15 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
                                                  L->b, ooff, L->n_outer, L->scores, L->keys,      \
                                                  L->topk_idx, L->topk_gate)
     if constexpr (std::is_same<T, bf16>::value) {
-      if (use_umma && R >= 512) {
+      if (use_umma && R > kRskMaxRows * kRskMaxChunks) {
         if (umma_router_forward(&L->umma, R, ooff, L->err_word, st) < 0)
           return arg_fail(CMOE_ERR_CUDA, L->umma.error);
-      } else if (R <= kRskMaxRows && d <= kRskMaxSlices * kRskSliceK) {
-        perm_fused = G <= kRskFuseGroups;
+      } else if (R <= kRskMaxRows * kRskMaxChunks && d <= kRskMaxSlices * kRskSliceK) {
+        const int chunks = (R + kRskMaxRows - 1) / kRskMaxRows;       // 64-row chunks: the grid's second dimension
+        perm_fused = G <= kRskFuseGroups && chunks == 1;
         const bool sub8 = n_r <= 8 && R > 16;
         (sub8 ? router_splitk_kernel<true> : router_splitk_kernel<false>)
-            <<<(d + kRskSliceK - 1) / kRskSliceK, kRskThreads, 0, st>>>(
+            <<<dim3((d + kRskSliceK - 1) / kRskSliceK, chunks), kRskThreads, 0, st>>>(
             xo, R, d, n_r, L->n_rp, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->rsk_part,
             L->rsk_ticket, L->scores, L->keys, L->topk_idx, L->topk_gate, perm_fused ? 1 : 0, G, L->counts,
             L->offsets, L->row_token, L->row_of, po);
@@ -444,8 +445,12 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
       const double rows_s = (double)R / L->n_outer, rows_r = G > 0 ? (double)P / G : 0.0;
       const double w_s = (double)R * L->cfg.n_shared, w_r = (double)P;
       const double ratio = (w_s + w_r) > 0 ? (pad(rows_s) * w_s + pad(rows_r) * w_r) / (w_s + w_r) : 1.0;
-      if (ratio <= 1.03) pair_mask |= 1;
-      if (ratio <= 1.08 && L->m >= 512) pair_mask |= 2;
+      if (R < 1024 && !L->hier) {          // a few tiles per SM: operand fetch per SM is the limit, not padded MMA work
+        pair_mask = 1 | (L->m >= 512 ? 2 : 0);
+      } else {
+        if (ratio <= 1.03) pair_mask |= 1;
+        if (ratio <= 1.08 && L->m >= 512) pair_mask |= 2;
+      }
     }
   }
   const int gather_mode = P <= kTmaGatherMaxRows ? 1 : 2;
@@ -1002,7 +1007,7 @@ int cmoe_layer_status(cmoe_layer* L, int32_t* device_error_word) {
   // Clear the error word and every ticket so that the next forward starts from a clean state.
   cudaStream_t st = L->last_stream;
   CU_TRY(cudaMemsetAsync(L->err_word, 0, 4, st));
-  CU_TRY(cudaMemsetAsync(L->rsk_ticket, 0, 4, st));
+  CU_TRY(cudaMemsetAsync(L->rsk_ticket, 0, 4 * kRskMaxChunks, st));
   if (L->dec_ticket) CU_TRY(cudaMemsetAsync(L->dec_ticket, 0, L->n_dec_ticket * 4, st));
   if (L->rt_ticket) CU_TRY(cudaMemsetAsync(L->rt_ticket, 0, L->n_rt_ticket * 4, st));
   CU_TRY(cudaStreamSynchronize(st));

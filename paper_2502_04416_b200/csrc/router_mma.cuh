@@ -188,7 +188,11 @@ namespace cmoe {
 // logic, then resets the ticket for the next call.  With at most kRskFuseGroups routed
 // groups the same block goes on to the histogram / scan / permutation of the selections
 // (and the groups' row ranges), which saves two launches per decode step.
+// Batches of up to kRskMaxChunks * 64 rows run the same kernel on a two-dimensional grid: block
+// (s, c) owns k slice s of the 64-row chunk c, and each chunk has its own scratch and ticket (the
+// permutation is then left to the permutation kernels).
 constexpr int kRskMaxRows = 64;
+constexpr int kRskMaxChunks = 8;
 constexpr int kRskSliceK = 128;
 constexpr int kRskMaxSlices = 64;           // d <= 8192
 constexpr int kRskThreads = 256;
@@ -209,6 +213,14 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
   grid_dep_wait();
   grid_dep_trigger();
   static_assert(kRskThreads == kPermChunk, "the fused permutation is written for one 256-row chunk");
+  // this block's 64-row chunk: from here on rows are counted within the chunk
+  const int row_base = blockIdx.y * kRskMaxRows;
+  n_rows = min(kRskMaxRows, n_rows - row_base);
+  xo += (size_t)row_base * d;
+  scores += (size_t)row_base * n_r; keys += (size_t)row_base * n_r;
+  topk_idx += (size_t)row_base * n_k; topk_gate += (size_t)row_base * n_k;
+  part += (size_t)blockIdx.y * gridDim.x * kRskMaxRows * 64;
+  ticket += blockIdx.y;
   __shared__ __align__(16) float unit[8][16][kRmStride];       // [unit = half*m_tiles + m-tile][row in tile][n]
   __shared__ int row_group[kRskMaxRows];
   __shared__ int is_last;
@@ -218,7 +230,7 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
   const int m_tiles = (n_rows + 15) >> 4;
   const int k_base = blockIdx.x * kRskSliceK;
   for (int r = threadIdx.x; r < kRskMaxRows; r += kRskThreads)
-    row_group[r] = (outer_off && r < n_rows) ? find_outer(outer_off, n_outer, r) : 0;
+    row_group[r] = (outer_off && r < n_rows) ? find_outer(outer_off, n_outer, row_base + r) : 0;
   __syncthreads();
   const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
   const int un = warp;                           // at most 2 * 4 units for 8 warps

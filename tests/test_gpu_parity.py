@@ -64,6 +64,20 @@ def test_small_shapes(name, d, m, tokens, path):
     layer.destroy()
 
 
+@pytest.mark.parametrize("tokens", [65, 128, 200, 256, 513, 1000])
+def test_mid_size_batches(tokens):
+    """65 to 1023 rows: split-K router over 64-row chunks (up to 512 rows), CTA-pair GEMMs from 256
+    rows, groups of a few dozen to a few hundred rows with ragged tiles."""
+    inp = _inputs("c2_llama2_7b", d_model=512, tokens=(1000,), m=1376)
+    lay = inp.layers[0]
+    rng = np.random.default_rng(3)
+    lay.gate_scale_u = rng.normal(scale=0.5, size=lay.shape.n_routed).astype(np.float32)
+    layer = parity.gpu_layer(lay, 1000)
+    st = parity.check_plain_layer(layer, lay, inp.x[:tokens])
+    assert st["differing"] <= st["near_tie"]
+    layer.destroy()
+
+
 def test_cta_pair_gemms():
     """Expert GEMMs on tcgen05 CTA pairs (cta_group::2): groups with odd and even m-tile counts."""
     inp = _inputs("c2_llama2_7b", d_model=256, tokens=(1300, 1027), m=1376 // 4 * 4)
@@ -85,6 +99,8 @@ def test_hierarchical_small(path):
     st = parity.check_hier_layer(layer, inp, inp.x)
     assert st["differing"] <= st["near_tie"]
     st = parity.check_hier_layer(layer, inp, inp.x[:3])          # most outer experts empty
+    st = parity.check_hier_layer(layer, inp, inp.x[:100])        # 200 outer rows: router chunks straddle outer experts
+    assert st["differing"] <= st["near_tie"]
     layer.destroy()
 
 
