@@ -120,6 +120,7 @@ __device__ __forceinline__ int umma2_pairs(const UmmaArgs& p, int g) {
   return ((m_tiles + 1) >> 1) * umma_n_tiles<MODE>(p, g);
 }
 
+template <int MODE>
 __device__ __forceinline__ Pair2Coord umma2_decode(const UmmaArgs& p, const int32_t* tile_start, int t) {
   int lo = 0, hi = p.n_groups;
   while (hi - lo > 1) {
@@ -128,9 +129,15 @@ __device__ __forceinline__ Pair2Coord umma2_decode(const UmmaArgs& p, const int3
   }
   const int local = t - tile_start[lo];
   const GroupRows r = p.gr[lo];
+  // bands of row-tile pairs, row tiles fastest inside a band, then n-tiles (see umma_decode)
   const int m_pairs = ((r.count + kUmmaBM - 1) / kUmmaBM + 1) >> 1;
+  const int n_tiles = umma_n_tiles<MODE>(p, lo);
+  const int band_mp = max(p.band_mt >> 1, 1);
+  const int per_band = band_mp * n_tiles;
+  const int band = local / per_band, in_band = local - band * per_band;
+  const int cur_mp = min(band_mp, m_pairs - band * band_mp);
   Pair2Coord c;
-  c.g = lo; c.mp = local % m_pairs; c.nt = local / m_pairs; c.row0 = r.row0; c.count = r.count;
+  c.g = lo; c.nt = in_band / cur_mp; c.mp = band * band_mp + in_band % cur_mp; c.row0 = r.row0; c.count = r.count;
   return c;
 }
 
@@ -193,7 +200,7 @@ umma2_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_co
       uint32_t it = 0;
       bool ok = true;
       for (int t = pair_id; t < total_tiles && ok; t += n_pairs) {
-        const Pair2Coord c = umma2_decode(p, tile_start, t);
+        const Pair2Coord c = umma2_decode<MODE>(p, tile_start, t);
         const GroupStatic g = p.gs[c.g];
         const int row = c.row0 + (2 * c.mp + (int)rank) * kUmmaBM;     // this CTA's m-tile
         const CUtensorMap* ta = g.is_shared ? &tm_a_s : &tm_a_r;
@@ -232,7 +239,7 @@ umma2_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_co
       uint32_t it = 0, tile_n = 0;
       bool ok = true;
       for (int t = pair_id; t < total_tiles && ok; t += n_pairs, ++tile_n) {
-        const Pair2Coord c = umma2_decode(p, tile_start, t);
+        const Pair2Coord c = umma2_decode<MODE>(p, tile_start, t);
         const GroupStatic g = p.gs[c.g];
         int k_blocks, n_mma;
         if (MODE == 1) { k_blocks = k_blocks_fixed; n_mma = 2 * (g.is_shared ? p.bn_s : p.bn_r); }
@@ -283,7 +290,7 @@ umma2_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_co
     uint32_t it = 0;
     bool ok = true;
     for (int t = pair_id; t < total_tiles && ok; t += n_pairs) {
-      const Pair2Coord c = umma2_decode(p, tile_start, t);
+      const Pair2Coord c = umma2_decode<MODE>(p, tile_start, t);
       const GroupStatic g = p.gs[c.g];
       const bool mine = !g.is_shared && p.use_gather == 2;
       const bf16* src_row[8];
@@ -324,7 +331,7 @@ umma2_grouped_kernel(const __grid_constant__ CUtensorMap tm_a_s, const __grid_co
     uint32_t tile_n = 0;
     bool ok = true;
     for (int t = pair_id; t < total_tiles && ok; t += n_pairs, ++tile_n) {
-      const Pair2Coord c = umma2_decode(p, tile_start, t);
+      const Pair2Coord c = umma2_decode<MODE>(p, tile_start, t);
       const GroupStatic g = p.gs[c.g];
       const uint32_t buf = tile_n & 1, use = tile_n >> 1;
       if (!mbar_wait(accf0 + 8 * buf, use & 1, abort_flag, p.err, kErrWaitAccFull)) { ok = false; break; }
@@ -461,11 +468,13 @@ inline int umma2_forward(UmmaPlan* P, Umma2Plan* Q, DecodePlan* D, const GroupRo
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
   a.use_gather = gather_mode;
   a.x_rows_ptr = (const bf16*)x_rows;
+  a.band_mt = umma_band_tiles(s.d);
   if (which & 1)
     launch_kernel(dep, umma2_grouped_kernel<1>, dim3(grid), dim3(kU2Threads1), kU2SmemBytes, st,
                   P->x_rows, P->has_r ? P->x_perm : P->x_rows, Q->b1_s, Q->b1_r, a);
   if (mid && (which & 1)) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
+  a.band_mt = umma_band_tiles(s.shared_width > s.m ? s.shared_width : s.m);
   if (which & 2)
     launch_kernel(dep, umma2_grouped_kernel<2>, dim3(grid), dim3(kUmmaThreads), kU2SmemBytes, st, P->a2_s, P->a2_r,
                   D->wd_s, D->wd_r, a);
