@@ -78,6 +78,8 @@ struct DecodeArgs {
   float* part;           // [kDecMaxSlots][kDecSlotFloats] slice partials
   int32_t* ticket;       // [tiles][4 epilogue warps], zero between launches
   int tok_box_rows;      // rows of the token-tile TMA box (16, 32 or 64): no more than the batch needs
+  int early_units;       // plain gate/up form: tiles of the shared expert (group 0) that need nothing from the router
+  int n_rows_plain;      // rows of the batch (the shared expert's rows of a plain layer)
   // W8: power-of-two scales of the FP8 weight rows
   const float* scale_gu; // [2][rows_w]: gate plane, then up plane, packed neuron order
   const float* scale_d;  // [n_groups][d]: per group and output channel
@@ -98,7 +100,11 @@ __global__ void __launch_bounds__(W8 ? kDecThreadsW8 : kUmmaThreads, 1)
 umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_constant__ CUtensorMap tm_w_r,
                    const __grid_constant__ CUtensorMap tm_x_s, const __grid_constant__ CUtensorMap tm_x_r,
                    const DecodeArgs p) {
-  grid_dep_wait();
+  // The plain gate/up form looks at what the preceding kernel (the router) wrote as late as it can: a CTA
+  // whose first unit is a tile of the shared expert (p.early_units of them) streams that tile at once
+  // and only then waits for the router, so the shared expert's weights move under the router's latency.
+  constexpr bool kLazy = MODE == 4 && !SPLIT;
+  if constexpr (!kLazy) grid_dep_wait();
   grid_dep_trigger();
   using Cfg = DecodeCfg<MODE, W8>;
   constexpr int kStages = Cfg::kStages;
@@ -116,6 +122,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   // barrier block: full[8] empty[8] acc_full[2] acc_empty[2], tmem slot, abort flag, W8: conv_full[4] conv_empty[4]
   const uint32_t full0 = bars, empty0 = bars + 64, accf0 = bars + 128, acce0 = bars + 144;
   const uint32_t cfull0 = bars + 192, cempty0 = bars + 224;
+  const uint32_t tbl_bar = bars + 168;                           // kLazy: the unit table has been built
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_gen + 160);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
   DecGroup* grp = reinterpret_cast<DecGroup*>(bars_gen + 256);       // SPLIT: [n_groups + 1]
@@ -128,6 +135,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
     for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 4); }
     for (int c = 0; c < kConv; ++c) { mbar_init(cfull0 + 8 * c, kDecCvtWarps); mbar_init(cempty0 + 8 * c, 1); }
+    mbar_init(tbl_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -136,7 +144,9 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
     tmem_alloc(smem_u32(tmem_slot), kDecTmemCols);
     tmem_relinquish();
   }
-  if constexpr (!SPLIT) {
+  if constexpr (kLazy) {
+    // the table is built by the producer warp when a role first needs it (build_table below)
+  } else if constexpr (!SPLIT) {
     for (int g = threadIdx.x; g < p.n_groups; g += blockDim.x) {
       const int span = MODE == 4 ? p.gs[g].width : (p.gs[g].width > 0 ? p.d : 0);
       tile_start[g + 1] = p.gr[g].count > 0 ? (span + 127) / 128 : 0;
@@ -194,8 +204,40 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int total_units = SPLIT ? grp[p.n_groups].unit0 : tile_start[p.n_groups];
+  int total_units = kLazy ? 0 : (SPLIT ? grp[p.n_groups].unit0 : tile_start[p.n_groups]);
   const int cta = blockIdx.x, n_ctas = gridDim.x;
+  // kLazy: this CTA's first unit (snake round 0 = unit `cta`) is tile `cta` of the shared expert, group 0,
+  // whose rows are all of the batch: nothing the router writes is needed for it
+  const bool early = kLazy && cta < p.early_units;
+  bool tbl_seen = !kLazy;
+  // producer warp: wait for the router, count every group's tiles, publish the table
+  auto build_table = [&]() {
+    grid_dep_wait();
+    for (int g = lane; g < p.n_groups; g += 32)
+      tile_start[g + 1] = p.gr[g].count > 0 ? (p.gs[g].width + 127) / 128 : 0;
+    __syncwarp();
+    if (lane == 0) {
+      int run = 0;
+      tile_start[0] = 0;
+      for (int g = 0; g < p.n_groups; ++g) { run += tile_start[g + 1]; tile_start[g + 1] = run; }
+      mbar_arrive(tbl_bar);
+    }
+    __syncwarp();
+    total_units = tile_start[p.n_groups];
+    tbl_seen = true;
+  };
+  // every other role: wait for the table (bounded), then for the router's writes
+  auto await_table = [&]() -> bool {
+    if (!mbar_wait(tbl_bar, 0, abort_flag, p.err, kErrWaitFull)) return false;
+    grid_dep_wait();
+    total_units = tile_start[p.n_groups];
+    tbl_seen = true;
+    return true;
+  };
+  auto group_rows = [&](int gidx, bool first_early) {            // rows of a group; the early unit's are known
+    if (first_early) { GroupRows r; r.row0 = 0; r.count = p.n_rows_plain; return r; }
+    return p.gr[gidx];
+  };
 
   // unit -> group, tile within the group, K slice
   struct Unit { int gi, nt, z, n_z, kb0, kb1; };
@@ -227,18 +269,22 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
     return u;
   };
 
+  Unit early_unit;
+  early_unit.gi = 0; early_unit.nt = cta; early_unit.z = 0; early_unit.n_z = 1; early_unit.kb0 = 0; early_unit.kb1 = 0;
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (whole warp)
     uint32_t it = 0;
     bool ok = true;
     for (int round = 0; ok; ++round) {
-      const int t = snake_tile(round, cta, n_ctas, total_units);
+      const bool fe = early && round == 0;
+      if (!fe && !tbl_seen) build_table();
+      const int t = fe ? cta : snake_tile(round, cta, n_ctas, total_units);
       if (t < 0) break;
-      const Unit un = find_unit(t);
+      const Unit un = fe ? early_unit : find_unit(t);
       const int gi = un.gi, nt = un.nt;
       const GroupStatic g = p.gs[gi];
       // mode 4: token rows of the group's outer expert; mode 5: the group's own H rows
-      const GroupRows r = MODE == 4 ? p.gr[g.outer] : p.gr[gi];
+      const GroupRows r = MODE == 4 ? group_rows(g.outer, fe) : p.gr[gi];
       const CUtensorMap* tw = g.is_shared ? &tm_w_s : &tm_w_r;
       const CUtensorMap* tx = g.is_shared ? &tm_x_s : &tm_x_r;
       const int j = g.is_shared ? 0 : (gi - p.n_outer) - g.outer * p.n_r;
@@ -265,12 +311,14 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
       uint32_t it = 0;
       bool ok = true;
       for (int round = 0; ok; ++round) {
-        const int t = snake_tile(round, cta, n_ctas, total_units);
+        const bool fe = early && round == 0;
+        if (!fe && !tbl_seen && !await_table()) { ok = false; break; }
+        const int t = fe ? cta : snake_tile(round, cta, n_ctas, total_units);
         if (t < 0) break;
-        const Unit un = find_unit(t);
+        const Unit un = fe ? early_unit : find_unit(t);
         const int gi = un.gi;
         const GroupStatic g = p.gs[gi];
-        const int n_mma = ((MODE == 4 ? p.gr[g.outer].count : p.gr[gi].count) + 15) & ~15;   // columns, rounded to 16
+        const int n_mma = ((MODE == 4 ? group_rows(g.outer, fe).count : p.gr[gi].count) + 15) & ~15;   // columns, rounded to 16
         const uint32_t idesc = umma_idesc(n_mma);
         const uint32_t buf = round & 1, use = round >> 1;
         if (!mbar_wait(acce0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.err, kErrWaitAccEmpty)) { ok = false; break; }
@@ -315,9 +363,11 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
     uint32_t it = 0;
     bool ok = true;
     for (int round = 0; ok; ++round) {
-      const int t = snake_tile(round, cta, n_ctas, total_units);
+      const bool fe = early && round == 0;
+      if (!fe && !tbl_seen && !await_table()) { ok = false; break; }
+      const int t = fe ? cta : snake_tile(round, cta, n_ctas, total_units);
       if (t < 0) break;
-      const Unit un = find_unit(t);
+      const Unit un = fe ? early_unit : find_unit(t);
       const GroupStatic g = p.gs[un.gi];
       const int k_end = SPLIT ? un.kb1 : ((MODE == 4 ? p.d : g.width) + kUmmaBK - 1) / kUmmaBK;
       for (int kb = un.kb0; kb < k_end; ++kb, ++it) {
@@ -355,12 +405,14 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
     const int quad = warp & 3;
     bool ok = true;
     for (int round = 0; ok; ++round) {
-      const int t = snake_tile(round, cta, n_ctas, total_units);
+      const bool fe = early && round == 0;
+      if (!fe && !tbl_seen && !await_table()) { ok = false; break; }
+      const int t = fe ? cta : snake_tile(round, cta, n_ctas, total_units);
       if (t < 0) break;
-      const Unit un = find_unit(t);
+      const Unit un = fe ? early_unit : find_unit(t);
       const int gi = un.gi, nt = un.nt;
       const GroupStatic g = p.gs[gi];
-      const GroupRows r = p.gr[gi];
+      const GroupRows r = group_rows(gi, fe);
       const uint32_t buf = round & 1, use = round >> 1;
       if (!mbar_wait(accf0 + 8 * buf, use & 1, abort_flag, p.err, kErrWaitAccFull)) { ok = false; break; }
       tc_fence_after();
@@ -635,6 +687,9 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n
   a.part = D->part; a.ticket = D->ticket;
   const int bi = decode_box_index(n_rows);
   a.tok_box_rows = 16 << bi;
+  // plain layer: group 0 is the shared expert and its rows are the whole batch, known here
+  a.early_units = (s.n_outer == 1 && P->has_s) ? (s.shared_width + 127) / 128 : 0;
+  a.n_rows_plain = n_rows;
   a.scale_gu = D->scale_gu; a.scale_d = D->scale_d; a.rows_w = (long long)s.n_outer * s.d_ff;
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
   if (D->fp8)       // the layer holds FP8 codes of its expert weights: stream those (half the bytes)
