@@ -167,7 +167,16 @@ def prepare_inputs(name: str):
 # DRAM bytes (read + write) per forward of the dominant kernels (the two expert GEMMs), from the ncu
 # captures summarised under profiles/; an entry is only valid for the kernel version it was taken on,
 # so the table is emptied whenever those kernels change and refilled from a new capture.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    ("c5_skew_13b", 16384): {"bytes": (1586.5 + 162.8 + 363.8 + 795.8) * 1e6,
+                             "source": "profiles/umma2_pair_gemm_c5_skew_13b.md"},
+    ("c2_llama2_7b", 4096): {"bytes": (282.2 + 34.5 + 138.5 + 68.2) * 1e6,
+                             "source": "profiles/launch_lists_c2_c3_c4_prefill_and_mid_size.md"},
+    ("c3_llama3_8b", 8192): {"bytes": (517.0 + 52.0 + 182.0 + 281.5) * 1e6,
+                             "source": "profiles/launch_lists_c2_c3_c4_prefill_and_mid_size.md"},
+    ("c4_hier_8x7b", 4096): {"bytes": (2038.5 + 111.7 + 1064.4 + 184.3) * 1e6,
+                             "source": "profiles/launch_lists_c2_c3_c4_prefill_and_mid_size.md"},
+}
 
 # Every (workload, T) point the metric is quoted on; the last one (the largest single-GPU
 # configuration) is the headline.
@@ -415,7 +424,7 @@ def measure_point(rig, inputs, layer, T, min_region_s, max_blocks, with_dense, f
            "value": replica_throughput(rig.world, T, 1, step_ms), "unit": UNIT,
            "launch": "CUDA graph replay" if use_graph else "direct launches, chained",
            "launches_per_step": launches_per_step, "routed_experts_touched": touched,
-           "roofline": {k: roof[k] for k in ("bound", "frac", "achieved", "peak", "unit", "kernel_ms", "whole_step_frac",
+           "roofline": {k: roof[k] for k in ("bound", "frac", "achieved", "peak", "unit", "kernel_ms", "traffic", "whole_step_frac",
                                              "whole_step_frac_first_block", "whole_step_frac_of_sustained",
                                              "other_bound_frac", "stage_ms")},
            "dense_cublas": dense, "clocks": clocks}
