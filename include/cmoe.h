@@ -114,8 +114,9 @@ int cmoe_ffn_forward(cmoe_layer* layer, const void* x, int32_t T, void* out, voi
  *                      belong to the caller and must stay valid until `stream` has passed
  *                      this call; out_host is complete when work enqueued on `stream` after
  *                      the call runs (or after synchronising `stream`).
- *   chunk_tokens     : tokens per chunk, clamped to [1, max_tokens]; <= 0 picks an eighth
- *                      of the batch rounded up to 128 rows, at least 512.
+ *   chunk_tokens     : tokens per chunk, clamped to [1, max_tokens]; <= 0 picks a sixteenth
+ *                      of the batch rounded up to 128 rows, at least 512 (the first copy in and
+ *                      the last copy out are not overlapped, so more chunks hide more of them).
  * The first call (and any later call with a larger chunk) allocates the staging: two device
  * buffers each for x and out of chunk_tokens rows, two streams and a few events, all freed by
  * cmoe_layer_destroy; other calls allocate nothing.  Routing read-back afterwards (cmoe_get_routing)

@@ -702,8 +702,8 @@ int cmoe_ffn_forward_host(cmoe_layer* L, const void* x_host, int32_t T, void* ou
   if (!x_host || !out_host) return arg_fail(CMOE_ERR_INVALID_ARG, "null x / out");
   const size_t row_bytes = (size_t)L->cfg.d_model * L->esz;
   int chunk = chunk_tokens;
-  if (chunk <= 0) {                                  // an eighth of the batch, in whole 128-row tiles, at least 512
-    chunk = ((T + 7) / 8 + 127) / 128 * 128;
+  if (chunk <= 0) {                                  // a sixteenth of the batch, in whole 128-row tiles, at least 512
+    chunk = ((T + 15) / 16 + 127) / 128 * 128;
     if (chunk < 512) chunk = 512;
   }
   if (chunk > L->cfg.max_tokens) chunk = L->cfg.max_tokens;
