@@ -89,6 +89,7 @@ struct cmoe_layer {
   // FP8 copy of the expert weights (cmoe_layer_quantise_fp8): codes in the packed layouts, scales
   uint8_t *w_gu8 = nullptr, *wd8 = nullptr;
   float *scale_gu = nullptr, *scale_d = nullptr;
+  void* fp8_tok = nullptr;  // E4M3 planes and scales of the token rows of a decode-sized forward (one allocation)
   bool fp8 = false;
   GroupStatic* gs = nullptr;
   std::vector<GroupStatic> gs_host;
@@ -157,7 +158,7 @@ void free_layer(cmoe_layer* L) {
   if (L->hio.s_in) cudaStreamDestroy(L->hio.s_in);
   if (L->hio.s_out) cudaStreamDestroy(L->hio.s_out);
   umma_plan_destroy(&L->umma);
-  cudaFree(L->w_gu8); cudaFree(L->wd8); cudaFree(L->scale_gu); cudaFree(L->scale_d);
+  cudaFree(L->w_gu8); cudaFree(L->wd8); cudaFree(L->scale_gu); cudaFree(L->scale_d); cudaFree(L->fp8_tok);
   cudaFree(L->w_gu); cudaFree(L->wd_p); cudaFree(L->w_rep);
   cudaFree(L->w_router); cudaFree(L->u); cudaFree(L->b); cudaFree(L->gs); cudaFree(L->ws);
   delete L;
@@ -381,6 +382,10 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
   const bool decode = use_umma && R <= kDecMaxRows;      // weights-on-M streaming kernels
   if (use_umma && !umma_bind_x(&L->umma, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   if (decode && !decode_bind_x(&L->umma, &L->decode, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
+  if (decode && L->fp8) {                          // E4M3 planes of the token rows: independent of the routing
+    if (decode_split_x(&L->umma, &L->decode, R, st, false) < 0) return arg_fail(CMOE_ERR_CUDA, "split_rows launch failed");
+    ++launches;
+  }
   GroupPlanOut po;                                // the permutation also writes every group's row range
   po.gr = L->gr; po.n_outer = L->n_outer; po.n_tokens = n_tok; po.outer_off = L->hier ? L->outer_off : nullptr;
   bool perm_fused = false;                        // decode: the router's last block also permutes
@@ -795,7 +800,29 @@ int cmoe_layer_quantise_fp8(cmoe_layer* L, void* stream) {
   }
   CU_TRY(cudaGetLastError());
   CU_TRY(cudaStreamSynchronize(st));
-  if (!decode_plan_attach_fp8(&L->umma, &L->decode, L->w_gu8, L->wd8, L->scale_gu, L->scale_d))
+  // token planes for batches of at most kDecMaxRows outer rows: x, H_s (that many rows), H_r (rows x N_k)
+  DecodeFp8Buffers f{};
+  f.w_gu8 = L->w_gu8; f.wd8 = L->wd8; f.scale_gu = L->scale_gu; f.scale_d = L->scale_d;
+  f.xq_rows = kDecMaxRows;
+  f.hr_rows = (size_t)kDecMaxRows * (L->cfg.top_k > 0 ? L->cfg.top_k : 1);
+  {
+    Arena a;
+    auto carve = [&](char* base) {
+      a.base = base; a.used = 0;
+      f.xq = a.take<uint8_t>(2 * f.xq_rows * d);
+      f.hq_s = a.take<uint8_t>(2 * f.xq_rows * (L->shared_width() > 0 ? L->shared_width() : 16));
+      f.hq_r = a.take<uint8_t>(2 * f.hr_rows * L->m);
+      f.x_scale = a.take<float>(f.xq_rows);
+      f.hs_scale = a.take<float>(f.xq_rows);
+      f.hr_scale = a.take<float>(f.hr_rows);
+    };
+    carve(nullptr);
+    const size_t bytes = a.used + 256;
+    CU_TRY(cudaMalloc(&L->fp8_tok, bytes));
+    CU_TRY(cudaMemset(L->fp8_tok, 0, bytes));
+    carve(static_cast<char*>(L->fp8_tok));
+  }
+  if (!decode_plan_attach_fp8(&L->umma, &L->decode, f))
     return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   L->fp8 = true;
   return CMOE_OK;

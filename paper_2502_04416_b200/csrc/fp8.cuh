@@ -88,4 +88,64 @@ quantise_rows_fp8_kernel(const bf16* w, int rows, int cols, long long ld, uint8_
   }
 }
 
+// Splits bf16 rows into two E4M3 planes for the FP8 tensor-core path: with the row's power-of-two
+// scale 2^e (largest magnitude brought to at most 448), hi = E4M3(v / 2^e) and lo = E4M3(16 (v / 2^e - hi)).
+// A bf16 value has 8 significant bits, hi keeps the top 4 and the remainder is a multiple of the
+// value's last place not above 8 of them, so lo holds it exactly unless it falls below E4M3's range
+// (values under 2^-13 of the row's maximum): v = (hi + lo / 16) 2^e.  One block per row.
+__device__ __forceinline__ void split_row_e4m3(const bf16* __restrict__ row, int cols, uint8_t* __restrict__ h,
+                                               uint8_t* __restrict__ l, float* __restrict__ scale_out) {
+  __shared__ float red[4];
+  float amax = 0.0f;
+  for (int c = 8 * threadIdx.x; c < cols; c += 8 * 128) {
+    float v[8];
+    load8(row + c, v);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) { const float a = fabsf(v[q]); amax = (a > amax) ? a : amax; }
+  }
+  amax = warp_max(amax);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  const int e = pow2_scale_exponent(fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3])));
+  if (threadIdx.x == 0) *scale_out = ldexpf(1.0f, e);
+  for (int c = 8 * threadIdx.x; c < cols; c += 8 * 128) {
+    float v[8];
+    load8(row + c, v);
+    uint32_t hw[2], lw[2];
+#pragma unroll
+    for (int q = 0; q < 8; q += 2) {
+      const float v0 = ldexpf(v[q], -e), v1 = ldexpf(v[q + 1], -e);
+      const uint16_t hq = f32x2_to_e4m3x2(v0, v1);
+      const float2 back = e4m3x2_to_f32x2(hq);
+      const uint16_t lq = f32x2_to_e4m3x2((v0 - back.x) * 16.0f, (v1 - back.y) * 16.0f);
+      hw[q >> 2] = (q & 2) ? (hw[q >> 2] | ((uint32_t)hq << 16)) : (uint32_t)hq;
+      lw[q >> 2] = (q & 2) ? (lw[q >> 2] | ((uint32_t)lq << 16)) : (uint32_t)lq;
+    }
+    *reinterpret_cast<uint2*>(h + c) = make_uint2(hw[0], hw[1]);
+    *reinterpret_cast<uint2*>(l + c) = make_uint2(lw[0], lw[1]);
+  }
+}
+
+// One segment of rows: src [rows, cols] bf16 (leading dimension ld) -> planes [2][plane_rows][cols], scales [rows].
+struct SplitSegment {
+  const bf16* src;
+  int rows, cols;
+  long long ld;
+  uint8_t* planes;
+  long long plane_rows;
+  float* scale;
+};
+
+// Blocks 0 .. a.rows-1 split the rows of segment a, the next b.rows blocks those of segment b (b.rows may be 0).
+__global__ void __launch_bounds__(128) split_rows_e4m3_kernel(const SplitSegment a, const SplitSegment b) {
+  grid_dep_wait();
+  grid_dep_trigger();
+  int r = blockIdx.x;
+  const SplitSegment& sg = r < a.rows ? a : b;
+  if (r >= a.rows) r -= a.rows;
+  if (r >= sg.rows) return;
+  uint8_t* hi = sg.planes + (size_t)r * sg.cols;
+  split_row_e4m3(sg.src + (size_t)r * sg.ld, sg.cols, hi, hi + (size_t)sg.plane_rows * sg.cols, sg.scale + r);
+}
+
 }  // namespace cmoe

@@ -24,10 +24,14 @@
 // then right to left), which balances long shared-expert units against short routed ones.
 // Same warp roles, bounded waits and teardown as the token-major kernels.
 //
-// W8 = true streams FP8 (E4M3) weights, half the bytes: TMA lands the codes of a k block in a
-// raw ring (unswizzled, 64 bytes per weight row), eight converter warps expand them to bf16 in
-// the 128-byte-swizzled layout of a short second ring (exact, see fp8.cuh), the MMAs read that,
-// and the epilogue multiplies each weight row's sums by its power-of-two scale.
+// W8 = true streams FP8 (E4M3) weights, half the bytes, and multiplies them as they are:
+// tcgen05.mma kind::f8f6f4 on the codes, no conversion.  The bf16 token rows (x, H) are split
+// beforehand (split_rows_e4m3_kernel) into two E4M3 planes, hi = the value rounded to E4M3 and
+// lo = 16 x the remainder, after a per-row power-of-two scale; a bf16 number has 8 significant
+// bits and each plane carries 4, so hi + lo/16 is the value itself (exactly, down to 2^-13 of the
+// row's largest magnitude).  A stage covers 128 k (128 bytes per weight row, the same TMA box
+// geometry as the bf16 tiles), each k step issues one MMA per (weight plane, token plane) into
+// its own accumulator columns, and the epilogue forms (hi + lo/16) x row scale x token scale.
 #pragma once
 
 #include "fp8.cuh"
@@ -37,7 +41,6 @@ namespace cmoe {
 
 constexpr int kDecMaxRows = 64;            // rows per group this path takes
 constexpr int kDecXBytes = kDecMaxRows * kUmmaBK * 2;      // 8 KB token tile
-constexpr int kDecTmemCols = 256;          // two buffers of (64 gate + 64 up) columns
 
 constexpr int kDecMaxSplit = 8;            // K slices per tile at most
 constexpr int kDecMinSliceKb = 6;          // k blocks per slice at least
@@ -48,22 +51,21 @@ constexpr int kDecSlotFloats = 128 * 2 * kDecMaxRows;      // 128 weight rows x 
 struct DecGroup { int32_t unit0, tile0, slot0; int16_t z, kb; };
 constexpr int kDecInvOff = 256 + ((kUmmaMaxGroups + 1) * (int)sizeof(DecGroup) + 15) / 16 * 16;   // per-warp token tables
 
-constexpr int kDecCvtWarps = 8;            // W8: warps that expand FP8 codes to bf16
-constexpr int kDecThreadsW8 = kUmmaThreads + 32 * kDecCvtWarps;
-
-// kWBytes: bf16 weight tile(s) of one k block (what the MMAs read); kRawBytes: what TMA lands per
-// stage (the same tile for bf16 weights, the FP8 codes for W8); kConv: bf16 tiles of the W8 ring.
+// kWBytes: weight tile(s) of one stage: 128 rows x 128 bytes per plane (64 bf16 or 128 E4M3 k values);
+// kXBytes: token tile(s) of one stage (W8: the hi and the lo plane).
 template <int MODE, bool W8> struct DecodeCfg;
-template <> struct DecodeCfg<4, false> { static constexpr int kWBytes = 2 * 128 * kUmmaBK * 2, kRawBytes = kWBytes, kStages = 5, kConv = 0; };
-template <> struct DecodeCfg<5, false> { static constexpr int kWBytes = 128 * kUmmaBK * 2, kRawBytes = kWBytes, kStages = 8, kConv = 0; };
-template <> struct DecodeCfg<4, true> { static constexpr int kWBytes = 2 * 128 * kUmmaBK * 2, kRawBytes = kWBytes / 2, kStages = 5, kConv = 2; };
-template <> struct DecodeCfg<5, true> { static constexpr int kWBytes = 128 * kUmmaBK * 2, kRawBytes = kWBytes / 2, kStages = 8, kConv = 3; };
+template <> struct DecodeCfg<4, false> { static constexpr int kWBytes = 2 * 128 * 128, kXBytes = kDecXBytes, kStages = 5; };
+template <> struct DecodeCfg<5, false> { static constexpr int kWBytes = 128 * 128, kXBytes = kDecXBytes, kStages = 8; };
+template <> struct DecodeCfg<4, true> { static constexpr int kWBytes = 2 * 128 * 128, kXBytes = 2 * kDecXBytes, kStages = 4; };
+template <> struct DecodeCfg<5, true> { static constexpr int kWBytes = 128 * 128, kXBytes = 2 * kDecXBytes, kStages = 6; };
 
 template <int MODE, bool W8 = false>
 constexpr int decode_smem_bytes() {
   using C = DecodeCfg<MODE, W8>;
-  return 1024 + C::kStages * (C::kRawBytes + kDecXBytes) + C::kConv * C::kWBytes + kDecInvOff + 4 * 64 * 4;
+  return 1024 + C::kStages * (C::kWBytes + C::kXBytes) + kDecInvOff + 4 * 64 * 4;
 }
+// TMEM columns: two accumulator buffers of (weight planes x token planes) x 64 token columns
+template <int MODE, bool W8> struct DecodeTmem { static constexpr int kCols = (MODE == 4 && W8) ? 512 : 256; };
 
 struct DecodeArgs {
   const GroupStatic* gs;
@@ -80,7 +82,9 @@ struct DecodeArgs {
   int tok_box_rows;      // rows of the token-tile TMA box (16, 32 or 64): no more than the batch needs
   int early_units;       // plain gate/up form: tiles of the shared expert (group 0) that need nothing from the router
   int n_rows_plain;      // rows of the batch (the shared expert's rows of a plain layer)
-  // W8: power-of-two scales of the FP8 weight rows
+  // W8: per-row power-of-two scales of the token planes (x or H rows), then of the FP8 weight rows
+  const float* tok_scale_s;   // rows of the shared groups' token space (mode 4: x rows; mode 5: H_s rows)
+  const float* tok_scale_r;   // mode 4: x rows again; mode 5: H_r rows
   const float* scale_gu; // [2][rows_w]: gate plane, then up plane, packed neuron order
   const float* scale_d;  // [n_groups][d]: per group and output channel
   long long rows_w;      // n_outer * d_ff
@@ -96,7 +100,7 @@ __device__ __forceinline__ int snake_tile(int round, int cta, int n_ctas, int to
 // SPLIT = false is the plain form (one unit per tile, no scratch); the host picks SPLIT = true
 // only when even the largest possible set of active experts leaves tiles to split.
 template <int MODE, bool SPLIT, bool W8 = false>
-__global__ void __launch_bounds__(W8 ? kDecThreadsW8 : kUmmaThreads, 1)
+__global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_constant__ CUtensorMap tm_w_r,
                    const __grid_constant__ CUtensorMap tm_x_s, const __grid_constant__ CUtensorMap tm_x_r,
                    const DecodeArgs p) {
@@ -109,19 +113,18 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   using Cfg = DecodeCfg<MODE, W8>;
   constexpr int kStages = Cfg::kStages;
   constexpr int kWBytes = Cfg::kWBytes;
-  constexpr int kRawBytes = Cfg::kRawBytes;
-  constexpr int kConv = Cfg::kConv;
-  constexpr int kStageBytes = kRawBytes + kDecXBytes;
+  constexpr int kStageBytes = kWBytes + Cfg::kXBytes;
+  constexpr int kBK = W8 ? 2 * kUmmaBK : kUmmaBK;                // k per stage: 128 bytes of a weight row
+  constexpr int kBufCols = DecodeTmem<MODE, W8>::kCols / 2;     // accumulator columns per buffer
+  constexpr int kUpCol = W8 ? 128 : 64;                          // mode 4: first column of the up accumulators
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
-  const uint32_t conv0 = base + kStages * kStageBytes;           // W8: ring of converted bf16 tiles
-  const uint32_t bars = conv0 + kConv * kWBytes;
-  uint8_t* bars_gen = gen + kStages * kStageBytes + kConv * kWBytes;
-  // barrier block: full[8] empty[8] acc_full[2] acc_empty[2], tmem slot, abort flag, W8: conv_full[4] conv_empty[4]
+  const uint32_t bars = base + kStages * kStageBytes;
+  uint8_t* bars_gen = gen + kStages * kStageBytes;
+  // barrier block: full[8] empty[8] acc_full[2] acc_empty[2], tmem slot, abort flag, table barrier
   const uint32_t full0 = bars, empty0 = bars + 64, accf0 = bars + 128, acce0 = bars + 144;
-  const uint32_t cfull0 = bars + 192, cempty0 = bars + 224;
   const uint32_t tbl_bar = bars + 168;                           // kLazy: the unit table has been built
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_gen + 160);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
@@ -134,14 +137,13 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 4); }
-    for (int c = 0; c < kConv; ++c) { mbar_init(cfull0 + 8 * c, kDecCvtWarps); mbar_init(cempty0 + 8 * c, 1); }
     mbar_init(tbl_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(tmem_slot), kDecTmemCols);
+    tmem_alloc(smem_u32(tmem_slot), DecodeTmem<MODE, W8>::kCols);
     tmem_relinquish();
   }
   if constexpr (kLazy) {
@@ -162,7 +164,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
     for (int g = threadIdx.x; g < p.n_groups; g += blockDim.x) {
       const int span = MODE == 4 ? p.gs[g].width : (p.gs[g].width > 0 ? p.d : 0);
       grp[g].tile0 = p.gr[g].count > 0 ? (span + 127) / 128 : 0;
-      grp[g].kb = (int16_t)(((MODE == 4 ? p.d : p.gs[g].width) + kUmmaBK - 1) / kUmmaBK);
+      grp[g].kb = (int16_t)(((MODE == 4 ? p.d : p.gs[g].width) + kBK - 1) / kBK);
     }
     __syncthreads();
     if (warp == 0) {                 // unit / tile / slot prefix sums over the groups, 32 groups per step
@@ -171,7 +173,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   #pragma unroll
       for (int o = 16; o > 0; o >>= 1) all_kb += __shfl_xor_sync(0xffffffffu, all_kb, o);
       int per_cta = (all_kb + (int)gridDim.x - 1) / (int)gridDim.x;    // k blocks a CTA streams if all share evenly
-      if (per_cta < kDecMinSliceKb) per_cta = kDecMinSliceKb;
+      if (per_cta < kDecMinSliceKb * kUmmaBK / kBK) per_cta = kDecMinSliceKb * kUmmaBK / kBK;
       // sum over split groups of tiles * z <= all_kb / per_cta <= CTAs, so the slots suffice for grids up to kDecMaxSlots
       const bool may_split = (int)gridDim.x <= kDecMaxSlots;
       int units = 0, tiles = 0, slots = 0;
@@ -288,18 +290,23 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
       const CUtensorMap* tw = g.is_shared ? &tm_w_s : &tm_w_r;
       const CUtensorMap* tx = g.is_shared ? &tm_x_s : &tm_x_r;
       const int j = g.is_shared ? 0 : (gi - p.n_outer) - g.outer * p.n_r;
-      const int k_end = SPLIT ? un.kb1 : ((MODE == 4 ? p.d : g.width) + kUmmaBK - 1) / kUmmaBK;
+      const int k_end = SPLIT ? un.kb1 : ((MODE == 4 ? p.d : g.width) + kBK - 1) / kBK;
       for (int kb = un.kb0; kb < k_end; ++kb, ++it) {
         const uint32_t s = it % kStages, n = it / kStages;
         if (!mbar_wait(empty0 + 8 * s, (n & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
         const uint32_t fb = full0 + 8 * s;
-        const uint32_t sw = base + s * kStageBytes, sx = sw + kRawBytes;
+        const uint32_t sw = base + s * kStageBytes, sx = sw + kWBytes;
         if (lane == 0) {
-          mbar_expect_tx(fb, kRawBytes + p.tok_box_rows * kUmmaBK * 2);
-          if (MODE == 4) tma_load_3d(sw, tw, fb, kb * kUmmaBK, g.w_row0 + nt * 128, 0);
-          else if (g.is_shared) tma_load_3d(sw, tw, fb, kb * kUmmaBK, nt * 128, g.outer);
-          else tma_load_4d(sw, tw, fb, kb * kUmmaBK, nt * 128, j, g.outer);
-          tma_load_2d(sx, tx, fb, kb * kUmmaBK, r.row0);
+          mbar_expect_tx(fb, kWBytes + (W8 ? 2 : 1) * p.tok_box_rows * 128);
+          if (MODE == 4) tma_load_3d(sw, tw, fb, kb * kBK, g.w_row0 + nt * 128, 0);
+          else if (g.is_shared) tma_load_3d(sw, tw, fb, kb * kBK, nt * 128, g.outer);
+          else tma_load_4d(sw, tw, fb, kb * kBK, nt * 128, j, g.outer);
+          if constexpr (W8) {                   // token planes [k, row, plane]: hi, then lo
+            tma_load_3d(sx, tx, fb, kb * kBK, r.row0, 0);
+            tma_load_3d(sx + kDecXBytes, tx, fb, kb * kBK, r.row0, 1);
+          } else {
+            tma_load_2d(sx, tx, fb, kb * kBK, r.row0);
+          }
         }
         __syncwarp();
       }
@@ -319,85 +326,39 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         const int gi = un.gi;
         const GroupStatic g = p.gs[gi];
         const int n_mma = ((MODE == 4 ? group_rows(g.outer, fe).count : p.gr[gi].count) + 15) & ~15;   // columns, rounded to 16
-        const uint32_t idesc = umma_idesc(n_mma);
+        const uint32_t idesc = W8 ? umma_idesc_e4m3(n_mma) : umma_idesc(n_mma);
         const uint32_t buf = round & 1, use = round >> 1;
         if (!mbar_wait(acce0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.err, kErrWaitAccEmpty)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * 128;
-        const int k_end = SPLIT ? un.kb1 : ((MODE == 4 ? p.d : g.width) + kUmmaBK - 1) / kUmmaBK;
+        const uint32_t d_tmem = tmem_base + buf * kBufCols;
+        const int k_end = SPLIT ? un.kb1 : ((MODE == 4 ? p.d : g.width) + kBK - 1) / kBK;
         for (int kb = un.kb0; kb < k_end; ++kb, ++it) {
           const uint32_t s = it % kStages, n = it / kStages;
-          uint32_t sw = base + s * kStageBytes;
-          const uint32_t sx = sw + kRawBytes;
-          if constexpr (W8) {
-            // the converters waited for the stage's bytes (weights and tokens) before converting
-            const uint32_t c = it % kConv, cn = it / kConv;
-            if (!mbar_wait(cfull0 + 8 * c, cn & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
-            sw = conv0 + c * kWBytes;
-          } else {
-            if (!mbar_wait(full0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
-          }
+          const uint32_t sw = base + s * kStageBytes, sx = sw + kWBytes;
+          if (!mbar_wait(full0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
           tc_fence_after();
+          // four k steps of 32 bytes per 128-byte row: 16 bf16 or 32 E4M3 values each
 #pragma unroll
-          for (int k = 0; k < kUmmaBK / 16; ++k) {
+          for (int k = 0; k < 4; ++k) {
             const uint32_t acc = (kb != un.kb0 || k != 0) ? 1u : 0u;
-            umma_bf16(d_tmem, umma_smem_desc(sw + k * 32), umma_smem_desc(sx + k * 32), idesc, acc);
-            if (MODE == 4)
-              umma_bf16(d_tmem + 64, umma_smem_desc(sw + 128 * kUmmaBK * 2 + k * 32),
-                        umma_smem_desc(sx + k * 32), idesc, acc);
+            const uint64_t a_g = umma_smem_desc(sw + k * 32), a_u = umma_smem_desc(sw + 128 * 128 + k * 32);
+            const uint64_t b_hi = umma_smem_desc(sx + k * 32);
+            if constexpr (W8) {
+              const uint64_t b_lo = umma_smem_desc(sx + kDecXBytes + k * 32);
+              umma_e4m3(d_tmem, a_g, b_hi, idesc, acc);
+              umma_e4m3(d_tmem + 64, a_g, b_lo, idesc, acc);
+              if (MODE == 4) {
+                umma_e4m3(d_tmem + kUpCol, a_u, b_hi, idesc, acc);
+                umma_e4m3(d_tmem + kUpCol + 64, a_u, b_lo, idesc, acc);
+              }
+            } else {
+              umma_bf16(d_tmem, a_g, b_hi, idesc, acc);
+              if (MODE == 4) umma_bf16(d_tmem + kUpCol, a_u, b_hi, idesc, acc);
+            }
           }
           umma_commit(empty0 + 8 * s);
-          if constexpr (W8) umma_commit(cempty0 + 8 * (it % kConv));
         }
         if (ok) umma_commit(accf0 + 8 * buf);
-      }
-    }
-  } else if (W8 && warp >= 6) {
-    // ------------------------------------------------------------ FP8 -> bf16 converters (W8, warps 6..13)
-    // A pass of one warp expands 8 weight rows x 64 codes (512 contiguous raw bytes, 16 per lane)
-    // into 8 rows x 128 bytes of the swizzled bf16 tile: lane l holds codes 16c..16c+15 of row l/4
-    // (c = l % 4) and writes the row's 16-byte chunks 2c and 2c+1 at positions (chunk ^ (row & 7)).
-    constexpr int kRows = kRawBytes / kUmmaBK;                    // weight rows per k block (gate + up planes)
-    constexpr int kPasses = kRows / 8 / kDecCvtWarps;
-    const int cw = warp - 6;
-    uint32_t it = 0;
-    bool ok = true;
-    for (int round = 0; ok; ++round) {
-      const bool fe = early && round == 0;
-      if (!fe && !tbl_seen && !await_table()) { ok = false; break; }
-      const int t = fe ? cta : snake_tile(round, cta, n_ctas, total_units);
-      if (t < 0) break;
-      const Unit un = fe ? early_unit : find_unit(t);
-      const GroupStatic g = p.gs[un.gi];
-      const int k_end = SPLIT ? un.kb1 : ((MODE == 4 ? p.d : g.width) + kUmmaBK - 1) / kUmmaBK;
-      for (int kb = un.kb0; kb < k_end; ++kb, ++it) {
-        const uint32_t s = it % kStages, n = it / kStages;
-        const uint32_t c = it % (kConv > 0 ? kConv : 1), cn = it / (kConv > 0 ? kConv : 1);
-        if (!mbar_wait(full0 + 8 * s, n & 1, abort_flag, p.err, kErrWaitFull)) { ok = false; break; }
-        if (!mbar_wait(cempty0 + 8 * c, (cn & 1) ^ 1, abort_flag, p.err, kErrWaitEmpty)) { ok = false; break; }
-        const uint32_t src = base + s * kStageBytes, dstb = conv0 + c * kWBytes;
-#pragma unroll
-        for (int ps = 0; ps < kPasses; ++ps) {
-          const int row = (cw * kPasses + ps) * 8 + (lane >> 2);          // 0 .. kRows-1 (plane = row / 128)
-          const int ch = lane & 3;
-          uint32_t w0, w1, w2, w3;
-          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                       : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3) : "r"(src + row * kUmmaBK + ch * 16));
-          uint32_t o[8];
-          e4m3x4_to_bf16x4(w0, o[0], o[1]);
-          e4m3x4_to_bf16x4(w1, o[2], o[3]);
-          e4m3x4_to_bf16x4(w2, o[4], o[5]);
-          e4m3x4_to_bf16x4(w3, o[6], o[7]);
-          const uint32_t rb = dstb + row * 128;                           // planes are 128 rows x 128 bytes apart
-          const int sw7 = row & 7;
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                       ::"r"(rb + (((2 * ch) ^ sw7) << 4)), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                       ::"r"(rb + (((2 * ch + 1) ^ sw7) << 4)), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> tcgen05.mma reads
-        __syncwarp();
-        if (lane == 0) mbar_arrive(cfull0 + 8 * c);
       }
     }
   } else {
@@ -420,15 +381,20 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
       const int span = MODE == 4 ? g.width : p.d;
       const int ld = MODE == 4 ? (g.is_shared ? p.ld_out_s : p.ld_out_r) : p.d;
       bf16* dst = (g.is_shared ? p.out_s : p.out_r) + (size_t)r.row0 * ld + wr;
-      const uint32_t taddr = tmem_base + buf * 128 + ((uint32_t)(quad * 32) << 16);
+      const uint32_t taddr = tmem_base + buf * kBufCols + ((uint32_t)(quad * 32) << 16);
       // Columns of the accumulator: mode 5 and shared groups, the group's own rows in order;
       // routed groups in mode 4, every row of the outer expert -> position in the group or -1.
       const bool lookup = MODE == 4 && !g.is_shared;
       int32_t* inv = inv_tables + quad * 64;
       int n_cols = r.count;
+      // W8: per-token scale of accumulator column c = tok_scale[c]: mode 4, the x rows of the outer expert;
+      // mode 5, the group's own H rows
+      const float* tok_scale = nullptr;
+      if constexpr (W8) tok_scale = (g.is_shared ? p.tok_scale_s : p.tok_scale_r) + r.row0;
       if (lookup) {
         const GroupRows rs = p.gr[g.outer];
         n_cols = rs.count;
+        if constexpr (W8) tok_scale = p.tok_scale_r + rs.row0;
         __syncwarp();
         inv[lane] = -1; inv[lane + 32] = -1;
         __syncwarp();
@@ -451,18 +417,34 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         if (row_live && c < n_cols) {
           const int pos = lookup ? inv[c] : c;
           if (pos >= 0) {
-            if constexpr (W8) { a *= sc_a; b *= sc_b; }
+            if constexpr (W8) { const float ts = __ldg(tok_scale + c); a *= sc_a * ts; b *= sc_b * ts; }
             const float v = MODE == 4 ? a / (1.0f + __expf(-a)) * b : a;
             dst[(size_t)pos * ld] = __float2bfloat16_rn(v);
           }
         }
       };
+      // 16 accumulator columns of this thread's weight row(s); W8: hi plane + lo plane / 16
+      auto load16 = [&](int c0, float (&a)[16], float (&b)[16]) {
+        tmem_ld16(taddr + c0, a);
+        if (MODE == 4) tmem_ld16(taddr + kUpCol + c0, b);
+        if constexpr (W8) {
+          float al[16], bl[16];
+          tmem_ld16(taddr + 64 + c0, al);
+          if (MODE == 4) tmem_ld16(taddr + kUpCol + 64 + c0, bl);
+          tmem_ld_wait();
+#pragma unroll
+          for (int q = 0; q < 16; ++q) {
+            a[q] = fmaf(al[q], 0.0625f, a[q]);
+            if (MODE == 4) b[q] = fmaf(bl[q], 0.0625f, b[q]);
+          }
+        } else {
+          tmem_ld_wait();
+        }
+      };
       if (!SPLIT || un.n_z == 1) {
         for (int c0 = 0; c0 < n_cols; c0 += 16) {
           float a[16], b[16];
-          tmem_ld16(taddr + c0, a);
-          if (MODE == 4) tmem_ld16(taddr + 64 + c0, b);
-          tmem_ld_wait();
+          load16(c0, a, b);
 #pragma unroll
           for (int q = 0; q < 16; ++q) finish(c0 + q, a[q], MODE == 4 ? b[q] : 0.0f);
         }
@@ -476,9 +458,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         float* mine = p.part + (size_t)(slot0 + un.z) * kDecSlotFloats + quad * 32 + lane;
         for (int c0 = 0; c0 < n_cols; c0 += 16) {
           float a[16], b[16];
-          tmem_ld16(taddr + c0, a);
-          if (MODE == 4) tmem_ld16(taddr + 64 + c0, b);
-          tmem_ld_wait();
+          load16(c0, a, b);
 #pragma unroll
           for (int q = 0; q < 16; ++q) {
             if (c0 + q < n_cols) {
@@ -515,7 +495,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, kDecTmemCols);
+    tmem_dealloc(tmem_base, DecodeTmem<MODE, W8>::kCols);
   }
 }
 
@@ -530,10 +510,16 @@ struct DecodePlan {
   // its rows, so that a stage carries as little besides weights as possible
   CUtensorMap x_rows[3];            // x (bound per forward for a plain layer)
   CUtensorMap h_s[3], h_r[3];       // H
-  // FP8 weights (set by decode_plan_attach_fp8): codes in the packed layouts, 64-byte x 128-row boxes
+  // FP8 weights (set by decode_plan_attach_fp8): codes in the packed layouts, boxes of 128 k x 128 rows;
+  // E4M3 planes [2][rows][cols] of the token rows (x, H_s, H_r) with their per-row scales
   bool fp8 = false;
   CUtensorMap w_gu8, wd8_s, wd8_r;
   const float *scale_gu = nullptr, *scale_d = nullptr;
+  uint8_t *xq = nullptr, *hq_s = nullptr, *hq_r = nullptr;
+  float *x_scale = nullptr, *hs_scale = nullptr, *hr_scale = nullptr;
+  size_t xq_rows = 0, hr_rows = 0;               // rows per plane of xq / hq_s, and of hq_r
+  CUtensorMap xq_map[3], hqs_map[3], hqr_map[3]; // token boxes of 16 / 32 / 64 rows
+  const void* x_ptr = nullptr;                   // x of this forward (decode_bind_x)
 };
 
 inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
@@ -594,18 +580,25 @@ inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
   return true;
 }
 
-// Tensor maps over the FP8 codes of the packed weights (same shapes as the bf16 maps, one byte per
-// element, no swizzle: the converter warps read the raw tile linearly).  Needs d, m and the shared
-// width to be multiples of 16 (TMA strides).
-inline bool decode_plan_attach_fp8(UmmaPlan* P, DecodePlan* D, const void* w_gu8, const void* wd8,
-                                   const float* scale_gu, const float* scale_d) {
+// FP8 buffers of a quantised layer, all owned by the caller.  Weight codes in the packed layouts (maps: one
+// byte per element, boxes of 128 k x 128 rows, 128-byte swizzle; d, m and the shared width must be multiples
+// of 16 for the TMA strides); token planes [2][rows][cols] for x (xq_rows rows), H_s (xq_rows) and H_r (hr_rows).
+struct DecodeFp8Buffers {
+  const void *w_gu8, *wd8;
+  const float *scale_gu, *scale_d;
+  uint8_t *xq, *hq_s, *hq_r;
+  float *x_scale, *hs_scale, *hr_scale;
+  size_t xq_rows, hr_rows;
+};
+
+inline bool decode_plan_attach_fp8(UmmaPlan* P, DecodePlan* D, const DecodeFp8Buffers& f) {
   const UmmaShape& s = P->shape;
   const size_t d = s.d, rows_w = (size_t)s.n_outer * s.d_ff;
   auto encode8 = [&](CUtensorMap* tm, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* str,
                      const cuuint32_t* box, const char* what) {
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     const CUresult r = P->encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), dims, str,
-                                 box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                 box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
       snprintf(P->error, sizeof(P->error), "cuTensorMapEncodeTiled(%s) failed with CUresult %d", what, (int)r);
@@ -613,28 +606,43 @@ inline bool decode_plan_attach_fp8(UmmaPlan* P, DecodePlan* D, const void* w_gu8
     }
     return true;
   };
+  // token planes [2][rows][cols]: box 128 k x (16 << i) rows x 1 plane
+  auto encode_planes = [&](CUtensorMap* maps, const void* base, size_t rows, size_t cols, const char* what) {
+    for (int i = 0; i < 3; ++i) {
+      const cuuint64_t dims[3] = {cols, rows, 2};
+      const cuuint64_t str[2] = {cols, rows * cols};
+      const cuuint32_t box[3] = {2 * kUmmaBK, (cuuint32_t)(16 << i), 1};
+      if (!encode8(&maps[i], base, 3, dims, str, box, what)) return false;
+    }
+    return true;
+  };
   bool ok = true;
   {
     const cuuint64_t dims[3] = {d, rows_w, 2};
     const cuuint64_t str[2] = {d, rows_w * d};
-    const cuuint32_t box[3] = {kUmmaBK, 128, 2};
-    ok = encode8(&D->w_gu8, w_gu8, 3, dims, str, box, "FP8 gate/up weights");
+    const cuuint32_t box[3] = {2 * kUmmaBK, 128, 2};
+    ok = encode8(&D->w_gu8, f.w_gu8, 3, dims, str, box, "FP8 gate/up weights");
   }
+  if (ok) ok = encode_planes(D->xq_map, f.xq, f.xq_rows, d, "E4M3 planes of x");
   if (ok && P->has_s) {
     const cuuint64_t dims[3] = {(cuuint64_t)s.shared_width, d, (cuuint64_t)s.n_outer};
     const cuuint64_t str[2] = {(cuuint64_t)s.shared_width, d * s.d_ff};
-    const cuuint32_t box[3] = {kUmmaBK, 128, 1};
-    ok = encode8(&D->wd8_s, wd8, 3, dims, str, box, "FP8 shared W_down");
+    const cuuint32_t box[3] = {2 * kUmmaBK, 128, 1};
+    ok = encode8(&D->wd8_s, f.wd8, 3, dims, str, box, "FP8 shared W_down") &&
+         encode_planes(D->hqs_map, f.hq_s, f.xq_rows, (size_t)s.shared_width, "E4M3 planes of H shared");
   }
   if (ok && P->has_r) {
     const cuuint64_t dims[4] = {(cuuint64_t)s.m, d, (cuuint64_t)s.n_r, (cuuint64_t)s.n_outer};
     const cuuint64_t str[3] = {(cuuint64_t)s.m, d * s.m, d * s.d_ff};
-    const cuuint32_t box[4] = {kUmmaBK, 128, 1, 1};
-    ok = encode8(&D->wd8_r, (const uint8_t*)wd8 + (size_t)s.shared_width * d, 4, dims, str, box, "FP8 routed W_down");
+    const cuuint32_t box[4] = {2 * kUmmaBK, 128, 1, 1};
+    ok = encode8(&D->wd8_r, (const uint8_t*)f.wd8 + (size_t)s.shared_width * d, 4, dims, str, box, "FP8 routed W_down") &&
+         encode_planes(D->hqr_map, f.hq_r, f.hr_rows, (size_t)s.m, "E4M3 planes of H routed");
   }
   if (!ok) return false;
-  if (!P->has_r) D->wd8_r = D->wd8_s;
-  if (!P->has_s) D->wd8_s = D->wd8_r;
+  for (int i = 0; i < 3; ++i) {
+    if (!P->has_r) { D->wd8_r = D->wd8_s; D->hqr_map[i] = D->hqs_map[i]; }
+    if (!P->has_s) { D->wd8_s = D->wd8_r; D->hqs_map[i] = D->hqr_map[i]; }
+  }
   cudaError_t e = cudaSuccess;
   auto attr = [&](auto kernel, int bytes) {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
@@ -647,7 +655,10 @@ inline bool decode_plan_attach_fp8(UmmaPlan* P, DecodePlan* D, const void* w_gu8
     snprintf(P->error, sizeof(P->error), "cudaFuncSetAttribute (FP8 decode): %s", cudaGetErrorString(e));
     return false;
   }
-  D->scale_gu = scale_gu; D->scale_d = scale_d;
+  D->scale_gu = f.scale_gu; D->scale_d = f.scale_d;
+  D->xq = f.xq; D->hq_s = f.hq_s; D->hq_r = f.hq_r;
+  D->x_scale = f.x_scale; D->hs_scale = f.hs_scale; D->hr_scale = f.hr_scale;
+  D->xq_rows = f.xq_rows; D->hr_rows = f.hr_rows;
   D->fp8 = true;
   return true;
 }
@@ -656,9 +667,18 @@ inline bool decode_plan_attach_fp8(UmmaPlan* P, DecodePlan* D, const void* w_gu8
 inline int decode_box_index(int n_rows) { return n_rows <= 16 ? 0 : (n_rows <= 32 ? 1 : 2); }
 
 inline bool decode_bind_x(UmmaPlan* P, DecodePlan* D, const void* x_rows, int n_rows) {
+  D->x_ptr = x_rows;
   if (P->buf.x_fixed) return true;
   const int bi = decode_box_index(n_rows);
   return umma_encode_rows(P, &D->x_rows[bi], x_rows, (size_t)n_rows, (size_t)P->shape.d, 16 << bi, "x (decode)");
+}
+
+// FP8 layers: the E4M3 planes of this forward's x rows (needs nothing from the router, so it is launched first).
+inline int decode_split_x(UmmaPlan* P, DecodePlan* D, int n_rows, cudaStream_t st, bool dep) {
+  SplitSegment a{(const bf16*)D->x_ptr, n_rows, P->shape.d, (long long)P->shape.d, D->xq, (long long)D->xq_rows, D->x_scale};
+  SplitSegment none{nullptr, 0, 0, 0, nullptr, 0, nullptr};
+  launch_kernel(dep, split_rows_e4m3_kernel, dim3(n_rows), dim3(128), 0, st, a, none);
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
 // Both decode GEMMs; requires umma_bind_x and decode_bind_x for this forward and n_rows <=
@@ -671,13 +691,13 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n
   const long long act_s = P->has_s ? (s.n_outer < n_rows ? s.n_outer : n_rows) : 0;
   const long long all_r = (long long)s.n_outer * s.n_r, picks = (long long)n_rows * s.n_k;
   const long long act_r = P->has_r ? (all_r < picks ? all_r : picks) : 0;
+  const int bk = D->fp8 ? 2 * kUmmaBK : kUmmaBK;               // k per stage, as in the kernel
   auto splits = [&](long long all_kb, int kb_max) {
     long long per_cta = (all_kb + P->n_sms - 1) / P->n_sms;
-    if (per_cta < kDecMinSliceKb) per_cta = kDecMinSliceKb;
+    if (per_cta < kDecMinSliceKb * kUmmaBK / bk) per_cta = kDecMinSliceKb * kUmmaBK / bk;
     return D->part != nullptr && P->n_sms <= kDecMaxSlots && kb_max / per_cta >= 2;
   };
-  const int kb_d = (s.d + kUmmaBK - 1) / kUmmaBK, kb_s = (s.shared_width + kUmmaBK - 1) / kUmmaBK,
-            kb_m = (s.m + kUmmaBK - 1) / kUmmaBK;
+  const int kb_d = (s.d + bk - 1) / bk, kb_s = (s.shared_width + bk - 1) / bk, kb_m = (s.m + bk - 1) / bk;
   const bool split1 = splits((act_s * ((s.shared_width + 127) / 128) + act_r * ((s.m + 127) / 128)) * kb_d, kb_d);
   const bool split2 = splits((long long)((s.d + 127) / 128) * (act_s * kb_s + act_r * kb_m),
                              (act_s && kb_s > kb_m) || !act_r ? kb_s : kb_m);
@@ -692,20 +712,30 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n
   a.n_rows_plain = n_rows;
   a.scale_gu = D->scale_gu; a.scale_d = D->scale_d; a.rows_w = (long long)s.n_outer * s.d_ff;
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
+  int extra = 0;
+  a.tok_scale_s = D->x_scale; a.tok_scale_r = D->x_scale;
   if (D->fp8)       // the layer holds FP8 codes of its expert weights: stream those (half the bytes)
     launch_kernel(dep, split1 ? umma_decode_kernel<4, true, true> : umma_decode_kernel<4, false, true>, dim3(P->n_sms),
-                  dim3(kDecThreadsW8), decode_smem_bytes<4, true>(), st, D->w_gu8, D->w_gu8, D->x_rows[bi],
-                  D->x_rows[bi], a);
+                  dim3(kUmmaThreads), decode_smem_bytes<4, true>(), st, D->w_gu8, D->w_gu8, D->xq_map[bi],
+                  D->xq_map[bi], a);
   else
     launch_kernel(dep, split1 ? umma_decode_kernel<4, true> : umma_decode_kernel<4, false>, dim3(P->n_sms),
                   dim3(kUmmaThreads), decode_smem_bytes<4>(), st, D->w_gu, D->w_gu, D->x_rows[bi], D->x_rows[bi], a);
   if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
   if (gate_up_only) {
-  } else if (D->fp8)
+  } else if (D->fp8) {
+    // E4M3 planes of H (shared rows, then routed rows), then the down GEMM on them
+    const int rows_r = P->has_r ? n_rows * s.n_k : 0, rows_s = P->has_s ? n_rows : 0;
+    SplitSegment hs{(const bf16*)P->buf.h_s, rows_s, s.shared_width, (long long)s.shared_width, D->hq_s,
+                    (long long)D->xq_rows, D->hs_scale};
+    SplitSegment hr{(const bf16*)P->buf.h_r, rows_r, s.m, (long long)s.m, D->hq_r, (long long)D->hr_rows, D->hr_scale};
+    launch_kernel(dep, split_rows_e4m3_kernel, dim3(rows_s + rows_r), dim3(128), 0, st, hs, hr);
+    extra = 1;
+    a.tok_scale_s = D->hs_scale; a.tok_scale_r = D->hr_scale;
     launch_kernel(dep, split2 ? umma_decode_kernel<5, true, true> : umma_decode_kernel<5, false, true>, dim3(P->n_sms),
-                  dim3(kDecThreadsW8), decode_smem_bytes<5, true>(), st, D->wd8_s, D->wd8_r, D->h_s[bi], D->h_r[bi], a);
-  else
+                  dim3(kUmmaThreads), decode_smem_bytes<5, true>(), st, D->wd8_s, D->wd8_r, D->hqs_map[bi], D->hqr_map[bi], a);
+  } else
     launch_kernel(dep, split2 ? umma_decode_kernel<5, true> : umma_decode_kernel<5, false>, dim3(P->n_sms),
                   dim3(kUmmaThreads), decode_smem_bytes<5>(), st, D->wd_s, D->wd_r, D->h_s[bi], D->h_r[bi], a);
   const cudaError_t e = cudaGetLastError();
@@ -713,7 +743,7 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n
     snprintf(P->error, sizeof(P->error), "decode GEMM launch: %s", cudaGetErrorString(e));
     return -1;
   }
-  return gate_up_only ? 1 : 2;
+  return (gate_up_only ? 1 : 2) + extra;
 }
 
 }  // namespace cmoe

@@ -139,6 +139,15 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// D[tmem] (+)= A[smem desc] * B[smem desc]^T, E4M3 inputs (32 k values per step), fp32 accumulate.
+__device__ __forceinline__ void umma_e4m3(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
 // mbarrier arrives once all tcgen05 operations issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -187,6 +196,11 @@ __global__ void wait_timeout_probe_kernel(int32_t* err_word, long long limit) {
   __syncwarp();
   if (threadIdx.x == 0) mbar_wait(bar, 0, &abort_flag, err_word, kErrWaitFull, limit);
   __syncwarp();
+}
+
+// Instruction descriptor of kind::f8f6f4: E4M3 x E4M3 (operand format code 0) -> fp32, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc_e4m3(int n) {
+  return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kUmmaBM >> 4) << 24);
 }
 
 // ----------------------------------------------------------------------------- kernel
