@@ -301,9 +301,9 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
           if (MODE == 4) tma_load_3d(sw, tw, fb, kb * kBK, g.w_row0 + nt * 128, 0);
           else if (g.is_shared) tma_load_3d(sw, tw, fb, kb * kBK, nt * 128, g.outer);
           else tma_load_4d(sw, tw, fb, kb * kBK, nt * 128, j, g.outer);
-          if constexpr (W8) {                   // token planes [k, row, plane]: hi, then lo
+          if constexpr (W8) {                   // token planes [k, row, plane]: the hi rows, directly behind them the lo rows
             tma_load_3d(sx, tx, fb, kb * kBK, r.row0, 0);
-            tma_load_3d(sx + kDecXBytes, tx, fb, kb * kBK, r.row0, 1);
+            tma_load_3d(sx + p.tok_box_rows * 128, tx, fb, kb * kBK, r.row0, 1);
           } else {
             tma_load_2d(sx, tx, fb, kb * kBK, r.row0);
           }
@@ -326,7 +326,9 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         const int gi = un.gi;
         const GroupStatic g = p.gs[gi];
         const int n_mma = ((MODE == 4 ? group_rows(g.outer, fe).count : p.gr[gi].count) + 15) & ~15;   // columns, rounded to 16
-        const uint32_t idesc = W8 ? umma_idesc_e4m3(n_mma) : umma_idesc(n_mma);
+        // W8: one MMA covers both token planes (N = hi rows + lo rows, adjacent in the stage): the decode
+        // kernels are bound by the number of MMAs a tile takes (~115 cycles each at these small N), not by bytes
+        const uint32_t idesc = W8 ? umma_idesc_e4m3(2 * p.tok_box_rows) : umma_idesc(n_mma);
         const uint32_t buf = round & 1, use = round >> 1;
         if (!mbar_wait(acce0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.err, kErrWaitAccEmpty)) { ok = false; break; }
         tc_fence_after();
@@ -344,13 +346,8 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
             const uint64_t a_g = umma_smem_desc(sw + k * 32), a_u = umma_smem_desc(sw + 128 * 128 + k * 32);
             const uint64_t b_hi = umma_smem_desc(sx + k * 32);
             if constexpr (W8) {
-              const uint64_t b_lo = umma_smem_desc(sx + kDecXBytes + k * 32);
               umma_e4m3(d_tmem, a_g, b_hi, idesc, acc);
-              umma_e4m3(d_tmem + 64, a_g, b_lo, idesc, acc);
-              if (MODE == 4) {
-                umma_e4m3(d_tmem + kUpCol, a_u, b_hi, idesc, acc);
-                umma_e4m3(d_tmem + kUpCol + 64, a_u, b_lo, idesc, acc);
-              }
+              if (MODE == 4) umma_e4m3(d_tmem + kUpCol, a_u, b_hi, idesc, acc);
             } else {
               umma_bf16(d_tmem, a_g, b_hi, idesc, acc);
               if (MODE == 4) umma_bf16(d_tmem + kUpCol, a_u, b_hi, idesc, acc);
@@ -428,9 +425,9 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         tmem_ld16(taddr + c0, a);
         if (MODE == 4) tmem_ld16(taddr + kUpCol + c0, b);
         if constexpr (W8) {
-          float al[16], bl[16];
-          tmem_ld16(taddr + 64 + c0, al);
-          if (MODE == 4) tmem_ld16(taddr + kUpCol + 64 + c0, bl);
+          float al[16], bl[16];                       // the lo plane's columns follow the hi plane's tok_box_rows
+          tmem_ld16(taddr + p.tok_box_rows + c0, al);
+          if (MODE == 4) tmem_ld16(taddr + kUpCol + p.tok_box_rows + c0, bl);
           tmem_ld_wait();
 #pragma unroll
           for (int q = 0; q < 16; ++q) {
