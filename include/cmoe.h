@@ -145,8 +145,9 @@ int cmoe_quantise_rows_fp8(const void* w, int32_t rows, int32_t cols, uint8_t* c
  * (the N_s shared experts form one block), so W_down has one scale per (expert, model dimension).
  * The router's representative rows keep their original values, so the routing does not change.
  * Afterwards every forward of the layer computes with the dequantised weights code * scale:
- * batches of at most 64 rows stream the FP8 codes (half the weight bytes of bf16) and expand
- * them to bf16 on the fly, larger batches read bf16 copies holding exactly the same values.
+ * batches of at most 64 rows stream the FP8 codes (half the weight bytes of bf16) into FP8
+ * tensor-core instructions, with every bf16 token row split into two E4M3 planes whose sum is
+ * the bf16 value itself; larger batches read bf16 copies holding exactly the same weight values.
  * The layer then owns 1.5x the weight memory.  Plain and hierarchical layers; needs d_model, the
  * expert width and the shared width to be multiples of 16.  Allocates (a set-up call, like create)
  * and synchronises `stream`.  Idempotent.  Errors: INVALID_ARG, UNSUPPORTED (fp32 layer, shape), CUDA. */
