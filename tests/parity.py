@@ -212,9 +212,10 @@ def stratified_tokens(n_tok: int, counts, offsets, row_token, seed: int, n_rando
 
 
 def check_hier_layer(layer: binding.Layer, inputs: wl.WorkloadInputs, x: np.ndarray,
-                     sample_tokens=None) -> dict:
+                     sample_tokens=None, expert_weights=None) -> dict:
     """Hierarchical layer: outer routing, per-outer-expert inner routing, flattened
-    permutation over n_outer*N_r groups, output."""
+    permutation over n_outer*N_r groups, output.  ``expert_weights``: per outer expert, the weights its
+    experts multiply by when they differ from the originals (a quantised layer)."""
     import torch
     w = inputs.workload
     s = w.shape
@@ -262,7 +263,8 @@ def check_hier_layer(layer: binding.Layer, inputs: wl.WorkloadInputs, x: np.ndar
         pos = np.array([p for p, _ in hit])
         toks = np.array([t for _, t in hit])
         rows = np.array([row_of_tok[(int(t), i)] for t in toks])
-        y = oracle.moe_forward(x[toks], lay.w_gate, lay.w_up, lay.w_down, lay.neuron_perm,
+        ew = expert_weights[i] if expert_weights is not None else dict(w_gate=lay.w_gate, w_up=lay.w_up, w_down=lay.w_down)
+        y = oracle.moe_forward(x[toks], ew["w_gate"], ew["w_up"], ew["w_down"], lay.neuron_perm,
                                s.n_experts, s.n_shared, sel_global[rows] - i * nr, gates_all[rows])
         wt = np.array([o_w[t, list(o_idx[t]).index(i)] for t in toks])
         want[pos] += wt[:, None] * y

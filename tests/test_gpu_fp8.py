@@ -95,6 +95,20 @@ def test_subnormal_codes_reach_the_output():
     layer.destroy()
 
 
+def test_quantised_hierarchical_layer():
+    """FP8 weights under a top-level router (Section 4.4): every outer expert's blocks get their own scales;
+    decode-sized batches (outer rows <= 64) stream the codes, larger ones read the dequantised bf16 copies."""
+    inp = wl.make_inputs(wl.shrunk(wl.WORKLOADS["c4_hier_8x7b"], d_model=256, tokens=(150,), m=224))
+    inners = [parity.gpu_layer(lay, 8) for lay in inp.layers]
+    layer = binding.Layer.create_hier(parity.to_device(inp.w_router, "bf16"), inners, 2, 150)
+    layer.quantise_fp8()
+    q = [_quantised(lay) for lay in inp.layers]
+    for t in (3, 20, 32, 150):
+        st = parity.check_hier_layer(layer, inp, inp.x[:t], expert_weights=q)
+        assert st["differing"] <= st["near_tie"]
+    layer.destroy()
+
+
 def test_quantise_refusals():
     inp = wl.make_inputs(wl.WORKLOADS["c1_tiny_fp32"])
     layer = parity.gpu_layer(inp.layers[0], 64)
