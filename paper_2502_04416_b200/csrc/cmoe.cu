@@ -379,7 +379,13 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
     xo = (const T*)L->xo;
   }
 
-  const bool decode = use_umma && R <= kDecMaxRows;      // weights-on-M streaming kernels
+  // Weights-on-M streaming kernels: up to 64 rows; on bf16 weights (the FP8 token planes stop at 64) the wide
+  // form takes up to 128 rows, or up to 96 when 128-neuron tiles pad the expert width by more than 5 %
+  // (measured: a 448-wide expert's token-major 112-neuron tiles win from there).  Path 2 keeps token-major tiles.
+  int decode_rows = kDecMaxRows;
+  if (!L->fp8 && L->gemm_path != 2)
+    decode_rows = ((L->m + 127) / 128 * 128) * 100LL <= 105LL * L->m ? kDecWideRows : 96;
+  const bool decode = use_umma && R <= decode_rows;
   if (use_umma && !umma_bind_x(&L->umma, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   if (decode && !decode_bind_x(&L->umma, &L->decode, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   if (decode && L->fp8) {                          // E4M3 planes of the token rows: independent of the routing

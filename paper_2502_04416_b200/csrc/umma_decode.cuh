@@ -39,8 +39,8 @@
 
 namespace cmoe {
 
-constexpr int kDecMaxRows = 64;            // rows per group this path takes
-constexpr int kDecXBytes = kDecMaxRows * kUmmaBK * 2;      // 8 KB token tile
+constexpr int kDecMaxRows = 64;            // rows per group of the narrow kernels (every FP8 and K-splitting form)
+constexpr int kDecWideRows = 128;          // rows per group of the wide bf16 kernels (NT = 128)
 
 constexpr int kDecMaxSplit = 8;            // K slices per tile at most
 constexpr int kDecMinSliceKb = 6;          // k blocks per slice at least
@@ -52,20 +52,25 @@ struct DecGroup { int32_t unit0, tile0, slot0; int16_t z, kb; };
 constexpr int kDecInvOff = 256 + ((kUmmaMaxGroups + 1) * (int)sizeof(DecGroup) + 15) / 16 * 16;   // per-warp token tables
 
 // kWBytes: weight tile(s) of one stage: 128 rows x 128 bytes per plane (64 bf16 or 128 E4M3 k values);
-// kXBytes: token tile(s) of one stage (W8: the hi and the lo plane).
-template <int MODE, bool W8> struct DecodeCfg;
-template <> struct DecodeCfg<4, false> { static constexpr int kWBytes = 2 * 128 * 128, kXBytes = kDecXBytes, kStages = 5; };
-template <> struct DecodeCfg<5, false> { static constexpr int kWBytes = 128 * 128, kXBytes = kDecXBytes, kStages = 8; };
-template <> struct DecodeCfg<4, true> { static constexpr int kWBytes = 2 * 128 * 128, kXBytes = 2 * kDecXBytes, kStages = 4; };
-template <> struct DecodeCfg<5, true> { static constexpr int kWBytes = 128 * 128, kXBytes = 2 * kDecXBytes, kStages = 6; };
+// kXBytes: token tile(s) of one stage, NT rows of 128 bytes (W8: the hi and the lo plane);
+// kStages: as many as 227 KB of shared memory hold, eight at most.
+template <int MODE, bool W8, int NT> struct DecodeCfg {
+  static constexpr int kWBytes = (MODE == 4 ? 2 : 1) * 128 * 128;
+  static constexpr int kXBytes = (W8 ? 2 : 1) * NT * 128;
+  static constexpr int kFit = (227 * 1024 - 1024 - kDecInvOff - 4 * NT * 4) / (kWBytes + kXBytes);
+  static constexpr int kStages = kFit > 8 ? 8 : kFit;   // 40 KB x 5, 24 x 8 (NT 64); 48 x 4, 32 x 6 (FP8, or NT 128)
+};
 
-template <int MODE, bool W8 = false>
+template <int MODE, bool W8 = false, int NT = kDecMaxRows>
 constexpr int decode_smem_bytes() {
-  using C = DecodeCfg<MODE, W8>;
-  return 1024 + C::kStages * (C::kWBytes + C::kXBytes) + kDecInvOff + 4 * 64 * 4;
+  using C = DecodeCfg<MODE, W8, NT>;
+  return 1024 + C::kStages * (C::kWBytes + C::kXBytes) + kDecInvOff + 4 * NT * 4;
 }
-// TMEM columns: two accumulator buffers of (weight planes x token planes) x 64 token columns
-template <int MODE, bool W8> struct DecodeTmem { static constexpr int kCols = (MODE == 4 && W8) ? 512 : 256; };
+// TMEM columns: two accumulator buffers of (weight planes x token planes) x NT token columns, 256 at least
+template <int MODE, bool W8, int NT> struct DecodeTmem {
+  static constexpr int kNeed = 2 * (MODE == 4 ? 2 : 1) * (W8 ? 2 : 1) * NT;
+  static constexpr int kCols = kNeed < 256 ? 256 : kNeed;
+};
 
 struct DecodeArgs {
   const GroupStatic* gs;
@@ -79,7 +84,7 @@ struct DecodeArgs {
   int32_t* err;
   float* part;           // [kDecMaxSlots][kDecSlotFloats] slice partials
   int32_t* ticket;       // [tiles][4 epilogue warps], zero between launches
-  int tok_box_rows;      // rows of the token-tile TMA box (16, 32 or 64): no more than the batch needs
+  int tok_box_rows;      // rows of the token-tile TMA box (16, 32, 64 or 128): no more than the batch needs
   int early_units;       // plain gate/up form: tiles of the shared expert (group 0) that need nothing from the router
   int n_rows_plain;      // rows of the batch (the shared expert's rows of a plain layer)
   // W8: per-row power-of-two scales of the token planes (x or H rows), then of the FP8 weight rows
@@ -99,7 +104,8 @@ __device__ __forceinline__ int snake_tile(int round, int cta, int n_ctas, int to
 
 // SPLIT = false is the plain form (one unit per tile, no scratch); the host picks SPLIT = true
 // only when even the largest possible set of active experts leaves tiles to split.
-template <int MODE, bool SPLIT, bool W8 = false>
+// NT: token columns per tile at most (64, or 128 for the wide bf16 form that takes batches of 65..128 rows).
+template <int MODE, bool SPLIT, bool W8 = false, int NT = kDecMaxRows>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_constant__ CUtensorMap tm_w_r,
                    const __grid_constant__ CUtensorMap tm_x_s, const __grid_constant__ CUtensorMap tm_x_r,
@@ -110,13 +116,15 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   constexpr bool kLazy = MODE == 4 && !SPLIT;
   if constexpr (!kLazy) grid_dep_wait();
   grid_dep_trigger();
-  using Cfg = DecodeCfg<MODE, W8>;
+  static_assert(NT == kDecMaxRows || (!SPLIT && !W8), "the wide form has no K split and no FP8 planes");
+  using Cfg = DecodeCfg<MODE, W8, NT>;
   constexpr int kStages = Cfg::kStages;
   constexpr int kWBytes = Cfg::kWBytes;
   constexpr int kStageBytes = kWBytes + Cfg::kXBytes;
   constexpr int kBK = W8 ? 2 * kUmmaBK : kUmmaBK;                // k per stage: 128 bytes of a weight row
-  constexpr int kBufCols = DecodeTmem<MODE, W8>::kCols / 2;     // accumulator columns per buffer
-  constexpr int kUpCol = W8 ? 128 : 64;                          // mode 4: first column of the up accumulators
+  constexpr int kTmemCols = DecodeTmem<MODE, W8, NT>::kCols;
+  constexpr int kBufCols = kTmemCols / 2;                        // accumulator columns per buffer
+  constexpr int kUpCol = (W8 ? 2 : 1) * NT;                      // mode 4: first column of the up accumulators
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -130,7 +138,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
   DecGroup* grp = reinterpret_cast<DecGroup*>(bars_gen + 256);       // SPLIT: [n_groups + 1]
   int32_t* tile_start = reinterpret_cast<int32_t*>(bars_gen + 256);  // !SPLIT: [n_groups + 1], same bytes
-  int32_t* inv_tables = reinterpret_cast<int32_t*>(bars_gen + kDecInvOff);     // [4 warps][64]
+  int32_t* inv_tables = reinterpret_cast<int32_t*>(bars_gen + kDecInvOff);     // [4 warps][NT]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -143,7 +151,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(tmem_slot), DecodeTmem<MODE, W8>::kCols);
+    tmem_alloc(smem_u32(tmem_slot), kTmemCols);
     tmem_relinquish();
   }
   if constexpr (kLazy) {
@@ -382,7 +390,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
       // Columns of the accumulator: mode 5 and shared groups, the group's own rows in order;
       // routed groups in mode 4, every row of the outer expert -> position in the group or -1.
       const bool lookup = MODE == 4 && !g.is_shared;
-      int32_t* inv = inv_tables + quad * 64;
+      int32_t* inv = inv_tables + quad * NT;
       int n_cols = r.count;
       // W8: per-token scale of accumulator column c = tok_scale[c]: mode 4, the x rows of the outer expert;
       // mode 5, the group's own H rows
@@ -393,7 +401,8 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         n_cols = rs.count;
         if constexpr (W8) tok_scale = p.tok_scale_r + rs.row0;
         __syncwarp();
-        inv[lane] = -1; inv[lane + 32] = -1;
+#pragma unroll
+        for (int c = 0; c < NT; c += 32) inv[c + lane] = -1;
         __syncwarp();
         for (int c = lane; c < r.count; c += 32) inv[__ldg(p.row_token + r.row0 + c) - rs.row0] = c;
         __syncwarp();
@@ -492,7 +501,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, DecodeTmem<MODE, W8>::kCols);
+    tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
@@ -503,10 +512,10 @@ struct DecodePlan {
   int32_t* ticket = nullptr;        // zeroed once; the kernels leave it zero
   CUtensorMap w_gu;                 // stacked gate/up rows, box 64 k x 128 rows x 2 planes
   CUtensorMap wd_s, wd_r;           // W_down blocks, 128-channel boxes
-  // token tiles come in boxes of 16, 32 or 64 rows (index 0..2): a launch uses the smallest that holds
+  // token tiles come in boxes of 16, 32, 64 or 128 rows (index 0..3): a launch uses the smallest that holds
   // its rows, so that a stage carries as little besides weights as possible
-  CUtensorMap x_rows[3];            // x (bound per forward for a plain layer)
-  CUtensorMap h_s[3], h_r[3];       // H
+  CUtensorMap x_rows[4];            // x (bound per forward for a plain layer)
+  CUtensorMap h_s[4], h_r[4];       // H
   // FP8 weights (set by decode_plan_attach_fp8): codes in the packed layouts, boxes of 128 k x 128 rows;
   // E4M3 planes [2][rows][cols] of the token rows (x, H_s, H_r) with their per-row scales
   bool fp8 = false;
@@ -537,7 +546,8 @@ inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
     ok = umma_encode(P, &D->wd_s, buf.w_down, 3, dims, str, box, "shared W_down (decode)") &&
          umma_encode_rows(P, &D->h_s[0], buf.h_s, s.max_outer_rows, s.shared_width, 16, "H shared (decode)") &&
          umma_encode_rows(P, &D->h_s[1], buf.h_s, s.max_outer_rows, s.shared_width, 32, "H shared (decode)") &&
-         umma_encode_rows(P, &D->h_s[2], buf.h_s, s.max_outer_rows, s.shared_width, 64, "H shared (decode)");
+         umma_encode_rows(P, &D->h_s[2], buf.h_s, s.max_outer_rows, s.shared_width, 64, "H shared (decode)") &&
+         umma_encode_rows(P, &D->h_s[3], buf.h_s, s.max_outer_rows, s.shared_width, 128, "H shared (decode)");
   }
   if (ok && P->has_r) {
     const cuuint64_t dims[4] = {(cuuint64_t)s.m, d, (cuuint64_t)s.n_r, (cuuint64_t)s.n_outer};
@@ -547,14 +557,16 @@ inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
                      "routed W_down (decode)") &&
          umma_encode_rows(P, &D->h_r[0], buf.h_r, s.max_routed_rows, s.m, 16, "H routed (decode)") &&
          umma_encode_rows(P, &D->h_r[1], buf.h_r, s.max_routed_rows, s.m, 32, "H routed (decode)") &&
-         umma_encode_rows(P, &D->h_r[2], buf.h_r, s.max_routed_rows, s.m, 64, "H routed (decode)");
+         umma_encode_rows(P, &D->h_r[2], buf.h_r, s.max_routed_rows, s.m, 64, "H routed (decode)") &&
+         umma_encode_rows(P, &D->h_r[3], buf.h_r, s.max_routed_rows, s.m, 128, "H routed (decode)");
   }
   if (ok && buf.x_fixed)
     ok = umma_encode_rows(P, &D->x_rows[0], buf.x_fixed, s.max_outer_rows, d, 16, "outer rows of x (decode)") &&
          umma_encode_rows(P, &D->x_rows[1], buf.x_fixed, s.max_outer_rows, d, 32, "outer rows of x (decode)") &&
-         umma_encode_rows(P, &D->x_rows[2], buf.x_fixed, s.max_outer_rows, d, 64, "outer rows of x (decode)");
+         umma_encode_rows(P, &D->x_rows[2], buf.x_fixed, s.max_outer_rows, d, 64, "outer rows of x (decode)") &&
+         umma_encode_rows(P, &D->x_rows[3], buf.x_fixed, s.max_outer_rows, d, 128, "outer rows of x (decode)");
   if (!ok) return false;
-  for (int i = 0; i < 3; ++i) {
+  for (int i = 0; i < 4; ++i) {
     if (!P->has_r) { D->wd_r = D->wd_s; D->h_r[i] = D->h_s[i]; }
     if (!P->has_s) { D->wd_s = D->wd_r; D->h_s[i] = D->h_r[i]; }
   }
@@ -569,6 +581,12 @@ inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(umma_decode_kernel<5, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              decode_smem_bytes<5>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(umma_decode_kernel<4, false, false, kDecWideRows>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             decode_smem_bytes<4, false, kDecWideRows>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(umma_decode_kernel<5, false, false, kDecWideRows>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             decode_smem_bytes<5, false, kDecWideRows>());
   if (e != cudaSuccess) {
     snprintf(P->error, sizeof(P->error), "cudaFuncSetAttribute (decode): %s", cudaGetErrorString(e));
     return false;
@@ -661,7 +679,7 @@ inline bool decode_plan_attach_fp8(UmmaPlan* P, DecodePlan* D, const DecodeFp8Bu
 }
 
 // Index of the smallest token box (16 << index rows) that holds n_rows rows.
-inline int decode_box_index(int n_rows) { return n_rows <= 16 ? 0 : (n_rows <= 32 ? 1 : 2); }
+inline int decode_box_index(int n_rows) { return n_rows <= 16 ? 0 : (n_rows <= 32 ? 1 : (n_rows <= 64 ? 2 : 3)); }
 
 inline bool decode_bind_x(UmmaPlan* P, DecodePlan* D, const void* x_rows, int n_rows) {
   D->x_ptr = x_rows;
@@ -679,7 +697,7 @@ inline int decode_split_x(UmmaPlan* P, DecodePlan* D, int n_rows, cudaStream_t s
 }
 
 // Both decode GEMMs; requires umma_bind_x and decode_bind_x for this forward and n_rows <=
-// kDecMaxRows outer rows.  The K-splitting form of a kernel is launched only when the device-side
+// kDecMaxRows outer rows (kDecWideRows with bf16 weights: the wide kernels, which never split K).  The K-splitting form of a kernel is launched only when the device-side
 // rule would split some group even if the largest possible set of experts were active for
 // n_rows rows (fewer active experts only split more).  Returns launches or -1.
 inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n_rows, int32_t* err_word,
@@ -695,8 +713,9 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n
     return D->part != nullptr && P->n_sms <= kDecMaxSlots && kb_max / per_cta >= 2;
   };
   const int kb_d = (s.d + bk - 1) / bk, kb_s = (s.shared_width + bk - 1) / bk, kb_m = (s.m + bk - 1) / bk;
-  const bool split1 = splits((act_s * ((s.shared_width + 127) / 128) + act_r * ((s.m + 127) / 128)) * kb_d, kb_d);
-  const bool split2 = splits((long long)((s.d + 127) / 128) * (act_s * kb_s + act_r * kb_m),
+  const bool wide = n_rows > kDecMaxRows;
+  const bool split1 = !wide && splits((act_s * ((s.shared_width + 127) / 128) + act_r * ((s.m + 127) / 128)) * kb_d, kb_d);
+  const bool split2 = !wide && splits((long long)((s.d + 127) / 128) * (act_s * kb_s + act_r * kb_m),
                              (act_s && kb_s > kb_m) || !act_r ? kb_s : kb_m);
   DecodeArgs a{};
   a.gs = P->buf.gs_dev; a.gr = gr; a.n_groups = P->n_groups; a.n_outer = s.n_outer; a.n_r = s.n_r;
@@ -711,7 +730,10 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
   int extra = 0;
   a.tok_scale_s = D->x_scale; a.tok_scale_r = D->x_scale;
-  if (D->fp8)       // the layer holds FP8 codes of its expert weights: stream those (half the bytes)
+  if (wide)
+    launch_kernel(dep, umma_decode_kernel<4, false, false, kDecWideRows>, dim3(P->n_sms), dim3(kUmmaThreads),
+                  decode_smem_bytes<4, false, kDecWideRows>(), st, D->w_gu, D->w_gu, D->x_rows[bi], D->x_rows[bi], a);
+  else if (D->fp8)  // the layer holds FP8 codes of its expert weights: stream those (half the bytes)
     launch_kernel(dep, split1 ? umma_decode_kernel<4, true, true> : umma_decode_kernel<4, false, true>, dim3(P->n_sms),
                   dim3(kUmmaThreads), decode_smem_bytes<4, true>(), st, D->w_gu8, D->w_gu8, D->xq_map[bi],
                   D->xq_map[bi], a);
@@ -721,6 +743,9 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n
   if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
   if (gate_up_only) {
+  } else if (wide) {
+    launch_kernel(dep, umma_decode_kernel<5, false, false, kDecWideRows>, dim3(P->n_sms), dim3(kUmmaThreads),
+                  decode_smem_bytes<5, false, kDecWideRows>(), st, D->wd_s, D->wd_r, D->h_s[bi], D->h_r[bi], a);
   } else if (D->fp8) {
     // E4M3 planes of H (shared rows, then routed rows), then the down GEMM on them
     const int rows_r = P->has_r ? n_rows * s.n_k : 0, rows_s = P->has_s ? n_rows : 0;

@@ -43,6 +43,19 @@ def test_plain_workloads_full_size(name):
     layer.destroy()
 
 
+@pytest.mark.parametrize("name,tokens", [("c2_llama2_7b", (100, 128)), ("c3_llama3_8b", (96,)), ("c5_skew_13b", (128,))])
+def test_wide_decode_full_width(name, tokens):
+    """65 to 128 rows at the full model width: the wide weights-on-M kernels (128 token columns per tile)."""
+    inputs = bench.prepare_inputs(name)
+    lay = inputs.layers[0]
+    layer = torch_io.layer_from_workload(inputs, 128)
+    for t in tokens:
+        st = parity.check_plain_layer(layer, lay, inputs.x[:t])
+        assert st["differing"] <= st["near_tie"]
+        assert sum(st["counts"]) == t * inputs.workload.shape.top_k
+    layer.destroy()
+
+
 def test_hierarchical_workload_full_size():
     inputs = bench.prepare_inputs("c4_hier_8x7b")
     w = inputs.workload

@@ -64,10 +64,10 @@ def test_small_shapes(name, d, m, tokens, path):
     layer.destroy()
 
 
-@pytest.mark.parametrize("tokens", [65, 128, 200, 256, 513, 1000])
+@pytest.mark.parametrize("tokens", [65, 100, 128, 129, 200, 256, 513, 1000])
 def test_mid_size_batches(tokens):
-    """65 to 1023 rows: split-K router over 64-row chunks (up to 512 rows), CTA-pair GEMMs from 256
-    rows, groups of a few dozen to a few hundred rows with ragged tiles."""
+    """65 to 1023 rows: split-K router over 64-row chunks (up to 512 rows), the wide weights-on-M kernels
+    up to 128 rows, CTA-pair GEMMs from 256 rows, groups of a few dozen to a few hundred rows with ragged tiles."""
     inp = _inputs("c2_llama2_7b", d_model=512, tokens=(1000,), m=1376)
     lay = inp.layers[0]
     rng = np.random.default_rng(3)
@@ -100,6 +100,8 @@ def test_hierarchical_small(path):
     assert st["differing"] <= st["near_tie"]
     st = parity.check_hier_layer(layer, inp, inp.x[:3])          # most outer experts empty
     st = parity.check_hier_layer(layer, inp, inp.x[:100])        # 200 outer rows: router chunks straddle outer experts
+    assert st["differing"] <= st["near_tie"]
+    st = parity.check_hier_layer(layer, inp, inp.x[:50])         # 100 outer rows: the wide weights-on-M kernels
     assert st["differing"] <= st["near_tie"]
     layer.destroy()
 
