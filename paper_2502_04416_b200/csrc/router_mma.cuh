@@ -188,9 +188,11 @@ namespace cmoe {
 // logic, then resets the ticket for the next call.  With at most kRskFuseGroups routed
 // groups the same block goes on to the histogram / scan / permutation of the selections
 // (and the groups' row ranges), which saves two launches per decode step.
-// Batches of up to kRskMaxChunks * 64 rows run the same kernel on a two-dimensional grid: block
-// (s, c) owns k slice s of the 64-row chunk c, and each chunk has its own scratch and ticket (the
-// permutation is then left to the permutation kernels).
+// Larger batches run the same kernel on a two-dimensional grid: block (s, c) owns k slice s of row chunk c
+// (chunk_rows = 16 for up to 64 rows, so that the chunks' reductions and gate logic run on different SMs;
+// 64 for up to kRskMaxChunks * 64 rows), and each chunk has its own scratch and ticket.  The chunks' last
+// blocks take a second ticket, and the block that takes the last of those permutes the whole batch (up to
+// kPermChunk rows; beyond that the permutation is left to the permutation kernels).
 constexpr int kRskMaxRows = 64;
 constexpr int kRskMaxChunks = 8;
 constexpr int kRskSliceK = 128;
@@ -205,7 +207,8 @@ __global__ void __launch_bounds__(kRskThreads)
 router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, int n_rp, int n_k,
                      const bf16* __restrict__ w_rep, const float* __restrict__ u, const float* __restrict__ b,
                      const int32_t* __restrict__ outer_off, int n_outer,
-                     float* __restrict__ part /*[slices][kRskMaxRows][64]*/, int32_t* __restrict__ ticket,
+                     float* __restrict__ part /*[chunks][slices][kRskMaxRows][64]*/,
+                     int32_t* __restrict__ ticket /*[kRskMaxChunks + 1], zero between launches*/, int chunk_rows,
                      float* __restrict__ scores, float* __restrict__ keys,
                      int32_t* topk_idx, float* __restrict__ topk_gate,
                      int fuse_permute, int n_groups, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
@@ -213,9 +216,12 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
   grid_dep_wait();
   grid_dep_trigger();
   static_assert(kRskThreads == kPermChunk, "the fused permutation is written for one 256-row chunk");
-  // this block's 64-row chunk: from here on rows are counted within the chunk
-  const int row_base = blockIdx.y * kRskMaxRows;
-  n_rows = min(kRskMaxRows, n_rows - row_base);
+  // this block's chunk of rows: from here on rows are counted within the chunk
+  const int n_rows_all = n_rows;
+  const int32_t* topk_idx_all = topk_idx;
+  int32_t* ticket_chunks = ticket + kRskMaxChunks;
+  const int row_base = blockIdx.y * chunk_rows;
+  n_rows = min(chunk_rows, n_rows - row_base);
   xo += (size_t)row_base * d;
   scores += (size_t)row_base * n_r; keys += (size_t)row_base * n_r;
   topk_idx += (size_t)row_base * n_k; topk_gate += (size_t)row_base * n_k;
@@ -331,7 +337,18 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
   }
   if (threadIdx.x == 0) *ticket = 0;
   if (!fuse_permute) return;
-  // ---- histogram / scan / stable permutation of the selections just written (one chunk)
+  if (gridDim.y > 1) {                             // the last chunk to finish permutes the batch
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = (atomicAdd(ticket_chunks, 1) == (int)gridDim.y - 1);
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    if (threadIdx.x == 0) *ticket_chunks = 0;
+    n_rows = n_rows_all;
+    topk_idx = const_cast<int32_t*>(topk_idx_all);
+  }
+  // ---- histogram / scan / stable permutation of the selections just written (at most kPermChunk rows)
   __syncthreads();
   int32_t* sm = reinterpret_cast<int32_t*>(&unit[0][0][0]);     // the partial sums are no longer needed
   int32_t* hist = sm;                              // [n_groups]

@@ -116,7 +116,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   constexpr bool kLazy = MODE == 4 && !SPLIT;
   if constexpr (!kLazy) grid_dep_wait();
   grid_dep_trigger();
-  static_assert(NT == kDecMaxRows || (!SPLIT && !W8), "the wide form has no K split and no FP8 planes");
+  static_assert(NT <= kDecMaxRows || (!SPLIT && !W8), "the wide form has no K split and no FP8 planes");
   using Cfg = DecodeCfg<MODE, W8, NT>;
   constexpr int kStages = Cfg::kStages;
   constexpr int kWBytes = Cfg::kWBytes;
@@ -402,7 +402,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         if constexpr (W8) tok_scale = p.tok_scale_r + rs.row0;
         __syncwarp();
 #pragma unroll
-        for (int c = 0; c < NT; c += 32) inv[c + lane] = -1;
+        for (int c = 0; c < NT; c += 32) if (c + lane < NT) inv[c + lane] = -1;
         __syncwarp();
         for (int c = lane; c < r.count; c += 32) inv[__ldg(p.row_token + r.row0 + c) - rs.row0] = c;
         __syncwarp();
@@ -506,6 +506,34 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
 }
 
 // ----------------------------------------------------------------------------- host
+// Both modes of one (weights, NT) family: dynamic shared memory above 48 KB has to be allowed per kernel.
+template <bool W8, int NT>
+inline void decode_allow_smem(cudaError_t* e) {
+  auto allow = [&](auto kernel, int bytes) {
+    if (*e == cudaSuccess) *e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  };
+  allow(umma_decode_kernel<4, false, W8, NT>, decode_smem_bytes<4, W8, NT>());
+  allow(umma_decode_kernel<5, false, W8, NT>, decode_smem_bytes<5, W8, NT>());
+  if constexpr (NT <= kDecMaxRows) {
+    allow(umma_decode_kernel<4, true, W8, NT>, decode_smem_bytes<4, W8, NT>());
+    allow(umma_decode_kernel<5, true, W8, NT>, decode_smem_bytes<5, W8, NT>());
+  }
+}
+
+// One decode GEMM: the instantiation for (mode, weights, NT), K-splitting or plain.
+template <int MODE, bool W8, int NT>
+inline void decode_launch(bool dep, bool split, int n_sms, cudaStream_t st, const CUtensorMap& w_s, const CUtensorMap& w_r,
+                          const CUtensorMap& x_s, const CUtensorMap& x_r, const DecodeArgs& a) {
+  constexpr int smem = decode_smem_bytes<MODE, W8, NT>();
+  if constexpr (NT <= kDecMaxRows) {
+    if (split) {
+      launch_kernel(dep, umma_decode_kernel<MODE, true, W8, NT>, dim3(n_sms), dim3(kUmmaThreads), smem, st, w_s, w_r, x_s, x_r, a);
+      return;
+    }
+  }
+  launch_kernel(dep, umma_decode_kernel<MODE, false, W8, NT>, dim3(n_sms), dim3(kUmmaThreads), smem, st, w_s, w_r, x_s, x_r, a);
+}
+
 struct DecodePlan {
   bool built = false;
   float* part = nullptr;            // kDecMaxSlots slots of slice partials (caller-owned workspace)
@@ -570,23 +598,9 @@ inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
     if (!P->has_r) { D->wd_r = D->wd_s; D->h_r[i] = D->h_s[i]; }
     if (!P->has_s) { D->wd_s = D->wd_r; D->h_s[i] = D->h_r[i]; }
   }
-  cudaError_t e = cudaFuncSetAttribute(umma_decode_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       decode_smem_bytes<4>());
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(umma_decode_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             decode_smem_bytes<4>());
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(umma_decode_kernel<5, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             decode_smem_bytes<5>());
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(umma_decode_kernel<5, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             decode_smem_bytes<5>());
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(umma_decode_kernel<4, false, false, kDecWideRows>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             decode_smem_bytes<4, false, kDecWideRows>());
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(umma_decode_kernel<5, false, false, kDecWideRows>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             decode_smem_bytes<5, false, kDecWideRows>());
+  cudaError_t e = cudaSuccess;
+  decode_allow_smem<false, kDecMaxRows>(&e);
+  decode_allow_smem<false, kDecWideRows>(&e);
   if (e != cudaSuccess) {
     snprintf(P->error, sizeof(P->error), "cudaFuncSetAttribute (decode): %s", cudaGetErrorString(e));
     return false;
@@ -659,13 +673,7 @@ inline bool decode_plan_attach_fp8(UmmaPlan* P, DecodePlan* D, const DecodeFp8Bu
     if (!P->has_s) { D->wd8_s = D->wd8_r; D->hqs_map[i] = D->hqr_map[i]; }
   }
   cudaError_t e = cudaSuccess;
-  auto attr = [&](auto kernel, int bytes) {
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  };
-  attr(umma_decode_kernel<4, false, true>, decode_smem_bytes<4, true>());
-  attr(umma_decode_kernel<4, true, true>, decode_smem_bytes<4, true>());
-  attr(umma_decode_kernel<5, false, true>, decode_smem_bytes<5, true>());
-  attr(umma_decode_kernel<5, true, true>, decode_smem_bytes<5, true>());
+  decode_allow_smem<true, kDecMaxRows>(&e);
   if (e != cudaSuccess) {
     snprintf(P->error, sizeof(P->error), "cudaFuncSetAttribute (FP8 decode): %s", cudaGetErrorString(e));
     return false;
@@ -730,22 +738,16 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
   int extra = 0;
   a.tok_scale_s = D->x_scale; a.tok_scale_r = D->x_scale;
-  if (wide)
-    launch_kernel(dep, umma_decode_kernel<4, false, false, kDecWideRows>, dim3(P->n_sms), dim3(kUmmaThreads),
-                  decode_smem_bytes<4, false, kDecWideRows>(), st, D->w_gu, D->w_gu, D->x_rows[bi], D->x_rows[bi], a);
-  else if (D->fp8)  // the layer holds FP8 codes of its expert weights: stream those (half the bytes)
-    launch_kernel(dep, split1 ? umma_decode_kernel<4, true, true> : umma_decode_kernel<4, false, true>, dim3(P->n_sms),
-                  dim3(kUmmaThreads), decode_smem_bytes<4, true>(), st, D->w_gu8, D->w_gu8, D->xq_map[bi],
-                  D->xq_map[bi], a);
-  else
-    launch_kernel(dep, split1 ? umma_decode_kernel<4, true> : umma_decode_kernel<4, false>, dim3(P->n_sms),
-                  dim3(kUmmaThreads), decode_smem_bytes<4>(), st, D->w_gu, D->w_gu, D->x_rows[bi], D->x_rows[bi], a);
+  const int sms = P->n_sms;
+  if (wide) decode_launch<4, false, kDecWideRows>(dep, false, sms, st, D->w_gu, D->w_gu, D->x_rows[bi], D->x_rows[bi], a);
+  else if (D->fp8)          // the layer holds FP8 codes of its expert weights: stream those (half the bytes)
+    decode_launch<4, true, kDecMaxRows>(dep, split1, sms, st, D->w_gu8, D->w_gu8, D->xq_map[bi], D->xq_map[bi], a);
+  else decode_launch<4, false, kDecMaxRows>(dep, split1, sms, st, D->w_gu, D->w_gu, D->x_rows[bi], D->x_rows[bi], a);
   if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
   if (gate_up_only) {
   } else if (wide) {
-    launch_kernel(dep, umma_decode_kernel<5, false, false, kDecWideRows>, dim3(P->n_sms), dim3(kUmmaThreads),
-                  decode_smem_bytes<5, false, kDecWideRows>(), st, D->wd_s, D->wd_r, D->h_s[bi], D->h_r[bi], a);
+    decode_launch<5, false, kDecWideRows>(dep, false, sms, st, D->wd_s, D->wd_r, D->h_s[bi], D->h_r[bi], a);
   } else if (D->fp8) {
     // E4M3 planes of H (shared rows, then routed rows), then the down GEMM on them
     const int rows_r = P->has_r ? n_rows * s.n_k : 0, rows_s = P->has_s ? n_rows : 0;
@@ -755,11 +757,10 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n
     launch_kernel(dep, split_rows_e4m3_kernel, dim3(rows_s + rows_r), dim3(128), 0, st, hs, hr);
     extra = 1;
     a.tok_scale_s = D->hs_scale; a.tok_scale_r = D->hr_scale;
-    launch_kernel(dep, split2 ? umma_decode_kernel<5, true, true> : umma_decode_kernel<5, false, true>, dim3(P->n_sms),
-                  dim3(kUmmaThreads), decode_smem_bytes<5, true>(), st, D->wd8_s, D->wd8_r, D->hqs_map[bi], D->hqr_map[bi], a);
-  } else
-    launch_kernel(dep, split2 ? umma_decode_kernel<5, true> : umma_decode_kernel<5, false>, dim3(P->n_sms),
-                  dim3(kUmmaThreads), decode_smem_bytes<5>(), st, D->wd_s, D->wd_r, D->h_s[bi], D->h_r[bi], a);
+    decode_launch<5, true, kDecMaxRows>(dep, split2, sms, st, D->wd8_s, D->wd8_r, D->hqs_map[bi], D->hqr_map[bi], a);
+  } else {
+    decode_launch<5, false, kDecMaxRows>(dep, split2, sms, st, D->wd_s, D->wd_r, D->h_s[bi], D->h_r[bi], a);
+  }
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
     snprintf(P->error, sizeof(P->error), "decode GEMM launch: %s", cudaGetErrorString(e));

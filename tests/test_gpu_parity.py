@@ -40,7 +40,7 @@ def test_c1_tiny_fp32(path):
 
 SMALL = [
     ("c2_llama2_7b", 256, None, (1, 16, 77, 300)),
-    ("c3_llama3_8b", 256, None, (33, 517)),
+    ("c3_llama3_8b", 256, None, (33, 50, 64, 517)),   # 17..64 rows, more than 8 router columns: 16-row router chunks
     ("c5_skew_13b", 320, None, (129, 700)),
     ("c2_llama2_7b", 512, 200, (1000,)),       # m = 200: neither a multiple of 16 nor of 64
     ("c2_llama2_7b", 1024, 768, (1, 7, 64)),   # decode GEMMs with K split 2-4 ways per tile
