@@ -25,6 +25,7 @@
 #include "simt_gemm.cuh"
 #include "umma2_gemm.cuh"
 #include "umma_decode.cuh"
+#include "gemv.cuh"
 #include "umma_gemm.cuh"
 
 using namespace cmoe;
@@ -382,10 +383,18 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
   // Weights-on-M streaming kernels: up to 64 rows; on bf16 weights (the FP8 token planes stop at 64) the wide
   // form takes up to 128 rows, or up to 96 when 128-neuron tiles pad the expert width by more than 5 %
   // (measured: a 448-wide expert's token-major 112-neuron tiles win from there).  Path 2 keeps token-major tiles.
+  // One row of a plain layer: plain-load weight streamers on the CUDA cores, the down projection and the
+  // combine in one launch (automatic path only; path 2 keeps the tensor-core kernels).
+  bool gemv = false;
+  GemvPlan gemv_ring{};
+  if constexpr (std::is_same<T, bf16>::value)
+    gemv = use_umma && !L->hier && L->gemm_path == 0 &&
+           gemv_plan((int)R, L->n_outer, L->n_groups_total(), n_k, n_r, d, L->shared_width(), L->m, L->cfg.n_shared > 0,
+                     L->fp8, &gemv_ring);
   int decode_rows = kDecMaxRows;
   if (!L->fp8 && L->gemm_path != 2)
     decode_rows = ((L->m + 127) / 128 * 128) * 100LL <= 105LL * L->m ? kDecWideRows : 96;
-  const bool decode = use_umma && R <= decode_rows;
+  const bool decode = use_umma && !gemv && R <= decode_rows;
   if (use_umma && !umma_bind_x(&L->umma, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   if (decode && !decode_bind_x(&L->umma, &L->decode, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   if (decode && L->fp8) {                          // E4M3 planes of the token rows: independent of the routing
@@ -415,7 +424,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
         const int chunk_rows = (R <= kRskMaxRows && n_r > 8) ? 16 : kRskMaxRows;
         const int chunks = (R + chunk_rows - 1) / chunk_rows;
         perm_fused = G <= kRskFuseGroups && R <= 2 * kRskMaxRows && (long long)R * n_k <= 4096;
-        const bool sub8 = n_r <= 8 && chunk_rows > 16;               // pays when a chunk's last block has more than 16 rows
+        const bool sub8 = n_r <= 8 && R > 16;                        // pays when a chunk's last block has more than 16 rows
         (sub8 ? router_splitk_kernel<true> : router_splitk_kernel<false>)
             <<<dim3((d + kRskSliceK - 1) / kRskSliceK, chunks), kRskThreads, 0, st>>>(
             xo, R, d, n_r, L->n_rp, n_k, (const bf16*)L->w_rep, L->u, L->b, ooff, L->n_outer, L->rsk_part,
@@ -477,7 +486,31 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
   }
 
   mark(2);
-  if (use_umma) {
+  if (gemv) {
+    if constexpr (std::is_same<T, bf16>::value) {
+      GemvArgs a{};
+      a.gs = L->umma.buf.gs_dev; a.gr = L->gr; a.n_groups = L->n_groups_total(); a.d = d; a.n_rows = (int)R; a.n_k = n_k;
+      a.x = xo;
+      a.w_gate_up = L->fp8 ? (const void*)L->w_gu8 : (const void*)L->w_gu;
+      a.w_down = L->fp8 ? (const void*)L->wd8 : (const void*)L->wd_p;
+      a.rows_w = (long long)L->n_outer * L->cfg.d_ff;
+      a.scale_gu = L->scale_gu; a.scale_d = L->scale_d;
+      a.h_s = (bf16*)L->h_s; a.h_r = (bf16*)L->h_r; a.ld_h_s = L->shared_width(); a.ld_h_r = L->m;
+      a.row_of = L->row_of; a.topk_gate = L->topk_gate;
+      a.out = out;
+      const int n = gemv_forward(a, gemv_ring, L->fp8, L->umma.n_sms, st, ev ? ev[3] : nullptr, dep, gate_up_only);
+      if (n < 0) return arg_fail(CMOE_ERR_CUDA, "gemv launch failed");
+      launches += n;
+    }
+    if (!gate_up_only) {                              // the second launch wrote `out`: nothing left to combine
+      mark(4);
+      mark(5);
+      if (ev) ++L->ev_count;
+      CU_TRY(cudaGetLastError());
+      L->launches = launches;
+      return CMOE_OK;
+    }
+  } else if (use_umma) {
     cudaEvent_t mid = ev ? ev[3] : nullptr;
     int n;
     if (decode) {

@@ -46,7 +46,7 @@ def test_quantise_rows_bit_exact():
 
 
 SHAPES = [
-    ("c2_llama2_7b", 256, None, (1, 16, 64, 300)),       # decode sizes stream FP8, 300 rows read the bf16 copies
+    ("c2_llama2_7b", 256, None, (1, 2, 16, 64, 300)),    # decode sizes stream FP8, 300 rows read the bf16 copies
     ("c3_llama3_8b", 256, None, (32, 5)),
     ("c2_llama2_7b", 1024, 768, (1, 7, 64)),             # K split 2-4 ways per tile
     ("c5_skew_13b", 320, None, (40,)),
@@ -118,7 +118,7 @@ def test_quantise_refusals():
     layer.destroy()
 
 
-@pytest.mark.parametrize("name,tokens", [("c2_llama2_7b", (1, 16, 64)), ("c3_llama3_8b", (32,))])
+@pytest.mark.parametrize("name,tokens", [("c2_llama2_7b", (1, 2, 16, 64)), ("c3_llama3_8b", (2, 32))])
 def test_quantised_decode_full_size(name, tokens):
     inputs = bench.prepare_inputs(name)
     lay = inputs.layers[0]

@@ -39,7 +39,7 @@ def test_c1_tiny_fp32(path):
 
 
 SMALL = [
-    ("c2_llama2_7b", 256, None, (1, 16, 77, 300)),
+    ("c2_llama2_7b", 256, None, (1, 2, 16, 77, 300)),   # 1 and 2 rows: the plain-load streamers
     ("c3_llama3_8b", 256, None, (33, 50, 64, 517)),   # 17..64 rows, more than 8 router columns: 16-row router chunks
     ("c5_skew_13b", 320, None, (129, 700)),
     ("c2_llama2_7b", 512, 200, (1000,)),       # m = 200: neither a multiple of 16 nor of 64
