@@ -151,26 +151,19 @@ __device__ __forceinline__ void gemv_list_groups(const GemvArgs& p, GemvGroups<T
   __syncthreads();
 }
 
+constexpr int kGemvEarly = 3;              // shared-expert neurons a warp may finish before the router has
+
 template <int TT, bool FP8>
 __global__ void __launch_bounds__(kGemvThreads, 2)
 gemv_gate_up_kernel(const GemvArgs p) {
   __shared__ GemvGroups<TT> L;
-  grid_dep_wait();
   grid_dep_trigger();
-  gemv_list_groups(p, L);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_warps = gridDim.x * kGemvWarps, gw = blockIdx.x * kGemvWarps + warp;
   const int chunks = p.d >> 3;                         // 8 weights per chunk
   constexpr int esz = FP8 ? 1 : 2;
-  for (int item = gw; item < L.total; item += n_warps) {
-    int lo = 0, hi = L.n;
-    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (L.start[mid] <= item) lo = mid; else hi = mid; }
-    const int n = item - L.start[lo];
-    const int count = L.count[lo] < TT ? L.count[lo] : TT;
-    const bf16* xr[TT];
-#pragma unroll
-    for (int j = 0; j < TT; ++j) xr[j] = p.x + (size_t)L.tok[lo][j < count ? j : 0] * p.d;
-    const size_t wrow = (size_t)(L.w_row0[lo] + n);
+  // gate and up pre-activations of one neuron (packed weight row wrow) for the token rows xr[0 .. TT)
+  auto neuron = [&](size_t wrow, const bf16* const (&xr)[TT], float (&g)[TT], float (&u)[TT]) {
     const char* wg = (const char*)p.w_gate_up + wrow * p.d * esz;
     const char* wu = wg + (size_t)p.rows_w * p.d * esz;
     float ag[TT], au[TT];
@@ -195,12 +188,60 @@ gemv_gate_up_kernel(const GemvArgs p) {
     float sg = 1.0f, su = 1.0f;
     if constexpr (FP8) { sg = __ldg(p.scale_gu + wrow); su = __ldg(p.scale_gu + p.rows_w + wrow); }
 #pragma unroll
-    for (int j = 0; j < TT; ++j) {
-      const float a = warp_sum(ag[j]) * sg, u = warp_sum(au[j]) * su;
-      if (lane == 0 && j < count) {
-        bf16* dst = L.is_shared[lo] ? p.h_s + (size_t)(L.row0[lo] + j) * p.ld_h_s : p.h_r + (size_t)(L.row0[lo] + j) * p.ld_h_r;
-        dst[n] = __float2bfloat16_rn(a / (1.0f + __expf(-a)) * u);
-      }
+    for (int j = 0; j < TT; ++j) { g[j] = warp_sum(ag[j]) * sg; u[j] = warp_sum(au[j]) * su; }
+  };
+  // Head start: group 0 of a plain layer with a shared expert is that expert, its rows are all the
+  // tokens, and neither its weights nor x depend on the router.  Each warp finishes up to kGemvEarly of
+  // its neurons while the router (the preceding kernel) runs, keeps the results in registers, and
+  // stores them after the wait, when the previous reader of H has certainly finished.
+  const GroupStatic g0 = p.gs[0];
+  const int early_width = (g0.is_shared && p.n_rows <= TT) ? g0.width : 0;
+  float early_h[kGemvEarly][TT];
+#pragma unroll
+  for (int i = 0; i < kGemvEarly; ++i) {
+    const int n = gw + i * n_warps;
+    if (n < early_width) {
+      const bf16* xr[TT];
+#pragma unroll
+      for (int j = 0; j < TT; ++j) xr[j] = p.x + (size_t)(j < p.n_rows ? j : 0) * p.d;
+      float g[TT], u[TT];
+      neuron((size_t)(g0.w_row0 + n), xr, g, u);
+#pragma unroll
+      for (int j = 0; j < TT; ++j) early_h[i][j] = g[j] / (1.0f + __expf(-g[j])) * u[j];
+    }
+  }
+  grid_dep_wait();
+#pragma unroll
+  for (int i = 0; i < kGemvEarly; ++i) {
+    const int n = gw + i * n_warps;
+    if (n < early_width && lane == 0) {
+#pragma unroll
+      for (int j = 0; j < TT; ++j)
+        if (j < p.n_rows) p.h_s[(size_t)j * p.ld_h_s + n] = __float2bfloat16_rn(early_h[i][j]);
+    }
+  }
+  gemv_list_groups(p, L);
+  // the active groups' neurons, concatenated; group 0 comes first, so an item below early_width of the first
+  // kGemvEarly rounds is one of those finished above
+  int round = 0;
+  for (int item = gw; item < L.total; item += n_warps, ++round) {
+    if (round < kGemvEarly && item < early_width) continue;
+    int lo = 0, hi = L.n;
+    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (L.start[mid] <= item) lo = mid; else hi = mid; }
+    const int n = item - L.start[lo];
+    const int count = L.count[lo] < TT ? L.count[lo] : TT;
+    const bf16* xr[TT];
+#pragma unroll
+    for (int j = 0; j < TT; ++j) xr[j] = p.x + (size_t)L.tok[lo][j < count ? j : 0] * p.d;
+    float g[TT], u[TT];
+    neuron((size_t)(L.w_row0[lo] + n), xr, g, u);
+    if (lane == 0) {
+#pragma unroll
+      for (int j = 0; j < TT; ++j)
+        if (j < count) {
+          bf16* dst = L.is_shared[lo] ? p.h_s + (size_t)(L.row0[lo] + j) * p.ld_h_s : p.h_r + (size_t)(L.row0[lo] + j) * p.ld_h_r;
+          dst[n] = __float2bfloat16_rn(g[j] / (1.0f + __expf(-g[j])) * u[j]);
+        }
     }
   }
 }
