@@ -393,7 +393,7 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
                      L->fp8, &gemv_ring);
   int decode_rows = kDecMaxRows;
   if (!L->fp8 && L->gemm_path != 2)
-    decode_rows = ((L->m + 127) / 128 * 128) * 100LL <= 105LL * L->m ? kDecWideRows : 96;
+    decode_rows = kDecWideRows;
   const bool decode = use_umma && !gemv && R <= decode_rows;
   if (use_umma && !umma_bind_x(&L->umma, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   if (decode && !decode_bind_x(&L->umma, &L->decode, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);

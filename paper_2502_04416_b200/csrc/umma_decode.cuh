@@ -85,6 +85,8 @@ struct DecodeArgs {
   float* part;           // [kDecMaxSlots][kDecSlotFloats] slice partials
   int32_t* ticket;       // [tiles][4 epilogue warps], zero between launches
   int tok_box_rows;      // rows of the token-tile TMA box (16, 32, 64 or 128): no more than the batch needs
+  int tile_rows_s, tile_rows_r;   // mode 4: neurons per tile of a shared / routed group (128, or less when 128 would pad
+                         // the group's width by more than 5 %: the rows past them in the 128-row MMA are dead)
   int early_units;       // plain gate/up form: tiles of the shared expert (group 0) that need nothing from the router
   int n_rows_plain;      // rows of the batch (the shared expert's rows of a plain layer)
   // W8: per-row power-of-two scales of the token planes (x or H rows), then of the FP8 weight rows
@@ -141,6 +143,13 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   int32_t* inv_tables = reinterpret_cast<int32_t*>(bars_gen + kDecInvOff);     // [4 warps][NT]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // rows of a tile of group g and the number of its tiles
+  auto tile_rows = [&](const GroupStatic& g) { return MODE == 4 ? (g.is_shared ? p.tile_rows_s : p.tile_rows_r) : 128; };
+  auto group_tiles = [&](int g) {
+    const GroupStatic gg = p.gs[g];
+    const int span = MODE == 4 ? gg.width : (gg.width > 0 ? p.d : 0), tr = tile_rows(gg);
+    return p.gr[g].count > 0 ? (span + tr - 1) / tr : 0;
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
@@ -157,10 +166,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   if constexpr (kLazy) {
     // the table is built by the producer warp when a role first needs it (build_table below)
   } else if constexpr (!SPLIT) {
-    for (int g = threadIdx.x; g < p.n_groups; g += blockDim.x) {
-      const int span = MODE == 4 ? p.gs[g].width : (p.gs[g].width > 0 ? p.d : 0);
-      tile_start[g + 1] = p.gr[g].count > 0 ? (span + 127) / 128 : 0;
-    }
+    for (int g = threadIdx.x; g < p.n_groups; g += blockDim.x) tile_start[g + 1] = group_tiles(g);
     __syncthreads();
     if (threadIdx.x == 0) {
       int run = 0;
@@ -170,8 +176,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   } else {
     // per group: tile count (in .tile0 for now) and k blocks per tile
     for (int g = threadIdx.x; g < p.n_groups; g += blockDim.x) {
-      const int span = MODE == 4 ? p.gs[g].width : (p.gs[g].width > 0 ? p.d : 0);
-      grp[g].tile0 = p.gr[g].count > 0 ? (span + 127) / 128 : 0;
+      grp[g].tile0 = group_tiles(g);
       grp[g].kb = (int16_t)(((MODE == 4 ? p.d : p.gs[g].width) + kBK - 1) / kBK);
     }
     __syncthreads();
@@ -223,8 +228,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
   // producer warp: wait for the router, count every group's tiles, publish the table
   auto build_table = [&]() {
     grid_dep_wait();
-    for (int g = lane; g < p.n_groups; g += 32)
-      tile_start[g + 1] = p.gr[g].count > 0 ? (p.gs[g].width + 127) / 128 : 0;
+    for (int g = lane; g < p.n_groups; g += 32) tile_start[g + 1] = group_tiles(g);
     __syncwarp();
     if (lane == 0) {
       int run = 0;
@@ -305,8 +309,9 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         const uint32_t fb = full0 + 8 * s;
         const uint32_t sw = base + s * kStageBytes, sx = sw + kWBytes;
         if (lane == 0) {
-          mbar_expect_tx(fb, kWBytes + (W8 ? 2 : 1) * p.tok_box_rows * 128);
-          if (MODE == 4) tma_load_3d(sw, tw, fb, kb * kBK, g.w_row0 + nt * 128, 0);
+          const int tr = tile_rows(g);
+          mbar_expect_tx(fb, (MODE == 4 ? 2 : 1) * tr * 128 + (W8 ? 2 : 1) * p.tok_box_rows * 128);
+          if (MODE == 4) tma_load_3d(sw, tw, fb, kb * kBK, g.w_row0 + nt * tr, 0);   // gate rows, then the up rows behind them
           else if (g.is_shared) tma_load_3d(sw, tw, fb, kb * kBK, nt * 128, g.outer);
           else tma_load_4d(sw, tw, fb, kb * kBK, nt * 128, j, g.outer);
           if constexpr (W8) {                   // token planes [k, row, plane]: the hi rows, directly behind them the lo rows
@@ -341,6 +346,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         if (!mbar_wait(acce0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.err, kErrWaitAccEmpty)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * kBufCols;
+        const uint32_t up_off = (uint32_t)tile_rows(g) * 128u;          // the up plane follows the tile's gate rows
         const int k_end = SPLIT ? un.kb1 : ((MODE == 4 ? p.d : g.width) + kBK - 1) / kBK;
         for (int kb = un.kb0; kb < k_end; ++kb, ++it) {
           const uint32_t s = it % kStages, n = it / kStages;
@@ -351,7 +357,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             const uint32_t acc = (kb != un.kb0 || k != 0) ? 1u : 0u;
-            const uint64_t a_g = umma_smem_desc(sw + k * 32), a_u = umma_smem_desc(sw + 128 * 128 + k * 32);
+            const uint64_t a_g = umma_smem_desc(sw + k * 32), a_u = umma_smem_desc(sw + up_off + k * 32);
             const uint64_t b_hi = umma_smem_desc(sx + k * 32);
             if constexpr (W8) {
               umma_e4m3(d_tmem, a_g, b_hi, idesc, acc);
@@ -382,7 +388,8 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
       const uint32_t buf = round & 1, use = round >> 1;
       if (!mbar_wait(accf0 + 8 * buf, use & 1, abort_flag, p.err, kErrWaitAccFull)) { ok = false; break; }
       tc_fence_after();
-      const int wr = nt * 128 + quad * 32 + lane;                 // neuron (mode 4) / channel (mode 5)
+      const int tr = tile_rows(g);
+      const int wr = nt * tr + quad * 32 + lane;                  // neuron (mode 4) / channel (mode 5)
       const int span = MODE == 4 ? g.width : p.d;
       const int ld = MODE == 4 ? (g.is_shared ? p.ld_out_s : p.ld_out_r) : p.d;
       bf16* dst = (g.is_shared ? p.out_s : p.out_r) + (size_t)r.row0 * ld + wr;
@@ -407,7 +414,7 @@ umma_decode_kernel(const __grid_constant__ CUtensorMap tm_w_s, const __grid_cons
         for (int c = lane; c < r.count; c += 32) inv[__ldg(p.row_token + r.row0 + c) - rs.row0] = c;
         __syncwarp();
       }
-      const bool row_live = wr < span;
+      const bool row_live = quad * 32 + lane < tr && wr < span;
       float sc_a = 1.0f, sc_b = 1.0f;                    // W8: power-of-two scales of this thread's weight row(s)
       if constexpr (W8) {
         if (row_live) {
@@ -538,7 +545,8 @@ struct DecodePlan {
   bool built = false;
   float* part = nullptr;            // kDecMaxSlots slots of slice partials (caller-owned workspace)
   int32_t* ticket = nullptr;        // zeroed once; the kernels leave it zero
-  CUtensorMap w_gu;                 // stacked gate/up rows, box 64 k x 128 rows x 2 planes
+  CUtensorMap w_gu, w_gu_r;         // stacked gate/up rows, box 64 k x tile rows (shared, routed groups) x 2 planes
+  int tile_rows_s = 128, tile_rows_r = 128;
   CUtensorMap wd_s, wd_r;           // W_down blocks, 128-channel boxes
   // token tiles come in boxes of 16, 32, 64 or 128 rows (index 0..3): a launch uses the smallest that holds
   // its rows, so that a stage carries as little besides weights as possible
@@ -547,7 +555,7 @@ struct DecodePlan {
   // FP8 weights (set by decode_plan_attach_fp8): codes in the packed layouts, boxes of 128 k x 128 rows;
   // E4M3 planes [2][rows][cols] of the token rows (x, H_s, H_r) with their per-row scales
   bool fp8 = false;
-  CUtensorMap w_gu8, wd8_s, wd8_r;
+  CUtensorMap w_gu8, w_gu8_r, wd8_s, wd8_r;
   const float *scale_gu = nullptr, *scale_d = nullptr;
   uint8_t *xq = nullptr, *hq_s = nullptr, *hq_r = nullptr;
   float *x_scale = nullptr, *hs_scale = nullptr, *hr_scale = nullptr;
@@ -556,16 +564,30 @@ struct DecodePlan {
   const void* x_ptr = nullptr;                   // x of this forward (decode_bind_x)
 };
 
+// Neurons per gate/up tile of a group of this width: 128 when that pads the width by at most 5 %, else the multiple
+// of 16 in [96, 128) with the least padding (448 -> 112: four exact tiles instead of 14 % of wasted weight rows).
+inline int decode_pick_tile_rows(int width) {
+  if (width <= 0 || (long long)((width + 127) / 128 * 128) * 100 <= (long long)width * 105) return 128;
+  int best = 128, best_pad = (width + 127) / 128 * 128;
+  for (int tr = 112; tr >= 96; tr -= 16) {
+    const int pad = (width + tr - 1) / tr * tr;
+    if (pad < best_pad) { best = tr; best_pad = pad; }
+  }
+  return best;
+}
+
 inline bool decode_plan_create(UmmaPlan* P, DecodePlan* D) {
   const UmmaShape& s = P->shape;
   const UmmaBuffers& buf = P->buf;
   const size_t d = s.d, rows_w = (size_t)s.n_outer * s.d_ff;
   bool ok = true;
-  {
+  D->tile_rows_s = decode_pick_tile_rows(P->has_s ? s.shared_width : 0);
+  D->tile_rows_r = decode_pick_tile_rows(P->has_r ? s.m : 0);
+  for (int r = 0; r < 2 && ok; ++r) {
     const cuuint64_t dims[3] = {d, rows_w, 2};
     const cuuint64_t str[2] = {d * 2, rows_w * d * 2};
-    const cuuint32_t box[3] = {kUmmaBK, 128, 2};
-    ok = umma_encode(P, &D->w_gu, buf.w_gate_up, 3, dims, str, box, "gate/up weights (decode)");
+    const cuuint32_t box[3] = {kUmmaBK, (cuuint32_t)(r ? D->tile_rows_r : D->tile_rows_s), 2};
+    ok = umma_encode(P, r ? &D->w_gu_r : &D->w_gu, buf.w_gate_up, 3, dims, str, box, "gate/up weights (decode)");
   }
   if (ok && P->has_s) {
     const cuuint64_t dims[3] = {(cuuint64_t)s.shared_width, d, (cuuint64_t)s.n_outer};
@@ -646,11 +668,11 @@ inline bool decode_plan_attach_fp8(UmmaPlan* P, DecodePlan* D, const DecodeFp8Bu
     return true;
   };
   bool ok = true;
-  {
+  for (int r = 0; r < 2 && ok; ++r) {
     const cuuint64_t dims[3] = {d, rows_w, 2};
     const cuuint64_t str[2] = {d, rows_w * d};
-    const cuuint32_t box[3] = {2 * kUmmaBK, 128, 2};
-    ok = encode8(&D->w_gu8, f.w_gu8, 3, dims, str, box, "FP8 gate/up weights");
+    const cuuint32_t box[3] = {2 * kUmmaBK, (cuuint32_t)(r ? D->tile_rows_r : D->tile_rows_s), 2};
+    ok = encode8(r ? &D->w_gu8_r : &D->w_gu8, f.w_gu8, 3, dims, str, box, "FP8 gate/up weights");
   }
   if (ok) ok = encode_planes(D->xq_map, f.xq, f.xq_rows, d, "E4M3 planes of x");
   if (ok && P->has_s) {
@@ -722,7 +744,8 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n
   };
   const int kb_d = (s.d + bk - 1) / bk, kb_s = (s.shared_width + bk - 1) / bk, kb_m = (s.m + bk - 1) / bk;
   const bool wide = n_rows > kDecMaxRows;
-  const bool split1 = !wide && splits((act_s * ((s.shared_width + 127) / 128) + act_r * ((s.m + 127) / 128)) * kb_d, kb_d);
+  const int trs = D->tile_rows_s, trr = D->tile_rows_r;
+  const bool split1 = !wide && splits((act_s * ((s.shared_width + trs - 1) / trs) + act_r * ((s.m + trr - 1) / trr)) * kb_d, kb_d);
   const bool split2 = !wide && splits((long long)((s.d + 127) / 128) * (act_s * kb_s + act_r * kb_m),
                              (act_s && kb_s > kb_m) || !act_r ? kb_s : kb_m);
   DecodeArgs a{};
@@ -732,17 +755,18 @@ inline int decode_forward(UmmaPlan* P, DecodePlan* D, const GroupRows* gr, int n
   const int bi = decode_box_index(n_rows);
   a.tok_box_rows = 16 << bi;
   // plain layer: group 0 is the shared expert and its rows are the whole batch, known here
-  a.early_units = (s.n_outer == 1 && P->has_s) ? (s.shared_width + 127) / 128 : 0;
+  a.tile_rows_s = trs; a.tile_rows_r = trr;
+  a.early_units = (s.n_outer == 1 && P->has_s) ? (s.shared_width + trs - 1) / trs : 0;
   a.n_rows_plain = n_rows;
   a.scale_gu = D->scale_gu; a.scale_d = D->scale_d; a.rows_w = (long long)s.n_outer * s.d_ff;
   a.out_s = (bf16*)P->buf.h_s; a.out_r = (bf16*)P->buf.h_r; a.ld_out_s = s.shared_width; a.ld_out_r = s.m;
   int extra = 0;
   a.tok_scale_s = D->x_scale; a.tok_scale_r = D->x_scale;
   const int sms = P->n_sms;
-  if (wide) decode_launch<4, false, kDecWideRows>(dep, false, sms, st, D->w_gu, D->w_gu, D->x_rows[bi], D->x_rows[bi], a);
+  if (wide) decode_launch<4, false, kDecWideRows>(dep, false, sms, st, D->w_gu, D->w_gu_r, D->x_rows[bi], D->x_rows[bi], a);
   else if (D->fp8)          // the layer holds FP8 codes of its expert weights: stream those (half the bytes)
-    decode_launch<4, true, kDecMaxRows>(dep, split1, sms, st, D->w_gu8, D->w_gu8, D->xq_map[bi], D->xq_map[bi], a);
-  else decode_launch<4, false, kDecMaxRows>(dep, split1, sms, st, D->w_gu, D->w_gu, D->x_rows[bi], D->x_rows[bi], a);
+    decode_launch<4, true, kDecMaxRows>(dep, split1, sms, st, D->w_gu8, D->w_gu8_r, D->xq_map[bi], D->xq_map[bi], a);
+  else decode_launch<4, false, kDecMaxRows>(dep, split1, sms, st, D->w_gu, D->w_gu_r, D->x_rows[bi], D->x_rows[bi], a);
   if (mid) cudaEventRecord(mid, st);
   a.out_s = (bf16*)P->buf.y_s; a.out_r = (bf16*)P->buf.y_r; a.ld_out_s = s.d; a.ld_out_r = s.d;
   if (gate_up_only) {
