@@ -380,9 +380,6 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
     xo = (const T*)L->xo;
   }
 
-  // Weights-on-M streaming kernels: up to 64 rows; on bf16 weights (the FP8 token planes stop at 64) the wide
-  // form takes up to 128 rows, or up to 96 when 128-neuron tiles pad the expert width by more than 5 %
-  // (measured: a 448-wide expert's token-major 112-neuron tiles win from there).  Path 2 keeps token-major tiles.
   // One row of a plain layer: plain-load weight streamers on the CUDA cores, the down projection and the
   // combine in one launch (automatic path only; path 2 keeps the tensor-core kernels).
   bool gemv = false;
@@ -391,9 +388,9 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
     gemv = use_umma && !L->hier && L->gemm_path == 0 &&
            gemv_plan((int)R, L->n_outer, L->n_groups_total(), n_k, n_r, d, L->shared_width(), L->m, L->cfg.n_shared > 0,
                      L->fp8, &gemv_ring);
-  int decode_rows = kDecMaxRows;
-  if (!L->fp8 && L->gemm_path != 2)
-    decode_rows = kDecWideRows;
+  // Weights-on-M streaming kernels: up to 64 rows; on bf16 weights (the FP8 token planes stop at 64) the wide
+  // form takes up to 128 rows.  Path 2 keeps token-major tiles from 65 rows.
+  const int decode_rows = (!L->fp8 && L->gemm_path != 2) ? kDecWideRows : kDecMaxRows;
   const bool decode = use_umma && !gemv && R <= decode_rows;
   if (use_umma && !umma_bind_x(&L->umma, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
   if (decode && !decode_bind_x(&L->umma, &L->decode, xo, R)) return arg_fail(CMOE_ERR_CUDA, L->umma.error);
