@@ -257,7 +257,8 @@ void carve_workspace(cmoe_layer* L, char* base) {
     L->xo = a.take<char>(R * d * esz);
   }
   if (esz == 2) {
-    const size_t t1 = (size_t)L->n_outer * ((L->shared_width() + 127) / 128 + nr * ((L->m + 127) / 128));
+    // gate/up tiles hold 96 to 128 neurons (decode_pick_tile_rows): count them at the smallest height
+    const size_t t1 = (size_t)L->n_outer * ((L->shared_width() + 95) / 96 + nr * ((L->m + 95) / 96));
     const size_t t2 = (size_t)L->n_groups_total() * ((d + 127) / 128);
     L->n_dec_ticket = 4 * (t1 > t2 ? t1 : t2);
     L->dec_ticket = a.take<int32_t>(L->n_dec_ticket);
