@@ -185,6 +185,9 @@ SWEEP_POINTS = [("c2_llama2_7b", 1), ("c2_llama2_7b", 16), ("c2_llama2_7b", 64),
                 ("c5_skew_13b", 16384)]
 HEADLINE = SWEEP_POINTS[-1]
 SWEEP_POINTS_FP8 = [("c2_llama2_7b", 1), ("c2_llama2_7b", 16), ("c2_llama2_7b", 64), ("c3_llama3_8b", 32)]
+# between the decode and the prefill regime (not points of the metric: reported beside the sweep)
+MID_POINTS = [("c2_llama2_7b", 128), ("c2_llama2_7b", 256), ("c2_llama2_7b", 1024),
+              ("c3_llama3_8b", 128), ("c3_llama3_8b", 256), ("c3_llama3_8b", 512), ("c3_llama3_8b", 1024)]
 
 
 def traffic_note(name, tokens, use_graph):
@@ -494,6 +497,7 @@ def run_gpu(args):
 
     # ---- the other (workload, T) points
     sweep = None
+    mid = []
     do_sweep = args.sweep == "on" or (args.sweep == "auto" and world == 1 and (name, T) == HEADLINE)
     if do_sweep:
         found = {(head["workload"], head["tokens"]): head}
@@ -501,7 +505,8 @@ def run_gpu(args):
         order = [name] + [n_ for n_ in dict.fromkeys(p_[0] for p_ in SWEEP_POINTS) if n_ != name]
         for n_ in order:
             ts = [t_ for m_, t_ in SWEEP_POINTS if m_ == n_ and (m_, t_) not in found]
-            if not ts:
+            ts_mid = [t_ for m_, t_ in MID_POINTS if m_ == n_]
+            if not ts and not ts_mid:
                 continue
             if n_ != name:
                 layer.destroy()
@@ -512,6 +517,9 @@ def run_gpu(args):
                 name = n_
             for t_ in ts:
                 found[(n_, t_)], _, _ = measure_point(rig, inputs, layer, t_, args.sweep_region_s, 200, with_dense=True)
+            for t_ in ts_mid:
+                rec, _, _ = measure_point(rig, inputs, layer, t_, args.sweep_region_s / 2, 200, with_dense=True)
+                mid.append(rec)
         sweep = [found[p_] for p_ in SWEEP_POINTS if p_ in found]
         # decode points again with FP8 expert weights (quantising a layer is permanent, so these come last)
         for n_ in dict.fromkeys(p_[0] for p_ in SWEEP_POINTS_FP8):
@@ -555,6 +563,7 @@ def run_gpu(args):
     }
     if sweep is not None:
         line["sweep"] = sweep
+        line["mid_size"] = mid
     rig.close()
     return line
 
