@@ -257,13 +257,14 @@ int cmoe_cluster_representatives(const int64_t* scaled_sq_dist, const int32_t* n
  * 2 and 3 return CMOE_ERR_INVALID_ARG if the layer cannot take the tensor-core path. */
 int cmoe_layer_set_gemm_path(cmoe_layer* layer, int32_t path);
 
-/* Launch chaining (on by default): on the bf16 tensor-core path of a plain layer every kernel
- * of a forward after the router is launched as a programmatic dependent of its predecessor,
- * so it may become resident (and fetch what does not depend on the predecessor) while the
+/* Launch chaining (on by default): on the bf16 tensor-core path every kernel of a forward
+ * after the expert router is launched as a programmatic dependent of its predecessor, so it
+ * may become resident (and fetch what does not depend on the predecessor) while the
  * predecessor drains, and waits on the device before touching anything the predecessor
  * produces.  Results are bit-identical either way; 0 restores ordinary stream-ordered
- * launches.  Has no effect on fp32 layers, hierarchical layers, CTA pairs, or while per-stage
- * timing is enabled (those always use ordinary launches).  Error: INVALID_ARG (null layer). */
+ * launches.  Has no effect on fp32 layers or while per-stage timing is enabled, and the
+ * prologue of a hierarchical layer (top-level router, its permutation, the row copy) always
+ * uses ordinary launches.  Error: INVALID_ARG (null layer). */
 int cmoe_layer_set_launch_chaining(cmoe_layer* layer, int32_t on);
 
 /* Sizes a caller needs to read the routing state back.  n_outer / outer_top_k

@@ -357,10 +357,11 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
   cudaEvent_t* ev = (L->ev_ring && !gate_up_only) ? &L->ev[(size_t)(L->ev_count % L->ev_ring) * (CMOE_N_STAGES + 1)] : nullptr;
   auto mark = [&](int i) { if (ev) cudaEventRecord(ev[i], st); };
   mark(0);
-  // Plain bf16 layers on the tensor path chain their kernels by programmatic dependent launch
-  // (every kernel after the router may become resident early and waits on the device for its
-  // predecessor); per-stage events, the hierarchical prologue and CTA pairs use ordinary launches.
-  const bool dep = use_umma && !L->hier && !ev && L->chain_launches;
+  // bf16 layers on the tensor path chain their kernels by programmatic dependent launch (every
+  // kernel after the expert router may become resident early and waits on the device for its
+  // predecessor); per-stage events and the prologue of a hierarchical layer (outer router, outer
+  // permutation, row copy) use ordinary launches.
+  const bool dep = use_umma && !ev && L->chain_launches;
 
   if (L->hier) {
     if constexpr (std::is_same<T, bf16>::value) {

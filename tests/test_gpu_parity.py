@@ -273,6 +273,25 @@ def test_launch_chaining_is_bit_identical():
     layer.destroy()
 
 
+def test_launch_chaining_hierarchical_is_bit_identical():
+    """The same for a layer under a top-level router (Section 4.4): the kernels after the expert router are chained."""
+    import torch
+    inp = _inputs("c4_hier_8x7b", d_model=256, tokens=(300,), m=224)
+    inners = [parity.gpu_layer(lay, 8) for lay in inp.layers]
+    layer = binding.Layer.create_hier(parity.to_device(inp.w_router, "bf16"), inners, 2, 300)
+    x = parity.to_device(inp.x, "bf16")
+    for t in (3, 20, 50, 100, 300):
+        layer.set_launch_chaining(False)
+        ref = layer.forward(x[:t]).clone()
+        layer.set_launch_chaining(True)
+        for _ in range(3):
+            got = layer.forward(x[:t]).clone()
+            torch.cuda.synchronize()
+            assert layer.status() == 0
+            assert torch.equal(got.view(torch.int16), ref.view(torch.int16)), t
+    layer.destroy()
+
+
 @pytest.mark.parametrize("n_rows,n_k,n_groups", [(1, 2, 6), (255, 2, 6), (256, 4, 28), (257, 4, 28),
                                                  (5000, 2, 56), (16384, 4, 14), (3000, 8, 1000),
                                                  (700, 1, 3), (40, 0, 5)])
