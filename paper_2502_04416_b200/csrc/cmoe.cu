@@ -239,7 +239,7 @@ void carve_workspace(cmoe_layer* L, char* base) {
   L->rsk_ticket = a.take<int32_t>(kRskMaxChunks + 1);
   L->share = a.take<float>(G ? G : 1);
   L->target = a.take<float>(G ? G : 1);
-  L->rsk_part = a.take<float>((size_t)kRskMaxChunks * kRskMaxSlices * kRskMaxRows * 64);
+  L->rsk_part = a.take<float>((size_t)kRskMaxTotalRows * kRskMaxSlices * 64);
   L->x_perm = a.take<char>(P * d * esz);
   L->h_s = a.take<char>(R * L->shared_width() * esz);
   L->h_r = a.take<char>(P * L->m * esz);
@@ -411,16 +411,16 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
                                                  L->b, ooff, L->n_outer, L->scores, L->keys,      \
                                                  L->topk_idx, L->topk_gate)
     if constexpr (std::is_same<T, bf16>::value) {
-      if (use_umma && R > kRskMaxRows * kRskMaxChunks) {
+      if (use_umma && R > kRskMaxTotalRows) {
         if (umma_router_forward(&L->umma, R, ooff, L->err_word, st) < 0)
           return arg_fail(CMOE_ERR_CUDA, L->umma.error);
-      } else if (R <= kRskMaxRows * kRskMaxChunks && d <= kRskMaxSlices * kRskSliceK) {
-        // Row chunks, the grid's second dimension: 64 rows, or 16 for at most 64 rows of a router with more than
-        // 8 columns, whose gate logic takes a warp per row (measured: 8B-shaped layer at 32 rows 97.9 -> 95.0 us;
-        // with up to 8 columns the four-rows-per-warp form on one 64-row chunk is 1 us faster).  The last
-        // chunk's block also permutes batches of up to 128 rows (7B-shaped layer at 128 rows 91.0 -> 88.9 us;
-        // at 256 rows the permutation kernels are as fast).
-        const int chunk_rows = (R <= kRskMaxRows && n_r > 8) ? 16 : kRskMaxRows;
+      } else if (R <= kRskMaxTotalRows && d <= kRskMaxSlices * kRskSliceK) {
+        // Row chunks, the grid's second dimension: 16 rows for a router with more than 8 columns, whose gate
+        // logic takes a warp per row (measured: 8B-shaped layer at 32 rows 97.9 -> 95.0 us, at 128 rows
+        // 118.9 -> 108.7 us); 64 rows with up to 8 columns, where the four-rows-per-warp form on 64-row chunks
+        // is 1 us faster.  The last chunk's block also permutes batches of up to 128 rows (7B-shaped layer at
+        // 128 rows 91.0 -> 88.9 us; at 256 rows the permutation kernels are as fast).
+        const int chunk_rows = n_r > 8 ? 16 : kRskMaxRows;
         const int chunks = (R + chunk_rows - 1) / chunk_rows;
         perm_fused = G <= kRskFuseGroups && R <= 2 * kRskMaxRows && (long long)R * n_k <= 4096;
         const bool sub8 = n_r <= 8 && R > 16;                        // pays when a chunk's last block has more than 16 rows

@@ -189,12 +189,14 @@ namespace cmoe {
 // groups the same block goes on to the histogram / scan / permutation of the selections
 // (and the groups' row ranges), which saves two launches per decode step.
 // Larger batches run the same kernel on a two-dimensional grid: block (s, c) owns k slice s of row chunk c
-// (chunk_rows = 16 for up to 64 rows, so that the chunks' reductions and gate logic run on different SMs;
-// 64 for up to kRskMaxChunks * 64 rows), and each chunk has its own scratch and ticket.  The chunks' last
+// (chunk_rows = 16, so that the chunks' reductions and gate logic run on many SMs, or 64 for routers of at
+// most 8 columns, whose gate logic runs four rows per warp; kRskMaxTotalRows rows at most), and each chunk
+// has its own scratch and ticket.  The chunks' last
 // blocks take a second ticket, and the block that takes the last of those permutes the whole batch (up to
 // kPermChunk rows; beyond that the permutation is left to the permutation kernels).
 constexpr int kRskMaxRows = 64;
-constexpr int kRskMaxChunks = 8;
+constexpr int kRskMaxChunks = 32;
+constexpr int kRskMaxTotalRows = 512;       // rows of a batch this kernel takes (scratch: a [slices][64] block per row)
 constexpr int kRskSliceK = 128;
 constexpr int kRskMaxSlices = 64;           // d <= 8192
 constexpr int kRskThreads = 256;
@@ -207,7 +209,7 @@ __global__ void __launch_bounds__(kRskThreads)
 router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, int n_rp, int n_k,
                      const bf16* __restrict__ w_rep, const float* __restrict__ u, const float* __restrict__ b,
                      const int32_t* __restrict__ outer_off, int n_outer,
-                     float* __restrict__ part /*[chunks][slices][kRskMaxRows][64]*/,
+                     float* __restrict__ part /*[chunks][slices][chunk_rows][64]*/,
                      int32_t* __restrict__ ticket /*[kRskMaxChunks + 1], zero between launches*/, int chunk_rows,
                      float* __restrict__ scores, float* __restrict__ keys,
                      int32_t* topk_idx, float* __restrict__ topk_gate,
@@ -225,7 +227,7 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
   xo += (size_t)row_base * d;
   scores += (size_t)row_base * n_r; keys += (size_t)row_base * n_r;
   topk_idx += (size_t)row_base * n_k; topk_gate += (size_t)row_base * n_k;
-  part += (size_t)blockIdx.y * gridDim.x * kRskMaxRows * 64;
+  part += (size_t)blockIdx.y * gridDim.x * chunk_rows * 64;
   ticket += blockIdx.y;
   __shared__ __align__(16) float unit[8][16][kRmStride];       // [unit = half*m_tiles + m-tile][row in tile][n]
   __shared__ int row_group[kRskMaxRows];
@@ -277,7 +279,7 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
   }
   __syncthreads();
   // slice partial = first half + second half
-  float* mine = part + (size_t)blockIdx.x * kRskMaxRows * 64;
+  float* mine = part + (size_t)blockIdx.x * chunk_rows * 64;
   for (int i = threadIdx.x; i < n_rows * n2; i += kRskThreads) {
     const int r = i / n2, n = i - r * n2;
     const int mt = r >> 4, rr = r & 15;
@@ -294,7 +296,7 @@ router_splitk_kernel(const bf16* __restrict__ xo, int n_rows, int d, int n_r, in
   float (*total)[kRmStride] = reinterpret_cast<float (*)[kRmStride]>(&unit[0][0][0]);   // [64][72]
   const int n_slices = (int)gridDim.x;
   const int n4 = n2 >> 2;                          // n2 is a multiple of 8: whole float4 groups
-  constexpr size_t kSliceStride4 = (size_t)kRskMaxRows * 64 / 4;
+  const size_t kSliceStride4 = (size_t)chunk_rows * 64 / 4;
   for (int i = threadIdx.x; i < n_rows * n4; i += kRskThreads) {
     const int r = i / n4, n = (i - r * n4) * 4;
     const float4* ps = reinterpret_cast<const float4*>(part + (size_t)r * 64 + n);
