@@ -137,6 +137,8 @@ def test_degenerate_structures(path):
         layer = parity.gpu_layer(lay, 70)
         layer.set_gemm_path(path)
         st = parity.check_plain_layer(layer, lay, inp.x)
+        parity.check_plain_layer(layer, lay, inp.x[:1])       # one row: the CUDA-core path on the automatic choice
+        parity.check_plain_layer(layer, lay, inp.x[5:6])
         if top_k == shape.n_routed:           # every expert on with unit gates: the dense FFN
             import torch
             got = parity.to_host(layer.forward(parity.to_device(inp.x, "bf16")))
