@@ -154,7 +154,7 @@ __device__ __forceinline__ void gemv_list_groups(const GemvArgs& p, GemvGroups<T
 constexpr int kGemvEarly = 3;              // shared-expert neurons a warp may finish before the router has
 
 template <int TT, bool FP8>
-__global__ void __launch_bounds__(kGemvThreads, 2)
+__global__ void __launch_bounds__(kGemvThreads, 4)
 gemv_gate_up_kernel(const GemvArgs p) {
   __shared__ GemvGroups<TT> L;
   grid_dep_trigger();
@@ -169,7 +169,7 @@ gemv_gate_up_kernel(const GemvArgs p) {
     float ag[TT], au[TT];
 #pragma unroll
     for (int j = 0; j < TT; ++j) { ag[j] = 0.0f; au[j] = 0.0f; }
-#pragma unroll 8
+#pragma unroll 4
     for (int c = lane; c < chunks; c += 32) {
       GemvChunk<FP8> cg, cu;
       cg.load(wg, c);
@@ -338,7 +338,7 @@ inline bool gemv_plan(int n_rows, int n_outer, int n_groups, int n_k, int n_r, i
 inline int gemv_forward(const GemvArgs& a, const GemvPlan& plan, bool fp8, int n_sms, cudaStream_t st, cudaEvent_t mid,
                         bool dep, bool gate_up_only) {
   const dim3 block(kGemvThreads);
-  const dim3 grid1(2 * n_sms);
+  const dim3 grid1(4 * n_sms);
   // down + combine: a warp takes kGemvCH channels per pass; as many passes as four blocks per SM need, evenly filled
   const int warps = 4 * n_sms * kGemvWarps, pairs = a.d / kGemvCH;
   const int passes = (pairs + warps - 1) / warps;
