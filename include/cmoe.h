@@ -249,8 +249,8 @@ int cmoe_cluster_representatives(const int64_t* scaled_sq_dist, const int32_t* n
  * rows each of the two GEMMs may run on CTA pairs: below 1024 rows because a pair fetches a third
  * less operand data per SM, from 1024 rows when the padding of the expert groups to 256-row
  * tiles is expected to stay small; batches of 65 to 128 rows stream the bf16 weights through the
- * decode-shaped kernels, weights on the MMA's M side; a single row of a plain layer up to 4096
- * wide runs on the CUDA cores with plain-load weight streams, down projection and combine in one
+ * decode-shaped kernels, weights on the MMA's M side; a single row of a plain layer
+ * runs on the CUDA cores with plain-load weight streams, down projection and combine in one
  * launch), 1 = always SIMT, 2 = tensor-core with
  * single-CTA token-major tiles only (decode-shaped kernels up to 64 rows), 3 = tensor-core on CTA
  * pairs (cta_group::2) for batches of at least 256 rows;

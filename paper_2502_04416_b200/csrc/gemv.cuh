@@ -17,8 +17,8 @@
 // sums by the per-row power-of-two scales; the token rows stay bf16.
 // The kernels are written for TT rows and instantiated for one: measured on 7B-, 8B- and 13B-shaped
 // layers, two rows already run faster on the tensor-core streamers (61 vs 64, 55 vs 60, 64 vs 80 us),
-// and so does one row of a 5120-wide model with FP8 weights (48 vs 53 us; bf16 weights: even), so
-// the path takes one row of models up to 4096 wide (44.6 vs 54.3 and 39.1 vs 45.3 us per forward).
+// one row is faster here (40.4 vs 54.3, 37.8 vs 45.3, 50.7 vs 59.6 us per forward; with FP8 weights
+// 35.0 vs 43.2, 35.0 vs 43.2, 45.6 vs 48.1).
 #pragma once
 
 #include "common.cuh"
@@ -27,7 +27,6 @@
 namespace cmoe {
 
 constexpr int kGemvMaxRows = 1;
-constexpr int kGemvMaxWidth = 4096;        // d_model
 constexpr int kGemvThreads = 256;
 constexpr int kGemvWarps = kGemvThreads / 32;
 constexpr int kGemvMaxGroups = 64;         // group tables in shared memory
@@ -326,7 +325,6 @@ struct GemvPlan { int unused; };
 inline bool gemv_plan(int n_rows, int n_outer, int n_groups, int n_k, int n_r, int d, int shared_width, int m, bool has_s,
                       bool fp8, GemvPlan* out) {
   if (n_rows < 1 || n_rows > kGemvMaxRows || n_outer != 1 || n_groups > kGemvMaxGroups || n_k > 16) return false;
-  if (d > kGemvMaxWidth) return false;
   const int align = fp8 ? 16 : 8;                  // 16-byte (8-byte: codes) chunks of 8 weights, rows aligned to them
   if (d % align || shared_width % align || m % align || d % kGemvCH) return false;
   (void)n_r; (void)has_s;
