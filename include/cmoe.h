@@ -246,9 +246,9 @@ int cmoe_cluster_representatives(const int64_t* scaled_sq_dist, const int32_t* n
 
 /* Choose the expert-GEMM implementation: 0 = automatic (tensor-core path when the
  * dtype is bf16 and the shape allows, else the plain SIMT path; for batches of at least 256
- * rows each of the two GEMMs may run on CTA pairs: below 1024 rows because a pair fetches a third
- * less operand data per SM, from 1024 rows when the padding of the expert groups to 256-row
- * tiles is expected to stay small; batches of 65 to 128 rows stream the bf16 weights through the
+ * rows each of the two GEMMs may run on CTA pairs: below 1024 rows when the experts are at least
+ * 1024 neurons wide (a pair fetches a third less operand data per SM), from 1024 rows when the
+ * padding of the expert groups to 256-row tiles is expected to stay small; batches of 65 to 128 rows stream the bf16 weights through the
  * decode-shaped kernels, weights on the MMA's M side; a single row of a plain layer
  * runs on the CUDA cores with plain-load weight streams, down projection and combine in one
  * launch), 1 = always SIMT, 2 = tensor-core with

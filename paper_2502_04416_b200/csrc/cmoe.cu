@@ -470,8 +470,12 @@ int forward_impl(cmoe_layer* L, const T* x, int n_tok, T* out, cudaStream_t st, 
       const double rows_s = (double)R / L->n_outer, rows_r = G > 0 ? (double)P / G : 0.0;
       const double w_s = (double)R * L->cfg.n_shared, w_r = (double)P;
       const double ratio = (w_s + w_r) > 0 ? (pad(rows_s) * w_s + pad(rows_r) * w_r) / (w_s + w_r) : 1.0;
-      if (R < 1024 && !L->hier) {          // a few tiles per SM: operand fetch per SM is the limit, not padded MMA work
-        pair_mask = 1 | (L->m >= 512 ? 2 : 0);
+      if (R < 1024 && !L->hier) {
+        // A few tiles per SM: operand fetch per SM is the limit, and a pair halves the weight bytes a CTA fetches,
+        // but every routed group is padded to 256 rows.  Measured at 256-768 rows: pairs win with wide experts
+        // (1376 neurons: 114 vs 126 us at 256 rows, 120 vs 127 at 512), single-CTA tiles with narrow ones (864:
+        // 134 vs 162 us at 256 rows, 165 vs 174 at 384; 448: 113 vs 127 at 256, 151 vs 167 at 768).
+        pair_mask = L->m >= 1024 ? 3 : 0;
       } else {
         if (ratio <= 1.03) pair_mask |= 1;
         if (ratio <= 1.08 && L->m >= 512) pair_mask |= 2;
